@@ -1,0 +1,269 @@
+#!/usr/bin/env python
+"""Benchmark of the transposable N:M mask search.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one pass of the approximate 2:4 search (Algorithm 1 + completion, packed mask, masked
+weights and objective in one fused pass) over the 12288 x 49152 bf16 matrix whose entries are N(0, 0.02)
+quantised to 256 levels (ties in nearly every block).  Prints ONE JSON line.
+
+`--impl reference` times the CPU oracle as it stands on a bounded sample of the same matrix.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import workloads  # noqa: E402
+
+FULL_ROWS, COLS = 12288, 49152
+ROWS = FULL_ROWS
+N_KEEP, M_BLOCK = 2, 4
+BYTES_PER_WEIGHT = 2 + 2 + 1.0 / 8          # read W, write masked W, write one mask bit (bf16)
+METRIC = "transposable-mask weights/s (2:4 approx, bf16, 1 GPU: achieved HBM GB/s vs peak in `roofline`)"
+WORKLOAD = "%dx49152 bf16, N(0,0.02) quantised to 256 levels (frequent ties), 2:4 approximate, per-step recompute"
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def time_oracle(W: np.ndarray, rows: int, threads: int):
+    from oracle import tm_oracle as orc
+    sample = np.ascontiguousarray(W[:rows])
+    t0 = time.perf_counter()
+    orc.find_mask(sample, N_KEEP, M_BLOCK, orc.APPROX, threads=threads)
+    dt = time.perf_counter() - t0
+    return sample.size / dt, dt
+
+
+def run_reference(args):
+    """The CPU oracle on a bounded row-strip sample per step (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import tm_oracle as orc
+    orc.build()
+    rows = 192
+    W = workloads.quantised_bf16(rows, COLS, 0.02, 5)
+    for _ in range(args.warmup):
+        orc.find_mask(W, N_KEEP, M_BLOCK, orc.APPROX, threads=1)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.find_mask(W, N_KEEP, M_BLOCK, orc.APPROX, threads=1)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = W.size / dt
+    sample = "first %d rows of the %dx%d matrix per step (%d weights), single thread" % (rows, FULL_ROWS, COLS, W.size)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "weights/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic", "config": {"workload": WORKLOAD % FULL_ROWS, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "weights/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "weights/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2102_08124_b200 as tm
+    from paper_2102_08124_b200 import build as tm_build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        tm_build.build()
+    if world > 1:
+        dist.barrier()
+    tm.load_library()
+
+    # every rank searches its own matrix (blocks are independent: no exchange on the data path)
+    ROWS = args.rows
+    Wh = workloads.quantised_bf16(ROWS, COLS, 0.02, 5 + rank)
+    W = torch.from_numpy(Wh.view(np.int16)).cuda().view(torch.bfloat16)
+    mask = torch.empty((ROWS, tm.tm_mask_words_per_row(COLS)), dtype=torch.int32, device="cuda")
+    masked = torch.empty_like(W)
+    obj = torch.zeros((1,), dtype=torch.float64, device="cuda")
+
+    def step():
+        tm.tm_find_mask_bf16(W, N_KEEP, M_BLOCK, tm.TM_APPROX, mask_out=mask, masked_w_out=masked, objective_out=obj)
+
+    def sync():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # warm-up: at least W steps and long enough for the clock sampler (started first) to see the GPU under load
+    sampler = ClockSampler(local_rank)
+    if rank == 0 and not args.skip_clocks:
+        sampler.start()
+    warm, t_warm = 0, time.perf_counter()
+    while warm < max(args.warmup, 3) or (not args.skip_clocks and time.perf_counter() - t_warm < 0.6):
+        step()
+        warm += 1
+        if warm % 8 == 0:
+            torch.cuda.synchronize()
+    sync()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync()
+    start.record()
+    for _ in range(args.steps):
+        step()
+    end.record()
+    sync()
+    ms = start.elapsed_time(end) / args.steps
+    clocks = sampler.stop() if (rank == 0 and not args.skip_clocks) else None
+    status = tm.tm_device_status()
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+
+    # end to end through the host-buffer entry point: pinned host input, results read back every step
+    e2e = None
+    if not args.skip_e2e:
+        Wp = torch.from_numpy(Wh.view(np.int16)).view(torch.bfloat16).pin_memory()
+        mask_h = torch.empty((ROWS, tm.tm_mask_words_per_row(COLS)), dtype=torch.int32).pin_memory()
+        masked_h = torch.empty_like(Wp).pin_memory()
+        e2e_steps = max(2, min(args.steps, 5))
+        for _ in range(2):
+            tm.tm_find_mask_host(Wp, N_KEEP, M_BLOCK, tm.TM_APPROX, mask_out=mask_h, masked_w_out=masked_h)
+        sync()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            _, _, obj_e2e, st_e2e = tm.tm_find_mask_host(Wp, N_KEEP, M_BLOCK, tm.TM_APPROX, mask_out=mask_h, masked_w_out=masked_h)
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / e2e_steps
+        te = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e_s = float(te.item())
+        e2e = {"value": world * ROWS * COLS / e2e_s, "unit": "weights/s", "h2d_bytes_per_step": int(Wp.numel() * 2),
+               "d2h_bytes_per_step": int(masked_h.numel() * 2 + mask_h.numel() * 4 + 8), "ms_per_step": e2e_s * 1e3,
+               "objective": obj_e2e, "status": st_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    weights = ROWS * COLS
+    peak, peak_src = measured_peak()
+    achieved = weights * BYTES_PER_WEIGHT / (ms * 1e-3) / 1e9
+    cpu_rows = min(768, ROWS)
+    cpu_value, cpu_dt = (None, 0.0) if args.skip_cpu else time_oracle(Wh, cpu_rows, 1)
+    line = {
+        "metric": METRIC, "value": world * weights / (ms_max * 1e-3), "unit": "weights/s", "n_gpus": world, "steps": args.steps,
+        "warmup": warm, "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD % ROWS, "N": N_KEEP, "M": M_BLOCK, "method": "approx", "outputs": "mask+masked_w+objective",
+                   "l2": "inputs (1.2 GB) larger than L2 (126 MB)", "device_status": status,
+                   "objective": float(obj.item())},
+        "e2e": e2e,
+        "gpu_launches": 2 * args.steps,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_source": peak_src, "algorithmic_bytes_per_launch": weights * BYTES_PER_WEIGHT,
+                     "frac_of_8000": achieved / 8000.0,
+                     "note": "duration = CUDA-event time of one step (search kernel + its tiny partial-zeroing and reduction launches)"},
+        "cpu_baseline": {"value": cpu_value, "unit": "weights/s", "cores": 1, "kind": "oracle",
+                         "sample": "first %d rows of the matrix (%d weights), %.1f s" % (cpu_rows, cpu_rows * COLS, cpu_dt)},
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="tm", choices=["tm", "reference"])
+    # profiling aids (ncu captures want a smaller case and none of the side measurements)
+    ap.add_argument("--rows", type=int, default=ROWS, help="rows of the matrix (default: the full workload)")
+    ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
+    ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    ap.add_argument("--skip-clocks", action="store_true", help="no nvidia-smi sampling and no extended warm-up")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,151 @@
+/*
+ * tm.h -- C ABI of the transposable N:M mask search for NVIDIA B200 (sm_100a).
+ *
+ * Method: "Accelerated Sparse Neural Training: A Provable and Efficient Method to Find N:M
+ * Transposable Masks" (arXiv 2102.08124), Section 4 "Computing transposable sparsity masks".
+ *
+ * The operation (Section 4, "Problem formulation", Eq. 1).  A weight matrix W[rows, cols] is tiled
+ * into independent M x M blocks anchored at element (0,0).  For every block the search returns a
+ * 0/1 mask S with exactly N ones in each block row and each block column -- so that W and its
+ * transpose obey the same N:M pattern -- chosen to maximise sum_ij S_ij |W_ij|.
+ *
+ *   method TM_EXACT         the optimum of Eq. 1 (the paper reaches it through the min-cost flow of
+ *                           Fig. 3; for M = 4 it is also reached by enumerating all 90 patterns).
+ *   method TM_APPROX        Algorithm 1 (greedy 2-approximation) followed by a deterministic
+ *                           completion to exactly N kept entries per line.  Algorithm 1 alone yields a
+ *                           cover that may prune more than M-N entries of a line; the paper does not
+ *                           say how to finish it, the completion is this library's:
+ *                             B. visit the pruned entries heavy -> light, keep an entry again when
+ *                                its row and its column both hold fewer than N kept entries;
+ *                             C. while a row is short: take the lightest kept entry (r', c') for
+ *                                which a short row r with (r, c') free and a short column c with
+ *                                (r', c) free exist, un-keep it, keep the heaviest such (r, c') and
+ *                                the heaviest such (r', c).
+ *   method TM_APPROX_COVER  Algorithm 1 only: at most N kept entries per line (the object the
+ *                           paper's Lemma, W(P) <= 2 W*, speaks about).
+ *
+ * Conventions the paper leaves open
+ *   - N counts KEPT entries per block row / column (Eq. 1).  Supported (N, M): (2, 4) and (4, 8).
+ *   - Order of magnitudes: by the bit pattern of |w| (sign cleared, so -0 == +0), ties broken by the
+ *     row-major position p = i*M + j inside the block; the earlier position is the lighter one.
+ *     Algorithm 1's degree test is read as "fewer than M-N pruned edges at the node".
+ *   - TM_EXACT compares candidate masks by (exact sum of kept |w|, code(S) = sum_p S_p 2^p),
+ *     larger wins; the sum is carried in integer arithmetic, never rounded.
+ *
+ * Layouts
+ *   W, masked_w_out   row-major, leading dimension ld (elements; ld == cols in the plain calls),
+ *                     fp32 or bf16.  rows and cols must be multiples of M (callers zero-pad).
+ *   mask_out          rows * tm_mask_words_per_row(cols) 32-bit words; the bit of element (r, c) is
+ *                     bit c % 32 of word r * wpr + c / 32; padding bits of the last word are 0.
+ *   masked_w_out      kept entries copied bit for bit, pruned entries +0.  May be NULL (mask only)
+ *                     or equal to W (in place).
+ *   objective_out     one double: sum over the whole matrix of kept |w| (fp32 adds per thread,
+ *                     fp64 across threads and CTAs in a fixed order: same input -> same bits).
+ *                     May be NULL.
+ *
+ * Ownership and execution.  Unless a function says otherwise every data pointer is a DEVICE
+ * pointer owned by the caller, calls are asynchronous on the stated stream, and nothing is
+ * synchronised.  Host-detectable errors are returned (nothing is launched); conditions only the
+ * device can see are OR-ed into a device status word (TM_DEV_* bits) that the caller reads after
+ * its own synchronisation -- the outputs are fully written and deterministic even then.
+ * There is no CPU fallback: without a CUDA device every compute entry point returns TM_ERR_CUDA.
+ */
+#ifndef TM_H_
+#define TM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TM_VERSION 100
+
+/* method */
+#define TM_EXACT 0
+#define TM_APPROX 1
+#define TM_APPROX_COVER 2
+
+/* dtype */
+#define TM_F32 0
+#define TM_BF16 1
+
+/* return codes (host-detected) */
+#define TM_OK 0
+#define TM_ERR_NULL 1       /* a required pointer is NULL */
+#define TM_ERR_SHAPE 2      /* negative size, rows or cols not a multiple of M, ld < cols, count < 0 */
+#define TM_ERR_NM 3         /* (N, M) is not (2, 4) or (4, 8) */
+#define TM_ERR_METHOD 4
+#define TM_ERR_DTYPE 5
+#define TM_ERR_ALIGN 6      /* W / masked_w_out row starts not aligned to one block row (M elements), mask_out not to 4 bytes */
+#define TM_ERR_CUDA 7       /* a CUDA runtime call failed (no device, launch error, allocation failure) */
+#define TM_ERR_WORKSPACE 8  /* workspace NULL, misaligned (256 bytes) or smaller than tm_workspace_bytes() */
+
+/* device status bits */
+#define TM_DEV_NONFINITE 1  /* an Inf or NaN was met in W (it is ordered by its bit pattern) */
+#define TM_DEV_INTERNAL 2   /* an iteration cap was hit (cannot happen; outputs fall back to a valid mask) */
+
+typedef struct tm_problem {
+    const void* W;          /* device, dtype, rows x ld */
+    int64_t rows, cols, ld; /* ld in elements */
+    int32_t dtype;          /* TM_F32 or TM_BF16 */
+    uint32_t* mask_out;     /* device, rows * wpr words, required */
+    void* masked_w_out;     /* device, same dtype/ld as W; NULL or == W allowed */
+    double* objective_out;  /* device, one double; may be NULL */
+} tm_problem;
+
+/* Number of 32-bit mask words per matrix row, ceil(cols / 32), and for the whole matrix. */
+size_t tm_mask_words_per_row(int64_t cols);
+size_t tm_mask_words(int64_t rows, int64_t cols);
+
+/*
+ * tm_find_mask / tm_find_mask_bf16 -- Section 4, Eq. 1 (TM_EXACT), Algorithm 1 (TM_APPROX*).
+ * One matrix, fp32 resp. bf16, ld == cols, on the legacy default stream (stream 0) of the current
+ * device.  All pointers are device pointers.  The first call on a device allocates a small scratch
+ * buffer (objective partials and a status word) that the library keeps until the process exits;
+ * tm_find_mask_batched() never allocates.  Device status bits of these calls accumulate in that
+ * scratch and are fetched with tm_device_status().
+ */
+int tm_find_mask(const void* W, int64_t rows, int64_t cols, int N, int M, int method,
+                 uint32_t* mask_out, void* masked_w_out, double* objective_out);
+int tm_find_mask_bf16(const void* W, int64_t rows, int64_t cols, int N, int M, int method,
+                      uint32_t* mask_out, void* masked_w_out, double* objective_out);
+
+/* Synchronises stream 0 of the current device, returns the OR of the TM_DEV_* bits raised by the
+ * plain calls since the last query in *status_host (host pointer) and clears them. */
+int tm_device_status(int* status_host);
+
+/*
+ * tm_find_mask_batched -- the same search for `count` matrices (a whole model) in one launch:
+ * the from-scratch setting of Section 4.1 re-derives every layer's mask periodically.
+ * probs_host: HOST array of descriptors (copied during the call; may be freed on return).
+ * workspace_dev: device scratch of at least tm_workspace_bytes(...) bytes, 256-byte aligned, owned
+ * by the caller, reusable across calls on the same stream (calls on different streams need
+ * different workspaces).  status_dev: device int, OR-ed with TM_DEV_* bits; may be NULL.
+ * cuda_stream: a cudaStream_t (NULL = legacy default stream).  Never allocates, never synchronises.
+ * All matrices share N, M and method; dtypes may differ.
+ */
+int tm_find_mask_batched(const tm_problem* probs_host, int count, int N, int M, int method,
+                         void* workspace_dev, size_t workspace_bytes, int* status_dev, void* cuda_stream);
+size_t tm_workspace_bytes(const tm_problem* probs_host, int count);
+
+/*
+ * tm_find_mask_host -- the search on HOST buffers (Eq. 1 / Algorithm 1 as above): copies W to the
+ * current device in row strips, runs the kernels and copies mask, masked weights and objective back,
+ * overlapping the three on separate streams; returns when the outputs are in host memory.
+ * Pinned host buffers make the copies asynchronous; pageable ones work but serialise.
+ * masked_w_out_host and objective_out_host may be NULL.  *status_out_host (may be NULL) receives
+ * the TM_DEV_* bits.  Allocates device staging buffers on first use and keeps them.
+ */
+int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols, int N, int M, int method,
+                      uint32_t* mask_out_host, void* masked_w_out_host, double* objective_out_host,
+                      int* status_out_host);
+
+const char* tm_status_string(int code);
+int tm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TM_H_ */

@@ -1,0 +1,12 @@
+"""Transposable N:M mask search on NVIDIA B200: Python binding of the C-ABI CUDA library.
+
+The binding only marshals arguments (torch tensors -> device pointers); every step of the search
+runs in the CUDA kernels of ``libtm.so``.  There is no CPU fallback: a missing library or a missing
+CUDA device raises.
+"""
+from .binding import (  # noqa: F401
+    TM_APPROX, TM_APPROX_COVER, TM_BF16, TM_DEV_INTERNAL, TM_DEV_NONFINITE, TM_EXACT, TM_F32,
+    TmError, library_path, load_library, tm_device_status, tm_find_mask, tm_find_mask_batched,
+    tm_find_mask_bf16, tm_find_mask_host, tm_mask_words, tm_mask_words_per_row, tm_status_string,
+    tm_version, tm_workspace_bytes,
+)

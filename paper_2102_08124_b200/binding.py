@@ -1,0 +1,210 @@
+"""ctypes binding of libtm.so: same entry points as include/tm.h, tensors in, tensors out.
+
+Argument marshalling only.  torch is used for device memory and streams."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+TM_EXACT, TM_APPROX, TM_APPROX_COVER = 0, 1, 2
+TM_F32, TM_BF16 = 0, 1
+TM_DEV_NONFINITE, TM_DEV_INTERNAL = 1, 2
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libtm.so")
+_lib = None
+
+
+class TmError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__("tm error %d: %s" % (code, what))
+        self.code = code
+
+
+class tm_problem(ctypes.Structure):
+    _fields_ = [("W", ctypes.c_void_p), ("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("ld", ctypes.c_int64),
+                ("dtype", ctypes.c_int32), ("mask_out", ctypes.c_void_p), ("masked_w_out", ctypes.c_void_p),
+                ("objective_out", ctypes.c_void_p)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Loads libtm.so (built in-tree by ``python -m paper_2102_08124_b200.build``).  Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise TmError(-1, "libtm.so is not built; run `python -m paper_2102_08124_b200.build` (there is no CPU fallback)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
+    lib.tm_mask_words_per_row.argtypes = [i64]; lib.tm_mask_words_per_row.restype = sz
+    lib.tm_mask_words.argtypes = [i64, i64]; lib.tm_mask_words.restype = sz
+    for f in (lib.tm_find_mask, lib.tm_find_mask_bf16):
+        f.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp, vp]; f.restype = i32
+    lib.tm_device_status.argtypes = [ctypes.POINTER(i32)]; lib.tm_device_status.restype = i32
+    lib.tm_find_mask_batched.argtypes = [ctypes.POINTER(tm_problem), i32, i32, i32, i32, vp, sz, vp, vp]
+    lib.tm_find_mask_batched.restype = i32
+    lib.tm_workspace_bytes.argtypes = [ctypes.POINTER(tm_problem), i32]; lib.tm_workspace_bytes.restype = sz
+    lib.tm_find_mask_host.argtypes = [vp, i32, i64, i64, i32, i32, i32, vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
+    lib.tm_find_mask_host.restype = i32
+    lib.tm_status_string.argtypes = [i32]; lib.tm_status_string.restype = ctypes.c_char_p
+    lib.tm_version.restype = i32
+    _lib = lib
+    return lib
+
+
+def tm_status_string(code: int) -> str:
+    return load_library().tm_status_string(code).decode()
+
+
+def tm_version() -> int:
+    return int(load_library().tm_version())
+
+
+def tm_mask_words_per_row(cols: int) -> int:
+    return int(load_library().tm_mask_words_per_row(cols))
+
+
+def tm_mask_words(rows: int, cols: int) -> int:
+    return int(load_library().tm_mask_words(rows, cols))
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise TmError(rc, tm_status_string(rc))
+
+
+def _dtype_code(t) -> int:
+    import torch
+    if t.dtype == torch.float32:
+        return TM_F32
+    if t.dtype == torch.bfloat16:
+        return TM_BF16
+    raise TmError(5, "W must be float32 or bfloat16")
+
+
+def _outputs(W, mask_out, masked_w_out, objective_out, want_masked, want_objective):
+    import torch
+    rows, cols = W.shape
+    if mask_out is None:
+        mask_out = torch.empty((rows, tm_mask_words_per_row(cols)), dtype=torch.int32, device=W.device)
+    if masked_w_out is None and want_masked:
+        masked_w_out = torch.empty_like(W)
+    if objective_out is None and want_objective:
+        objective_out = torch.empty((1,), dtype=torch.float64, device=W.device)
+    return mask_out, masked_w_out, objective_out
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _plain(fn_name, W, N, M, method, mask_out, masked_w_out, objective_out, want_masked, want_objective):
+    import torch
+    lib = load_library()
+    if not (W.is_cuda and W.dim() == 2 and W.is_contiguous()):
+        raise TmError(2, "W must be a contiguous 2-D CUDA tensor")
+    mask_out, masked_w_out, objective_out = _outputs(W, mask_out, masked_w_out, objective_out, want_masked, want_objective)
+    with torch.cuda.device(W.device):
+        _check(getattr(lib, fn_name)(_ptr(W), W.shape[0], W.shape[1], N, M, method, _ptr(mask_out), _ptr(masked_w_out), _ptr(objective_out)))
+    return mask_out, masked_w_out, objective_out
+
+
+def tm_find_mask(W, N: int, M: int, method: int, mask_out=None, masked_w_out=None, objective_out=None,
+                 want_masked: bool = True, want_objective: bool = True):
+    """fp32 matrix on the legacy default stream.  Returns (mask int32[rows, wpr], masked W or None, objective[1] or None)."""
+    import torch
+    if W.dtype != torch.float32:
+        raise TmError(5, "tm_find_mask takes float32; use tm_find_mask_bf16 for bfloat16")
+    return _plain("tm_find_mask", W, N, M, method, mask_out, masked_w_out, objective_out, want_masked, want_objective)
+
+
+def tm_find_mask_bf16(W, N: int, M: int, method: int, mask_out=None, masked_w_out=None, objective_out=None,
+                      want_masked: bool = True, want_objective: bool = True):
+    import torch
+    if W.dtype != torch.bfloat16:
+        raise TmError(5, "tm_find_mask_bf16 takes bfloat16")
+    return _plain("tm_find_mask_bf16", W, N, M, method, mask_out, masked_w_out, objective_out, want_masked, want_objective)
+
+
+def tm_device_status() -> int:
+    s = ctypes.c_int(0)
+    _check(load_library().tm_device_status(ctypes.byref(s)))
+    return s.value
+
+
+def _problem_array(Ws: Sequence, masks, maskeds, objectives):
+    arr = (tm_problem * max(len(Ws), 1))()
+    for k, W in enumerate(Ws):
+        arr[k].W = W.data_ptr(); arr[k].rows = W.shape[0]; arr[k].cols = W.shape[1]; arr[k].ld = W.stride(0) if W.shape[0] > 1 else W.shape[1]
+        arr[k].dtype = _dtype_code(W)
+        arr[k].mask_out = masks[k].data_ptr()
+        arr[k].masked_w_out = maskeds[k].data_ptr() if maskeds is not None and maskeds[k] is not None else None
+        arr[k].objective_out = objectives[k:k + 1].data_ptr() if objectives is not None else None
+    return arr
+
+
+def tm_workspace_bytes(count: int) -> int:
+    return int(load_library().tm_workspace_bytes(None, count))
+
+
+def tm_find_mask_batched(Ws: Sequence, N: int, M: int, method: int, masks=None, maskeds=None, objectives=None,
+                         workspace=None, status=None, stream=None, want_masked: bool = True):
+    """One launch for a list of 2-D CUDA tensors (fp32 and/or bf16; rows may be strided, stride(1) == 1).
+
+    Returns (masks, maskeds, objectives float64[count], status int32[1], workspace uint8[...]).  Runs on
+    `stream` (a torch.cuda.Stream) or on torch's current stream; nothing is synchronised."""
+    import torch
+    lib = load_library()
+    if len(Ws) == 0:
+        return [], [], None, status, workspace
+    dev = Ws[0].device
+    for W in Ws:
+        if not (W.is_cuda and W.dim() == 2 and (W.shape[1] <= 1 or W.stride(1) == 1) and W.device == dev):
+            raise TmError(2, "every W must be a 2-D CUDA tensor with unit column stride on one device")
+    if masks is None:
+        masks = [torch.empty((W.shape[0], tm_mask_words_per_row(W.shape[1])), dtype=torch.int32, device=dev) for W in Ws]
+    if maskeds is None and want_masked:
+        maskeds = [torch.empty_strided(W.shape, W.stride(), dtype=W.dtype, device=dev) for W in Ws]
+    if maskeds is not None:
+        for W, Y in zip(Ws, maskeds):                      # the ABI has one leading dimension per matrix
+            if Y is not None and (Y.shape != W.shape or Y.stride() != W.stride() or Y.dtype != W.dtype):
+                raise TmError(2, "masked_w_out must have the shape, strides and dtype of W")
+    if objectives is None:
+        objectives = torch.empty((len(Ws),), dtype=torch.float64, device=dev)
+    if status is None:
+        status = torch.zeros((1,), dtype=torch.int32, device=dev)
+    need = tm_workspace_bytes(len(Ws))
+    if workspace is None:
+        workspace = torch.empty((need,), dtype=torch.uint8, device=dev)
+    arr = _problem_array(Ws, masks, maskeds, objectives)
+    with torch.cuda.device(dev):
+        s = stream if stream is not None else torch.cuda.current_stream(dev)
+        _check(lib.tm_find_mask_batched(arr, len(Ws), N, M, method, _ptr(workspace), workspace.numel(), _ptr(status),
+                                        ctypes.c_void_p(s.cuda_stream)))
+    return masks, maskeds, objectives, status, workspace
+
+
+def tm_find_mask_host(W, N: int, M: int, method: int, mask_out=None, masked_w_out=None, want_masked: bool = True,
+                      device: Optional[int] = None):
+    """Host tensors in, host tensors out (pinned memory lets the copies overlap the kernels).
+
+    W: 2-D contiguous CPU tensor, float32 or bfloat16.  Returns (mask, masked or None, objective float, status int)."""
+    import torch
+    lib = load_library()
+    if W.is_cuda or W.dim() != 2 or not W.is_contiguous():
+        raise TmError(2, "W must be a contiguous 2-D CPU tensor")
+    rows, cols = W.shape
+    if mask_out is None:
+        mask_out = torch.empty((rows, tm_mask_words_per_row(cols)), dtype=torch.int32).pin_memory()
+    if masked_w_out is None and want_masked:
+        masked_w_out = torch.empty_like(W).pin_memory()
+    obj = ctypes.c_double(0.0); st = ctypes.c_int(0)
+    with torch.cuda.device(device if device is not None else torch.cuda.current_device()):
+        _check(lib.tm_find_mask_host(_ptr(W), _dtype_code(W), rows, cols, N, M, method, _ptr(mask_out), _ptr(masked_w_out),
+                                     ctypes.byref(obj), ctypes.byref(st)))
+    return mask_out, masked_w_out, obj.value, st.value

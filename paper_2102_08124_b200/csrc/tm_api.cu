@@ -1,0 +1,303 @@
+// C ABI of the transposable N:M mask search (see include/tm.h): argument validation, work
+// partitioning and kernel dispatch.  Nothing here computes masks on the host.
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "../../include/tm.h"
+#include "tm_launch.h"
+
+namespace {
+
+using tmask::DevProblem;
+
+constexpr int kMaxCtas = 1024;        // upper bound used to size workspaces (grid = min(4 * SMs, kMaxCtas))
+constexpr int kMaxDevices = 64;
+constexpr size_t kAlign = 256;
+constexpr size_t kHeaderBytes = 256;  // reserved head of every workspace
+
+size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+size_t table_bytes(int count) { return align_up(sizeof(DevProblem) * (size_t)(count > 0 ? count : 1)); }
+size_t partial_bytes(int count) { return align_up(sizeof(double) * (size_t)(count > 0 ? count : 1) * kMaxCtas * 8); }
+
+struct DeviceState {
+    bool ready = false;
+    int sms = 0;
+    void* scratch = nullptr;          // workspace of the plain calls: [status | table | partials]
+    size_t scratch_bytes = 0;
+    // staging of tm_find_mask_host
+    void* stage_w = nullptr; void* stage_masked = nullptr; void* stage_mask = nullptr; void* stage_ws = nullptr; double* stage_obj = nullptr;
+    size_t stage_w_bytes = 0, stage_masked_bytes = 0, stage_mask_bytes = 0, stage_ws_bytes = 0;
+    cudaStream_t s_in = nullptr, s_run = nullptr, s_out = nullptr;
+};
+DeviceState g_dev[kMaxDevices];
+std::mutex g_mutex;
+
+int current_device(DeviceState** st) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return TM_ERR_CUDA; }
+    DeviceState& d = g_dev[dev];
+    if (!d.ready) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!d.ready) {
+            if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+            d.ready = true;
+        }
+    }
+    *st = &d;
+    return TM_OK;
+}
+
+int check_nm(int N, int M) { return ((N == 2 && M == 4) || (N == 4 && M == 8)) ? TM_OK : TM_ERR_NM; }
+int check_method(int m) { return (m == TM_EXACT || m == TM_APPROX || m == TM_APPROX_COVER) ? TM_OK : TM_ERR_METHOD; }
+
+int check_problem(const tm_problem& p, int M) {
+    if (p.dtype != TM_F32 && p.dtype != TM_BF16) return TM_ERR_DTYPE;
+    if (p.rows < 0 || p.cols < 0 || p.rows % M || p.cols % M || p.ld < p.cols) return TM_ERR_SHAPE;
+    if (p.rows == 0 || p.cols == 0) return TM_OK;
+    if (!p.W || !p.mask_out) return TM_ERR_NULL;
+    const size_t elem = p.dtype == TM_F32 ? 4 : 2;
+    const size_t vec = (size_t)M * elem < 16 ? (size_t)M * elem : 16;    // width of the vector accesses
+    if ((uintptr_t)p.W % vec || ((size_t)p.ld * elem) % vec) return TM_ERR_ALIGN;
+    if (p.masked_w_out && (uintptr_t)p.masked_w_out % vec) return TM_ERR_ALIGN;
+    if ((uintptr_t)p.mask_out % 4 || (p.objective_out && (uintptr_t)p.objective_out % 8)) return TM_ERR_ALIGN;
+    return TM_OK;
+}
+
+DevProblem to_dev(const tm_problem& p, int M, long long item_begin) {
+    DevProblem d;
+    d.W = p.W; d.mask = p.mask_out; d.masked = p.masked_w_out; d.objective = p.objective_out;
+    d.rows = p.rows; d.cols = p.cols; d.ld = p.ld; d.item_begin = item_begin; d.dtype = p.dtype;
+    d.wpr = (int)((p.cols + 31) / 32);
+    d.bcols = (int)(p.cols / M);
+    d.chunks = (d.bcols + 31) / 32;
+    return d;
+}
+
+long long items_of(const DevProblem& d, int M) { return (d.rows / M) * (long long)d.chunks; }
+
+// Validates, builds the descriptor table in the workspace and launches.  ws layout: [header | table | partials].
+int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes, int* status_dev,
+        cudaStream_t stream, const DeviceState& dev) {
+    int rc;
+    if ((rc = check_nm(N, M)) != TM_OK) return rc;
+    if ((rc = check_method(method)) != TM_OK) return rc;
+    if (count < 0) return TM_ERR_SHAPE;
+    if (count == 0) return TM_OK;
+    if (!probs) return TM_ERR_NULL;
+    for (int k = 0; k < count; ++k)
+        if ((rc = check_problem(probs[k], M)) != TM_OK) return rc;
+    if (!ws || (uintptr_t)ws % kAlign || ws_bytes < tm_workspace_bytes(probs, count)) return TM_ERR_WORKSPACE;
+
+    std::vector<DevProblem> table((size_t)count);
+    long long total = 0;
+    for (int k = 0; k < count; ++k) { table[k] = to_dev(probs[k], M, total); total += items_of(table[k], M); }
+
+    tmask::LaunchArgs a;
+    a.count = count; a.total_items = total; a.N = N; a.M = M; a.method = method; a.stream = stream; a.status = status_dev;
+    char* base = static_cast<char*>(ws);
+    a.partials = reinterpret_cast<double*>(base + kHeaderBytes + table_bytes(count));
+    const long long want = (total + tmask::generic_warps_per_cta() - 1) / tmask::generic_warps_per_cta();
+    const int cap = dev.sms * 4 < kMaxCtas ? dev.sms * 4 : kMaxCtas;
+    a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));
+    a.single = table[0];
+    if (count == 1) {
+        a.table = nullptr;
+    } else {
+        DevProblem* dtab = reinterpret_cast<DevProblem*>(base + kHeaderBytes);
+        // pageable source: the runtime stages the bytes before returning, so `table` may die here
+        if (cudaMemcpyAsync(dtab, table.data(), sizeof(DevProblem) * (size_t)count, cudaMemcpyHostToDevice, stream) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+        a.table = dtab;
+    }
+    if (tmask::launch_generic(a) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    return TM_OK;
+}
+
+int ensure_scratch(DeviceState& d) {
+    if (d.scratch) return TM_OK;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (d.scratch) return TM_OK;
+    const size_t bytes = kHeaderBytes + table_bytes(1) + partial_bytes(1);
+    void* p = nullptr;
+    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    if (cudaMemset(p, 0, kHeaderBytes) != cudaSuccess) { cudaGetLastError(); cudaFree(p); return TM_ERR_CUDA; }
+    d.scratch = p; d.scratch_bytes = bytes;
+    return TM_OK;
+}
+
+int plain_call(const void* W, int dtype, int64_t rows, int64_t cols, int N, int M, int method,
+               uint32_t* mask_out, void* masked_w_out, double* objective_out) {
+    tm_problem p;
+    p.W = W; p.rows = rows; p.cols = cols; p.ld = cols; p.dtype = dtype;
+    p.mask_out = mask_out; p.masked_w_out = masked_w_out; p.objective_out = objective_out;
+    // validate before touching the device
+    int rc;
+    if ((rc = check_nm(N, M)) != TM_OK) return rc;
+    if ((rc = check_method(method)) != TM_OK) return rc;
+    if ((rc = check_problem(p, M)) != TM_OK) return rc;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != TM_OK) return rc;
+    if ((rc = ensure_scratch(*d)) != TM_OK) return rc;
+    return run(&p, 1, N, M, method, d->scratch, d->scratch_bytes, static_cast<int*>(d->scratch), nullptr, *d);
+}
+
+int grow(void** p, size_t* have, size_t want) {
+    if (*have >= want) return TM_OK;
+    if (*p) cudaFree(*p);
+    *p = nullptr; *have = 0;
+    if (cudaMalloc(p, want) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    *have = want;
+    return TM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t tm_mask_words_per_row(int64_t cols) { return cols > 0 ? (size_t)((cols + 31) / 32) : 0; }
+size_t tm_mask_words(int64_t rows, int64_t cols) { return rows > 0 ? (size_t)rows * tm_mask_words_per_row(cols) : 0; }
+
+size_t tm_workspace_bytes(const tm_problem* /*probs_host*/, int count) {
+    return kHeaderBytes + table_bytes(count) + partial_bytes(count);
+}
+
+int tm_find_mask(const void* W, int64_t rows, int64_t cols, int N, int M, int method,
+                 uint32_t* mask_out, void* masked_w_out, double* objective_out) {
+    return plain_call(W, TM_F32, rows, cols, N, M, method, mask_out, masked_w_out, objective_out);
+}
+
+int tm_find_mask_bf16(const void* W, int64_t rows, int64_t cols, int N, int M, int method,
+                      uint32_t* mask_out, void* masked_w_out, double* objective_out) {
+    return plain_call(W, TM_BF16, rows, cols, N, M, method, mask_out, masked_w_out, objective_out);
+}
+
+int tm_device_status(int* status_host) {
+    if (!status_host) return TM_ERR_NULL;
+    DeviceState* d = nullptr;
+    int rc = current_device(&d);
+    if (rc != TM_OK) return rc;
+    *status_host = 0;
+    if (!d->scratch) return TM_OK;
+    if (cudaStreamSynchronize(nullptr) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    if (cudaMemcpy(status_host, d->scratch, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    if (cudaMemset(d->scratch, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    return TM_OK;
+}
+
+int tm_find_mask_batched(const tm_problem* probs_host, int count, int N, int M, int method,
+                         void* workspace_dev, size_t workspace_bytes, int* status_dev, void* cuda_stream) {
+    int rc;
+    if ((rc = check_nm(N, M)) != TM_OK) return rc;
+    if ((rc = check_method(method)) != TM_OK) return rc;
+    if (count < 0) return TM_ERR_SHAPE;
+    if (count > 0 && !probs_host) return TM_ERR_NULL;
+    for (int k = 0; k < count; ++k)
+        if ((rc = check_problem(probs_host[k], M)) != TM_OK) return rc;
+    if (count > 0 && (!workspace_dev || (uintptr_t)workspace_dev % kAlign || workspace_bytes < tm_workspace_bytes(probs_host, count)))
+        return TM_ERR_WORKSPACE;
+    if (count == 0) return TM_OK;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != TM_OK) return rc;
+    return run(probs_host, count, N, M, method, workspace_dev, workspace_bytes, status_dev, static_cast<cudaStream_t>(cuda_stream), *d);
+}
+
+int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols, int N, int M, int method,
+                      uint32_t* mask_out_host, void* masked_w_out_host, double* objective_out_host, int* status_out_host) {
+    int rc;
+    if ((rc = check_nm(N, M)) != TM_OK) return rc;
+    if ((rc = check_method(method)) != TM_OK) return rc;
+    if (dtype != TM_F32 && dtype != TM_BF16) return TM_ERR_DTYPE;
+    if (rows < 0 || cols < 0 || rows % M || cols % M) return TM_ERR_SHAPE;
+    if (status_out_host) *status_out_host = 0;
+    if (objective_out_host) *objective_out_host = 0.0;
+    if (rows == 0 || cols == 0) return TM_OK;
+    if (!W_host || !mask_out_host) return TM_ERR_NULL;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != TM_OK) return rc;
+
+    const size_t elem = dtype == TM_F32 ? 4 : 2;
+    const size_t row_bytes = (size_t)cols * elem, wpr = tm_mask_words_per_row(cols);
+    // row strips: copy-in, search and copy-out of neighbouring strips overlap on three streams
+    const int64_t brows = rows / M;
+    const int strips = (int)(brows < 16 ? brows : 16);
+    const int64_t strip_brows = (brows + strips - 1) / strips;
+    const size_t one_ws = tm_workspace_bytes(nullptr, 1);
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!d->s_in) {
+            if (cudaStreamCreateWithFlags(&d->s_in, cudaStreamNonBlocking) != cudaSuccess ||
+                cudaStreamCreateWithFlags(&d->s_run, cudaStreamNonBlocking) != cudaSuccess ||
+                cudaStreamCreateWithFlags(&d->s_out, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+        }
+        if ((rc = grow(&d->stage_w, &d->stage_w_bytes, (size_t)rows * row_bytes)) != TM_OK) return rc;
+        if (masked_w_out_host && (rc = grow(&d->stage_masked, &d->stage_masked_bytes, (size_t)rows * row_bytes)) != TM_OK) return rc;
+        if ((rc = grow(&d->stage_mask, &d->stage_mask_bytes, (size_t)rows * wpr * 4)) != TM_OK) return rc;
+        if ((rc = grow(&d->stage_ws, &d->stage_ws_bytes, (one_ws + kAlign) * 16 + kAlign)) != TM_OK) return rc;
+    }
+    char* ws = static_cast<char*>(d->stage_ws);
+    int* status_dev = reinterpret_cast<int*>(ws);                       // first 256 bytes: status + 16 objectives
+    double* obj_dev = reinterpret_cast<double*>(ws + 64);
+    if (cudaMemsetAsync(ws, 0, kAlign, d->s_run) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+
+    std::vector<cudaEvent_t> ev_in((size_t)strips), ev_run((size_t)strips);
+    bool ok = true;
+    for (int s = 0; s < strips && ok; ++s) {
+        ok &= cudaEventCreateWithFlags(&ev_in[s], cudaEventDisableTiming) == cudaSuccess;
+        ok &= cudaEventCreateWithFlags(&ev_run[s], cudaEventDisableTiming) == cudaSuccess;
+    }
+    for (int s = 0; s < strips && ok; ++s) {
+        const int64_t r0 = s * strip_brows * M;
+        int64_t r1 = (s + 1) * strip_brows * M; if (r1 > rows) r1 = rows;
+        if (r0 >= r1) { ok &= cudaEventRecord(ev_in[s], d->s_in) == cudaSuccess; ok &= cudaEventRecord(ev_run[s], d->s_run) == cudaSuccess; continue; }
+        const size_t off = (size_t)r0 * row_bytes, nbytes = (size_t)(r1 - r0) * row_bytes;
+        ok &= cudaMemcpyAsync(static_cast<char*>(d->stage_w) + off, static_cast<const char*>(W_host) + off, nbytes, cudaMemcpyHostToDevice, d->s_in) == cudaSuccess;
+        ok &= cudaEventRecord(ev_in[s], d->s_in) == cudaSuccess;
+        ok &= cudaStreamWaitEvent(d->s_run, ev_in[s], 0) == cudaSuccess;
+        tm_problem p;
+        p.W = static_cast<char*>(d->stage_w) + off; p.rows = r1 - r0; p.cols = cols; p.ld = cols; p.dtype = dtype;
+        p.mask_out = static_cast<uint32_t*>(d->stage_mask) + (size_t)r0 * wpr;
+        p.masked_w_out = masked_w_out_host ? static_cast<char*>(d->stage_masked) + off : nullptr;
+        p.objective_out = obj_dev + s;
+        rc = run(&p, 1, N, M, method, ws + kAlign + (size_t)s * (one_ws + kAlign), one_ws, status_dev, d->s_run, *d);
+        if (rc != TM_OK) { ok = false; break; }
+        ok &= cudaEventRecord(ev_run[s], d->s_run) == cudaSuccess;
+        ok &= cudaStreamWaitEvent(d->s_out, ev_run[s], 0) == cudaSuccess;
+        ok &= cudaMemcpyAsync(mask_out_host + (size_t)r0 * wpr, p.mask_out, (size_t)(r1 - r0) * wpr * 4, cudaMemcpyDeviceToHost, d->s_out) == cudaSuccess;
+        if (masked_w_out_host)
+            ok &= cudaMemcpyAsync(static_cast<char*>(masked_w_out_host) + off, p.masked_w_out, nbytes, cudaMemcpyDeviceToHost, d->s_out) == cudaSuccess;
+    }
+    double obj_host[16] = {0}; int status_host = 0;
+    if (ok) {
+        ok &= cudaStreamSynchronize(d->s_run) == cudaSuccess;
+        ok &= cudaMemcpy(obj_host, obj_dev, sizeof(double) * (size_t)strips, cudaMemcpyDeviceToHost) == cudaSuccess;
+        ok &= cudaMemcpy(&status_host, status_dev, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess;
+        ok &= cudaStreamSynchronize(d->s_out) == cudaSuccess;
+    } else {
+        cudaStreamSynchronize(d->s_in); cudaStreamSynchronize(d->s_run); cudaStreamSynchronize(d->s_out);
+    }
+    for (int s = 0; s < strips; ++s) { if (ev_in[s]) cudaEventDestroy(ev_in[s]); if (ev_run[s]) cudaEventDestroy(ev_run[s]); }
+    if (!ok) { cudaGetLastError(); return rc != TM_OK ? rc : TM_ERR_CUDA; }
+    if (objective_out_host) { double t = 0.0; for (int s = 0; s < strips; ++s) t += obj_host[s]; *objective_out_host = t; }
+    if (status_out_host) *status_out_host = status_host;
+    return TM_OK;
+}
+
+const char* tm_status_string(int code) {
+    switch (code) {
+    case TM_OK: return "ok";
+    case TM_ERR_NULL: return "a required pointer is NULL";
+    case TM_ERR_SHAPE: return "bad shape: sizes must be non-negative multiples of M and ld >= cols";
+    case TM_ERR_NM: return "unsupported (N, M): only (2, 4) and (4, 8)";
+    case TM_ERR_METHOD: return "unknown method";
+    case TM_ERR_DTYPE: return "unknown dtype";
+    case TM_ERR_ALIGN: return "misaligned pointer or row pitch";
+    case TM_ERR_CUDA: return "CUDA runtime error (no device, launch or allocation failure)";
+    case TM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    default: return "unknown status";
+    }
+}
+
+int tm_version(void) { return TM_VERSION; }
+
+}  // extern "C"

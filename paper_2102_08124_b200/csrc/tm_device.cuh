@@ -1,0 +1,34 @@
+// Shared device-side definitions of the transposable N:M mask search kernels.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace tmask {
+
+constexpr int kMethodExact = 0;
+constexpr int kMethodApprox = 1;
+constexpr int kMethodCover = 2;
+constexpr int kF32 = 0;
+constexpr int kBF16 = 1;
+constexpr int kDevNonFinite = 1;
+constexpr int kDevInternal = 2;
+
+// One matrix of a (possibly batched) call, as the kernels see it.
+struct DevProblem {
+    const void* W;
+    uint32_t* mask;
+    void* masked;        // may be null, may alias W
+    double* objective;   // may be null
+    long long rows, cols, ld;
+    long long item_begin;  // index of this problem's first work item in the call-wide numbering
+    int dtype;
+    int wpr;             // mask words per row
+    int bcols;           // blocks per block row
+    int chunks;          // work items per block row
+};
+
+// Magnitudes travel as the fp32 bit pattern of |w| (bf16 widened exactly): for finite values the
+// unsigned order of the patterns is the order of |w|, and -0 == +0.
+__device__ __forceinline__ float pattern_as_float(uint32_t u) { return __uint_as_float(u); }
+
+}  // namespace tmask

@@ -1,0 +1,221 @@
+// Generic kernels of the transposable N:M mask search: one thread per M x M block, plain vector
+// loads and stores.  They accept every supported (N, M, method, dtype, ld) and every shape; the
+// bandwidth-tuned kernels take over the cases they cover.
+//
+// Work item = 32 consecutive blocks of one block row: the lanes of a warp load M rows of 32*M
+// contiguous elements (fully coalesced), solve their blocks in registers, exchange mask bits with
+// shuffles into whole 32-bit words, and write masked weights with the same vector width.  Every warp
+// owns a contiguous range of items, so objective partials are produced in a fixed order.
+#include "tm_launch.h"
+#include "tm_solvers.cuh"
+
+namespace tmask {
+
+namespace {
+
+constexpr int kWarpsPerCta = 8;
+
+template <int M>
+__device__ __forceinline__ void load_block(const DevProblem& P, long long row0, long long col0, bool active, uint32_t (&w)[M * M]) {
+    // raw element bits, one row of the block per vector load
+    if (!active) {
+#pragma unroll
+        for (int p = 0; p < M * M; ++p) w[p] = 0;
+        return;
+    }
+    if (P.dtype == kF32) {
+        const float* base = reinterpret_cast<const float*>(P.W) + row0 * P.ld + col0;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+#pragma unroll
+            for (int v = 0; v < M / 4; ++v) {
+                const uint4 t = __ldg(reinterpret_cast<const uint4*>(base + i * P.ld) + v);
+                w[i * M + 4 * v + 0] = t.x; w[i * M + 4 * v + 1] = t.y; w[i * M + 4 * v + 2] = t.z; w[i * M + 4 * v + 3] = t.w;
+            }
+        }
+    } else {
+        const uint16_t* base = reinterpret_cast<const uint16_t*>(P.W) + row0 * P.ld + col0;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            if constexpr (M == 4) {
+                const uint2 t = __ldg(reinterpret_cast<const uint2*>(base + i * P.ld));
+                w[i * 4 + 0] = t.x << 16; w[i * 4 + 1] = t.x & 0xFFFF0000u; w[i * 4 + 2] = t.y << 16; w[i * 4 + 3] = t.y & 0xFFFF0000u;
+            } else {
+                const uint4 t = __ldg(reinterpret_cast<const uint4*>(base + i * P.ld));
+                const uint32_t r[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+                for (int v = 0; v < 4; ++v) { w[i * 8 + 2 * v] = r[v] << 16; w[i * 8 + 2 * v + 1] = r[v] & 0xFFFF0000u; }
+            }
+        }
+    }
+}
+
+// w holds fp32 patterns (bf16 widened); pruned entries are already zeroed
+template <int M>
+__device__ __forceinline__ void store_block(const DevProblem& P, long long row0, long long col0, const uint32_t (&w)[M * M]) {
+    if (P.dtype == kF32) {
+        float* base = reinterpret_cast<float*>(P.masked) + row0 * P.ld + col0;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+#pragma unroll
+            for (int v = 0; v < M / 4; ++v)
+                reinterpret_cast<uint4*>(base + i * P.ld)[v] = make_uint4(w[i * M + 4 * v], w[i * M + 4 * v + 1], w[i * M + 4 * v + 2], w[i * M + 4 * v + 3]);
+        }
+    } else {
+        uint16_t* base = reinterpret_cast<uint16_t*>(P.masked) + row0 * P.ld + col0;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            if constexpr (M == 4) {
+                *reinterpret_cast<uint2*>(base + i * P.ld) =
+                    make_uint2((w[i * 4] >> 16) | (w[i * 4 + 1] & 0xFFFF0000u), (w[i * 4 + 2] >> 16) | (w[i * 4 + 3] & 0xFFFF0000u));
+            } else {
+                uint32_t r[4];
+#pragma unroll
+                for (int v = 0; v < 4; ++v) r[v] = (w[i * 8 + 2 * v] >> 16) | (w[i * 8 + 2 * v + 1] & 0xFFFF0000u);
+                *reinterpret_cast<uint4*>(base + i * P.ld) = make_uint4(r[0], r[1], r[2], r[3]);
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ const DevProblem& find_problem(const DevProblem* table, int count, long long item, int& k) {
+    // items are numbered problem after problem; k is the caller's last position
+    while (k + 1 < count && table[k + 1].item_begin <= item) ++k;
+    return table[k];
+}
+
+template <int N, int M, int METHOD>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, int count, long long total_items,
+               double* __restrict__ partials, int* __restrict__ status_out) {
+    const int lane = threadIdx.x & 31;
+    const long long gw = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    const long long nwarps = (long long)gridDim.x * kWarpsPerCta;
+    const long long per = (total_items + nwarps - 1) / nwarps;
+    const long long begin = gw * per;
+    const long long end = min(total_items, begin + per);
+    const DevProblem* tab = table ? table : &single;
+
+    int k = 0, status = 0;
+    double acc = 0.0;
+    int acc_k = -1;
+    constexpr int kLanesPerWord = 32 / M;          // lanes whose blocks share one mask word
+    constexpr int kWordsPerItem = M;               // 32 blocks * M columns / 32 bits
+
+    for (long long item = begin; item < end; ++item) {
+        const DevProblem& P = find_problem(tab, count, item, k);
+        if (k != acc_k) {
+            if (acc_k >= 0) {
+                for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+                if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
+            }
+            acc = 0.0; acc_k = k;
+        }
+        const long long local = item - P.item_begin;
+        const long long bi = local / P.chunks;
+        const int chunk = (int)(local - bi * P.chunks);
+        const int bj = chunk * 32 + lane;
+        const bool active = bj < P.bcols;
+        const long long row0 = bi * M, col0 = (long long)bj * M;
+
+        uint32_t w[M * M], u[M * M];
+        load_block<M>(P, row0, col0, active, w);
+        bool bad = false;
+#pragma unroll
+        for (int p = 0; p < M * M; ++p) { u[p] = w[p] & 0x7FFFFFFFu; bad |= (u[p] >> 23) == 0xFFu; }
+        if (bad) status |= kDevNonFinite;
+
+        uint64_t kept;
+        if constexpr (METHOD == kMethodExact) {
+            if constexpr (M == 4) kept = exact_2_4(u);
+            else kept = exact_ssp<N, M>(u, status);
+        } else {
+            kept = cover_mask<N, M>(u);
+            if constexpr (METHOD == kMethodApprox) {
+                int rk[M], ck[M]; bool full = true;
+                line_counts<M>(kept, rk, ck);
+#pragma unroll
+                for (int i = 0; i < M; ++i) full &= rk[i] == N;
+                if (!full) kept = complete_mask<N, M>(u, kept, status);
+            }
+        }
+        if (!active) kept = 0;
+
+        // objective: fp32 adds inside the block, fp64 across blocks
+        float s = 0.f;
+#pragma unroll
+        for (int p = 0; p < M * M; ++p) s += ((kept >> p) & 1) ? pattern_as_float(u[p]) : 0.f;
+        acc += (double)s;
+
+        // masked weights
+        if (P.masked && active) {
+#pragma unroll
+            for (int p = 0; p < M * M; ++p) w[p] = ((kept >> p) & 1) ? w[p] : 0u;
+            store_block<M>(P, row0, col0, w);
+        }
+
+        // mask words: row i of the item spans kWordsPerItem words; a lane's M bits sit at M*(lane % kLanesPerWord)
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            uint32_t bits = (uint32_t)((kept >> (i * M)) & ((1u << M) - 1)) << (M * (lane % kLanesPerWord));
+#pragma unroll
+            for (int o = 1; o < kLanesPerWord; o <<= 1) bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, o);
+            const int word = chunk * kWordsPerItem + lane / kLanesPerWord;
+            if (lane % kLanesPerWord == 0 && word < P.wpr) P.mask[(row0 + i) * P.wpr + word] = bits;
+        }
+    }
+    if (acc_k >= 0) {
+        for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
+    }
+    status |= __shfl_xor_sync(0xFFFFFFFFu, status, 16);
+    status |= __shfl_xor_sync(0xFFFFFFFFu, status, 8);
+    status |= __shfl_xor_sync(0xFFFFFFFFu, status, 4);
+    status |= __shfl_xor_sync(0xFFFFFFFFu, status, 2);
+    status |= __shfl_xor_sync(0xFFFFFFFFu, status, 1);
+    if (lane == 0 && status && status_out) atomicOr(status_out, status);
+}
+
+// objective[k] = sum of the problem's partials in a fixed order (one CTA per problem)
+__global__ void __launch_bounds__(256)
+reduce_kernel(const DevProblem single, const DevProblem* __restrict__ table, const double* __restrict__ partials, long long stride) {
+    const DevProblem& P = table ? table[blockIdx.x] : single;
+    __shared__ double sm[256];
+    double s = 0.0;
+    for (long long i = threadIdx.x; i < stride; i += 256) s += partials[(long long)blockIdx.x * stride + i];
+    sm[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o; o >>= 1) {
+        if ((int)threadIdx.x < o) sm[threadIdx.x] += sm[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0 && P.objective) *P.objective = sm[0];
+}
+
+template <int N, int M>
+cudaError_t launch_nm(const LaunchArgs& a) {
+    const dim3 grid((unsigned)a.ctas), block(kWarpsPerCta * 32);
+    switch (a.method) {
+    case kMethodExact: generic_kernel<N, M, kMethodExact><<<grid, block, 0, a.stream>>>(a.single, a.table, a.count, a.total_items, a.partials, a.status); break;
+    case kMethodApprox: generic_kernel<N, M, kMethodApprox><<<grid, block, 0, a.stream>>>(a.single, a.table, a.count, a.total_items, a.partials, a.status); break;
+    default: generic_kernel<N, M, kMethodCover><<<grid, block, 0, a.stream>>>(a.single, a.table, a.count, a.total_items, a.partials, a.status); break;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int generic_warps_per_cta() { return kWarpsPerCta; }
+
+cudaError_t launch_generic(const LaunchArgs& a) {
+    cudaError_t e = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * kWarpsPerCta, a.stream);
+    if (e != cudaSuccess) return e;
+    if (a.total_items > 0) {
+        e = (a.M == 4) ? launch_nm<2, 4>(a) : launch_nm<4, 8>(a);
+        if (e != cudaSuccess) return e;
+    }
+    reduce_kernel<<<a.count, 256, 0, a.stream>>>(a.single, a.table, a.partials, (long long)a.ctas * kWarpsPerCta);
+    return cudaGetLastError();
+}
+
+}  // namespace tmask

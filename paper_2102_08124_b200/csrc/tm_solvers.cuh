@@ -1,0 +1,362 @@
+// Per-block solvers of the transposable N:M mask search, one thread per M x M block.
+//
+// Every routine takes the block as M*M magnitudes u[p] (fp32 bit pattern of |w|, p = i*M + j) and
+// returns the kept set as a bit mask (bit p = S_ij of Eq. 1).  The order of entries is (u, p):
+// among equal magnitudes the earlier position is the lighter one.
+//
+//   cover_mask      Algorithm 1 through its closed form: the pruned list is the union of the M-N
+//                   lightest entries of every row and of every column (an entry among its row's
+//                   M-N lightest meets row degree < M-N when the sorted scan reaches it; an entry in
+//                   neither set finds both degrees full).
+//   complete_mask   this library's completion: greedy fill heavy -> light, then 2-for-1 swaps.
+//   exact_2_4       the optimum of Eq. 1 for M = 4 by scoring all 90 valid patterns.
+//   exact_ssp       the optimum for any M <= 8 by successive shortest paths on the flow network of
+//                   Fig. 3 (rows supply M-N units, columns demand M-N, unit-capacity coefficient
+//                   edges; a unit on (i,j) prunes W_ij).
+//
+// Exact arithmetic.  |w_p| = sig_p * 2^(E_p - 150); with Emin the smallest exponent among the
+// block's non-zero entries, q_p = sig_p << (E_p - Emin) is an integer proportional to |w_p|.  When
+// the block's exponent spread is small the sums fit native integers; otherwise the same code runs
+// on a 384-bit integer type, so that masks are always compared as exact real numbers.
+#pragma once
+#include "tm_device.cuh"
+
+namespace tmask {
+
+// ------------------------------------------------------------------------------------------
+// order helpers
+// ------------------------------------------------------------------------------------------
+template <int M>
+__device__ __forceinline__ void line_counts(uint64_t kept, int* rk, int* ck) {
+    constexpr uint64_t rowm = (M == 8) ? 0xFFull : 0xFull;
+    constexpr uint64_t colm = (M == 8) ? 0x0101010101010101ull : 0x1111ull;
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+        rk[i] = __popcll(kept & (rowm << (i * M)));
+        ck[i] = __popcll(kept & (colm << i));
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Algorithm 1 (closed form)
+// ------------------------------------------------------------------------------------------
+template <int N, int M>
+__device__ __forceinline__ uint64_t cover_mask(const uint32_t (&u)[M * M]) {
+    // number of heavier entries in the same row / column, from each unordered pair compared once
+    unsigned char rh[M * M], ch[M * M];
+#pragma unroll
+    for (int p = 0; p < M * M; ++p) { rh[p] = 0; ch[p] = 0; }
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+#pragma unroll
+        for (int a = 0; a < M; ++a) {
+#pragma unroll
+            for (int b = a + 1; b < M; ++b) {
+                // row i: positions i*M+a < i*M+b  -> b heavier iff u_b >= u_a
+                const bool bh = u[i * M + b] >= u[i * M + a];
+                rh[i * M + a] += bh; rh[i * M + b] += !bh;
+                // column i: positions a*M+i < b*M+i
+                const bool dh = u[b * M + i] >= u[a * M + i];
+                ch[a * M + i] += dh; ch[b * M + i] += !dh;
+            }
+        }
+    }
+    uint64_t kept = 0;
+#pragma unroll
+    for (int p = 0; p < M * M; ++p)
+        if (rh[p] < N && ch[p] < N) kept |= 1ull << p;   // not among the M-N lightest of its row nor of its column
+    return kept;
+}
+
+// ------------------------------------------------------------------------------------------
+// Completion (steps B and C)
+// ------------------------------------------------------------------------------------------
+template <int N, int M>
+__device__ __noinline__ uint64_t complete_mask(const uint32_t (&u)[M * M], uint64_t kept, int& status) {
+    uint32_t ul[M * M];                       // dynamically indexed copy
+#pragma unroll
+    for (int p = 0; p < M * M; ++p) ul[p] = u[p];
+    int rk[M], ck[M];
+    // B: heaviest free entry whose row and column are both short, until none is left
+    for (int it = 0; it < M * M; ++it) {
+        line_counts<M>(kept, rk, ck);
+        int best = -1; uint32_t bu = 0;
+        for (int p = 0; p < M * M; ++p) {
+            if (((kept >> p) & 1) || rk[p / M] >= N || ck[p % M] >= N) continue;
+            if (best < 0 || ul[p] >= bu) { best = p; bu = ul[p]; }   // ascending p: ties go to the later one
+        }
+        if (best < 0) break;
+        kept |= 1ull << best;
+    }
+    // C: 2-for-1 swaps while a row is short (at most N*N/4 of them)
+    for (int it = 0; it <= (N * N) / 4; ++it) {
+        line_counts<M>(kept, rk, ck);
+        bool any_short = false;
+        for (int i = 0; i < M; ++i) any_short |= rk[i] < N;
+        if (!any_short) return kept;
+        if (it == (N * N) / 4) break;
+        int x = -1, xa = -1, xb = -1; uint32_t xu = 0;
+        for (int p = 0; p < M * M; ++p) {      // lightest eligible kept entry
+            if (!((kept >> p) & 1)) continue;
+            if (x >= 0 && ul[p] >= xu) continue;
+            const int r2 = p / M, c2 = p % M;
+            int a = -1, b = -1;
+            for (int r = 0; r < M; ++r) {
+                const int e = r * M + c2;
+                if (rk[r] < N && !((kept >> e) & 1) && (a < 0 || ul[e] >= ul[a])) a = e;
+            }
+            for (int c = 0; c < M; ++c) {
+                const int e = r2 * M + c;
+                if (ck[c] < N && !((kept >> e) & 1) && (b < 0 || ul[e] >= ul[b])) b = e;
+            }
+            if (a >= 0 && b >= 0) { x = p; xu = ul[p]; xa = a; xb = b; }
+        }
+        if (x < 0) break;
+        kept = (kept & ~(1ull << x)) | (1ull << xa) | (1ull << xb);
+    }
+    status |= kDevInternal;
+    return kept;
+}
+
+// ------------------------------------------------------------------------------------------
+// exact integer images
+// ------------------------------------------------------------------------------------------
+struct Wide {                      // 384-bit two's-complement integer, little-endian limbs
+    unsigned long long w[6];
+};
+__device__ __forceinline__ Wide wide_zero() { Wide r; for (int i = 0; i < 6; ++i) r.w[i] = 0; return r; }
+__device__ __forceinline__ Wide wide_add(const Wide& a, const Wide& b) {
+    Wide r; unsigned long long carry = 0;
+    for (int i = 0; i < 6; ++i) {
+        const unsigned long long s = a.w[i] + b.w[i];
+        const unsigned long long c1 = s < a.w[i];
+        r.w[i] = s + carry;
+        carry = c1 | (r.w[i] < s);
+    }
+    return r;
+}
+__device__ __forceinline__ Wide wide_neg(const Wide& a) {
+    Wide r; unsigned long long carry = 1;
+    for (int i = 0; i < 6; ++i) { r.w[i] = ~a.w[i] + carry; carry = (carry && r.w[i] == 0) ? 1 : 0; }
+    return r;
+}
+__device__ __forceinline__ bool wide_less(const Wide& a, const Wide& b) {   // signed a < b
+    const bool sa = a.w[5] >> 63, sb = b.w[5] >> 63;
+    if (sa != sb) return sa;
+    for (int i = 5; i >= 0; --i) if (a.w[i] != b.w[i]) return a.w[i] < b.w[i];
+    return false;
+}
+__device__ __forceinline__ Wide wide_shl(unsigned long long v, unsigned shift) {
+    Wide r = wide_zero();
+    const unsigned limb = shift >> 6, off = shift & 63;
+    r.w[limb] = v << off;
+    if (off && limb + 1 < 6) r.w[limb + 1] = v >> (64 - off);
+    return r;
+}
+
+// Uniform access to the two cost types.
+template <class T> struct CostOps;
+template <> struct CostOps<long long> {
+    static __device__ __forceinline__ long long zero() { return 0; }
+    static __device__ __forceinline__ long long add(long long a, long long b) { return a + b; }
+    static __device__ __forceinline__ bool less(long long a, long long b) { return a < b; }
+    static __device__ __forceinline__ long long image(uint32_t sig, int shift) { return (long long)sig << shift; }
+};
+template <> struct CostOps<Wide> {
+    static __device__ __forceinline__ Wide zero() { return wide_zero(); }
+    static __device__ __forceinline__ Wide add(const Wide& a, const Wide& b) { return wide_add(a, b); }
+    static __device__ __forceinline__ bool less(const Wide& a, const Wide& b) { return wide_less(a, b); }
+    static __device__ __forceinline__ Wide image(uint32_t sig, int shift) { return wide_shl(sig, (unsigned)shift); }
+};
+
+__device__ __forceinline__ void split_float(uint32_t u, uint32_t& sig, int& E) {
+    const uint32_t e = u >> 23, m = u & 0x7FFFFFu;
+    sig = e ? (m | 0x800000u) : m;
+    E = e ? (int)e : 1;
+}
+// smallest / largest exponent among the non-zero entries; returns false for an all-zero block
+template <int CNT>
+__device__ __forceinline__ bool exponent_range(const uint32_t (&u)[CNT], int& Emin, int& Emax) {
+    Emin = 1 << 20; Emax = 0;
+#pragma unroll
+    for (int p = 0; p < CNT; ++p) {
+        uint32_t sig; int E; split_float(u[p], sig, E);
+        if (sig) { Emin = min(Emin, E); Emax = max(Emax, E); }
+    }
+    return Emax != 0;
+}
+
+// ------------------------------------------------------------------------------------------
+// Exact, M = 4, N = 2: the 90 valid patterns
+// ------------------------------------------------------------------------------------------
+// A row keeps 2 of 4 columns: six choices, as nibbles in ascending value.
+struct Patterns24 {
+    unsigned char k[90][4];     // choice index of rows 0..3, patterns in ascending code order
+    int count;
+};
+constexpr unsigned char kRowChoice[6] = {0x3, 0x5, 0x6, 0x9, 0xA, 0xC};
+constexpr Patterns24 make_patterns24() {
+    Patterns24 t{};
+    int n = 0;
+    // code = row3:row2:row1:row0 nibbles, so ascending code = lexicographic in (row3, row2, row1, row0)
+    for (int k3 = 0; k3 < 6; ++k3) for (int k2 = 0; k2 < 6; ++k2) for (int k1 = 0; k1 < 6; ++k1) for (int k0 = 0; k0 < 6; ++k0) {
+        bool ok = true;
+        for (int c = 0; c < 4; ++c) {
+            const int s = ((kRowChoice[k0] >> c) & 1) + ((kRowChoice[k1] >> c) & 1) + ((kRowChoice[k2] >> c) & 1) + ((kRowChoice[k3] >> c) & 1);
+            if (s != 2) ok = false;
+        }
+        if (ok) { t.k[n][0] = (unsigned char)k0; t.k[n][1] = (unsigned char)k1; t.k[n][2] = (unsigned char)k2; t.k[n][3] = (unsigned char)k3; ++n; }
+    }
+    t.count = n;
+    return t;
+}
+constexpr Patterns24 kPatterns24 = make_patterns24();
+static_assert(kPatterns24.count == 90, "a 4x4 block has 90 masks with two ones per row and column");
+
+template <int n> struct Pattern24 {
+    static constexpr int k0 = kPatterns24.k[n][0], k1 = kPatterns24.k[n][1], k2 = kPatterns24.k[n][2], k3 = kPatterns24.k[n][3];
+    static constexpr uint32_t code = (uint32_t)kRowChoice[k0] | ((uint32_t)kRowChoice[k1] << 4) |
+                                     ((uint32_t)kRowChoice[k2] << 8) | ((uint32_t)kRowChoice[k3] << 12);
+};
+
+// patterns n, n+1, ... in ascending code order: ">=" lets the larger code win ties
+template <class T, int n>
+__device__ __forceinline__ void score_patterns24(const T (&lo)[6][6], const T (&hi)[6][6], T& best, uint32_t& best_code) {
+    if constexpr (n < 90) {
+        using P = Pattern24<n>;
+        const T s = CostOps<T>::add(lo[P::k0][P::k1], hi[P::k2][P::k3]);
+        if (n == 0 || !CostOps<T>::less(s, best)) { best = s; best_code = P::code; }
+        score_patterns24<T, n + 1>(lo, hi, best, best_code);
+    }
+}
+
+template <class T>
+__device__ __forceinline__ uint64_t exact_2_4_scored(const uint32_t (&u)[16], int Emin) {
+    using Ops = CostOps<T>;
+    // sums of the two kept entries of a row, then of two rows, then the 90 totals
+    T rs[4][6];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        T q[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t sig; int E; split_float(u[i * 4 + j], sig, E);
+            q[j] = sig ? Ops::image(sig, E - Emin) : Ops::zero();
+        }
+        // same order as kRowChoice: columns {0,1} {0,2} {1,2} {0,3} {1,3} {2,3}
+        rs[i][0] = Ops::add(q[0], q[1]); rs[i][1] = Ops::add(q[0], q[2]); rs[i][2] = Ops::add(q[1], q[2]);
+        rs[i][3] = Ops::add(q[0], q[3]); rs[i][4] = Ops::add(q[1], q[3]); rs[i][5] = Ops::add(q[2], q[3]);
+    }
+    T lo[6][6], hi[6][6];
+#pragma unroll
+    for (int a = 0; a < 6; ++a)
+#pragma unroll
+        for (int b = 0; b < 6; ++b) { lo[a][b] = Ops::add(rs[0][a], rs[1][b]); hi[a][b] = Ops::add(rs[2][a], rs[3][b]); }
+    T best = Ops::zero(); uint32_t best_code = 0;
+    score_patterns24<T, 0>(lo, hi, best, best_code);
+    return best_code;
+}
+
+__device__ __noinline__ uint64_t exact_2_4_wide(const uint32_t (&u)[16], int Emin) { return exact_2_4_scored<Wide>(u, Emin); }
+
+__device__ __forceinline__ uint64_t exact_2_4(const uint32_t (&u)[16]) {
+    int Emin, Emax;
+    if (!exponent_range<16>(u, Emin, Emax)) { Emin = 1; Emax = 1; }     // all zero: every sum is 0, the largest code wins
+    // 24 significand bits + spread + 3 bits for eight terms must stay below 2^62
+    if (Emax - Emin <= 34) return exact_2_4_scored<long long>(u, Emin);
+    return exact_2_4_wide(u, Emin);
+}
+
+// ------------------------------------------------------------------------------------------
+// Exact, any M <= 8: successive shortest paths on the network of Fig. 3
+// ------------------------------------------------------------------------------------------
+// Cost of the coefficient edge of entry p: q_p * 2^64 + 2^p (the tie rule folded into the cost:
+// minimising the pruned cost maximises (sum of kept |w|, code)).
+struct Cost128 { __int128 v; };
+template <> struct CostOps<Cost128> {
+    static __device__ __forceinline__ Cost128 zero() { return Cost128{0}; }
+    static __device__ __forceinline__ Cost128 add(Cost128 a, Cost128 b) { return Cost128{a.v + b.v}; }
+    static __device__ __forceinline__ Cost128 neg(Cost128 a) { return Cost128{-a.v}; }
+    static __device__ __forceinline__ bool less(Cost128 a, Cost128 b) { return a.v < b.v; }
+    static __device__ __forceinline__ Cost128 edge(uint32_t sig, int shift, int p) {
+        return Cost128{((__int128)((long long)sig << shift) << 64) + ((__int128)1 << p)};
+    }
+};
+struct CostWide { Wide v; };
+template <> struct CostOps<CostWide> {
+    static __device__ __forceinline__ CostWide zero() { return CostWide{wide_zero()}; }
+    static __device__ __forceinline__ CostWide add(const CostWide& a, const CostWide& b) { return CostWide{wide_add(a.v, b.v)}; }
+    static __device__ __forceinline__ CostWide neg(const CostWide& a) { return CostWide{wide_neg(a.v)}; }
+    static __device__ __forceinline__ bool less(const CostWide& a, const CostWide& b) { return wide_less(a.v, b.v); }
+    static __device__ __forceinline__ CostWide edge(uint32_t sig, int shift, int p) {
+        Wide q = wide_shl(sig, (unsigned)shift), c;
+        c.w[0] = 1ull << p;
+        for (int l = 1; l < 6; ++l) c.w[l] = q.w[l - 1];
+        return CostWide{c};
+    }
+};
+
+template <class C, int N, int M>
+__device__ __noinline__ uint64_t exact_ssp_run(const uint32_t (&u)[M * M], int Emin, int& status) {
+    using Ops = CostOps<C>;
+    C cost[M * M];
+    for (int p = 0; p < M * M; ++p) {
+        uint32_t sig; int E; split_float(u[p], sig, E);
+        cost[p] = Ops::edge(sig, sig ? E - Emin : 0, p);
+    }
+    uint64_t pruned = 0;
+    int supply[M], demand[M];
+    for (int i = 0; i < M; ++i) { supply[i] = M - N; demand[i] = M - N; }
+    for (int unit = 0; unit < M * (M - N); ++unit) {
+        // Bellman-Ford over the residual graph; nodes 0..M-1 rows, M..2M-1 columns
+        C dist[2 * M]; int pre[2 * M]; unsigned reach = 0;
+        for (int i = 0; i < M; ++i) if (supply[i] > 0) { dist[i] = Ops::zero(); pre[i] = -1; reach |= 1u << i; }
+        bool changed = true;
+        for (int round = 0; round < 2 * M + 1 && changed; ++round) {
+            changed = false;
+            for (int i = 0; i < M; ++i) {
+                if (!((reach >> i) & 1)) continue;
+                for (int j = 0; j < M; ++j) {
+                    if ((pruned >> (i * M + j)) & 1) continue;          // forward arc: prune (i,j)
+                    const C d = Ops::add(dist[i], cost[i * M + j]);
+                    if (!((reach >> (M + j)) & 1) || Ops::less(d, dist[M + j])) { dist[M + j] = d; pre[M + j] = i; reach |= 1u << (M + j); changed = true; }
+                }
+            }
+            for (int j = 0; j < M; ++j) {
+                if (!((reach >> (M + j)) & 1)) continue;
+                for (int i = 0; i < M; ++i) {
+                    if (!((pruned >> (i * M + j)) & 1)) continue;       // backward arc: un-prune (i,j)
+                    const C d = Ops::add(dist[M + j], Ops::neg(cost[i * M + j]));
+                    if (!((reach >> i) & 1) || Ops::less(d, dist[i])) { dist[i] = d; pre[i] = M + j; reach |= 1u << i; changed = true; }
+                }
+            }
+        }
+        if (changed) status |= kDevInternal;                           // a negative cycle cannot exist
+        int sink = -1;
+        for (int j = 0; j < M; ++j)
+            if (demand[j] > 0 && ((reach >> (M + j)) & 1) && (sink < 0 || Ops::less(dist[M + j], dist[M + sink]))) sink = j;
+        if (sink < 0) { status |= kDevInternal; break; }
+        int v = M + sink, steps = 0;
+        demand[sink]--;
+        while (pre[v] >= 0 && steps++ < 2 * M + 2) {                     // walk back, toggling arcs
+            const int w = pre[v];
+            if (v >= M) pruned |= 1ull << (w * M + (v - M));            // row w -> column v-M
+            else pruned &= ~(1ull << (v * M + (w - M)));                // column w-M -> row v
+            v = w;
+        }
+        if (v < M && pre[v] < 0) supply[v]--; else status |= kDevInternal;
+    }
+    const uint64_t all = (M == 8) ? ~0ull : ((1ull << (M * M)) - 1);
+    return ~pruned & all;
+}
+
+template <int N, int M>
+__device__ __forceinline__ uint64_t exact_ssp(const uint32_t (&u)[M * M], int& status) {
+    int Emin, Emax;
+    if (!exponent_range<M * M>(u, Emin, Emax)) { Emin = 1; Emax = 1; }
+    // path costs add at most M*M signed terms: 24 + spread + 6 bits must stay below 2^62
+    if (Emax - Emin <= 31) return exact_ssp_run<Cost128, N, M>(u, Emin, status);
+    return exact_ssp_run<CostWide, N, M>(u, Emin, status);
+}
+
+}  // namespace tmask

@@ -1,0 +1,180 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element, on the same
+seeded inputs.  Masks and masked weights must be bit-identical; the objective within 1e-6 relative."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2102_08124_b200 as tm
+import workloads
+from oracle import tm_oracle as orc
+from tests.gpu_util import assert_parity, gpu_find_mask, to_device, to_host_bits
+
+pytestmark = pytest.mark.gpu
+
+METHODS = [tm.TM_EXACT, tm.TM_APPROX, tm.TM_APPROX_COVER]
+
+
+@pytest.mark.parametrize("method", METHODS)
+@pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_small_ragged_shapes(N, M, method, dtype):
+    # several work items per block row, a ragged last item, a partial last mask word
+    for rows, cols, seed in [(5 * M, 70 * M, 1), (M, M, 2), (3 * M, 33 * M, 3), (2 * M, 32 * M, 4)]:
+        W = workloads.normal_f32(rows, cols, 0.02, seed)
+        if dtype == "bf16":
+            W = workloads.f32_to_bf16_bits(W)
+        assert_parity(W, N, M, method)
+
+
+@pytest.mark.parametrize("method", METHODS)
+def test_config1(method):
+    assert_parity(workloads.config1()[0], 2, 4, method)
+
+
+@pytest.mark.parametrize("method", METHODS)
+@pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
+def test_ties_everywhere(N, M, method):
+    rng = np.random.Generator(np.random.PCG64(7))
+    W = rng.integers(-2, 3, size=(8 * M, 48 * M)).astype(np.float32)
+    assert_parity(W, N, M, method)
+    assert_parity(workloads.f32_to_bf16_bits(W), N, M, method)
+    assert_parity(workloads.quantised_bf16(8 * M, 64 * M, 0.02, 5), N, M, method)
+
+
+@pytest.mark.parametrize("method", METHODS)
+@pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
+def test_adversarial_blocks(N, M, method):
+    blocks = workloads.adversarial_blocks_f32(M)                       # [n, M, M]
+    W = np.ascontiguousarray(blocks.transpose(1, 0, 2).reshape(M, -1))
+    assert_parity(W, N, M, method)
+    assert_parity(np.zeros((2 * M, 40 * M), np.float32), N, M, method)
+    assert_parity(np.full((2 * M, 40 * M), -1.5, np.float32), N, M, method)
+
+
+@pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
+def test_extreme_exponent_spread_uses_exact_sums(N, M):
+    rng = np.random.Generator(np.random.PCG64(9))
+    W = np.ldexp(rng.standard_normal((4 * M, 40 * M)), rng.integers(-125, 120, size=(4 * M, 40 * M))).astype(np.float32)
+    W[::3, ::5] = (rng.integers(0, 50, size=W[::3, ::5].shape).astype(np.uint32)).view(np.float32)   # subnormals
+    assert_parity(W, N, M, tm.TM_EXACT)
+
+
+def test_near_tie_block_needs_exact_sums():
+    B, u = np.float32(2.0 ** 40), np.float32(2.0 ** -23)
+    blk = np.array([[B, 0, 0, 0], [0, B, 0, 0], [B, 0, np.float32(1.0) + u, 1], [0, B, 1, 1]], np.float32)
+    W = np.tile(blk, (3, 50))
+    assert_parity(W, 2, 4, tm.TM_EXACT)
+
+
+@pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
+def test_nonfinite_inputs_raise_the_status_bit(N, M):
+    W = workloads.normal_f32(2 * M, 40 * M, 0.02, 11)
+    W[1, 3] = np.inf; W[M + 1, 7 * M] = np.nan; W[0, 39 * M + 1] = -np.inf
+    for method in METHODS:
+        assert_parity(W, N, M, method, rel=None)                        # outputs follow the bit-pattern order; the sum is Inf/NaN
+
+
+@pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
+def test_optional_outputs_and_in_place(N, M):
+    W = workloads.normal_f32(4 * M, 45 * M, 0.02, 13)
+    want = orc.find_mask(W, N, M, orc.APPROX)
+    got = gpu_find_mask(W, N, M, tm.TM_APPROX, want_masked=False, want_objective=False)
+    assert got["masked"] is None and got["objective"] is None and np.array_equal(got["mask"], want["mask"])
+    Wd = to_device(W)
+    mask, masked, obj = tm.tm_find_mask(Wd, N, M, tm.TM_APPROX, masked_w_out=Wd)      # in place
+    torch.cuda.synchronize()
+    assert masked.data_ptr() == Wd.data_ptr()
+    assert np.array_equal(to_host_bits(Wd), want["masked"].view(np.uint32))
+    assert np.array_equal(to_host_bits(mask), want["mask"])
+
+
+def test_empty_matrices():
+    for rows, cols in [(0, 64), (64, 0), (0, 0)]:
+        W = torch.empty((rows, cols), device="cuda")
+        mask, masked, obj = tm.tm_find_mask(W, 2, 4, tm.TM_APPROX)
+        torch.cuda.synchronize()
+        assert float(obj.item()) == 0.0 and mask.numel() == rows * ((cols + 31) // 32)
+
+
+def test_same_input_same_bits():
+    W = workloads.normal_f32(512, 1024, 0.02, 17)
+    a = gpu_find_mask(W, 2, 4, tm.TM_APPROX); b = gpu_find_mask(W, 2, 4, tm.TM_APPROX)
+    assert np.array_equal(a["mask"], b["mask"]) and np.array_equal(a["masked"], b["masked"])
+    assert a["objective"] == b["objective"]                              # fixed-order reduction
+
+
+def _batched_parity(mats, N, M, method, strided=False):
+    Ws = []
+    for m in mats:
+        d = to_device(m)
+        if strided:                                                      # rows embedded in a wider buffer
+            wide = torch.zeros((d.shape[0], d.shape[1] + 16), dtype=d.dtype, device="cuda")
+            wide[:, : d.shape[1]] = d
+            d = wide[:, : d.shape[1]]
+        Ws.append(d)
+    masks, maskeds, objs, status, ws = tm.tm_find_mask_batched(Ws, N, M, method)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for k, m in enumerate(mats):
+        want = orc.find_mask(m, N, M, method, threads=orc.max_threads())
+        assert np.array_equal(to_host_bits(masks[k]), want["mask"]), k
+        wmasked = want["masked"].view(np.uint16 if m.dtype == np.uint16 else np.uint32)
+        assert np.array_equal(to_host_bits(maskeds[k].contiguous()), wmasked), k
+        assert abs(float(objs[k].item()) - want["objective"]) <= 1e-6 * want["objective"] + 1e-300, k
+
+
+@pytest.mark.parametrize("method", [tm.TM_APPROX, tm.TM_EXACT])
+def test_batched_mixed_dtypes_and_strides(method):
+    mats = [workloads.normal_f32(16, 148, 0.1, 21), workloads.normal_bf16(64, 264, 0.02, 22),
+            workloads.normal_f32(4, 4, 1.0, 23), workloads.normal_bf16(8, 4096, 0.02, 24), np.zeros((0, 64), np.float32)]
+    _batched_parity(mats[:4], 2, 4, method)
+    _batched_parity(mats[:4], 2, 4, method, strided=True)
+
+
+def test_batched_4_8():
+    mats = [workloads.laplace_f32(32, 264, 0.05, 31), workloads.normal_bf16(16, 520, 0.02, 32)]
+    for method in METHODS:
+        _batched_parity(mats, 4, 8, method)
+
+
+def test_config2_whole_model_approx():
+    _batched_parity(workloads.config2(), 2, 4, tm.TM_APPROX)
+
+
+def test_config2_whole_model_exact_sampled_layers():
+    mats = workloads.config2()
+    Ws = [to_device(m) for m in mats]
+    masks, maskeds, objs, status, ws = tm.tm_find_mask_batched(Ws, 2, 4, tm.TM_EXACT)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for k in (0, 1, 5, 12, 53):                                           # stem (zero-padded), small, mid, fc
+        m = mats[k]
+        rows = min(m.shape[0], 128)
+        want = orc.find_mask(np.ascontiguousarray(m[:rows]), 2, 4, orc.EXACT, threads=orc.max_threads())
+        assert np.array_equal(to_host_bits(masks[k])[:rows], want["mask"]), k
+    for k, m in enumerate(mats):                                           # properties that hold at any size
+        bits = orc.unpack_mask(to_host_bits(masks[k]), m.shape[1])
+        r, c = m.shape
+        assert (bits.reshape(r // 4, 4, c // 4, 4).sum(axis=1) == 2).all() and (bits.reshape(r // 4, 4, c // 4, 4).sum(axis=3) == 2).all()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_host_buffer_entry_point(dtype):
+    W = workloads.normal_f32(72, 520, 0.02, 41)
+    if dtype == "bf16":
+        Wb = workloads.f32_to_bf16_bits(W)
+        Wt = torch.from_numpy(Wb.view(np.int16)).view(torch.bfloat16).pin_memory()
+        ref = Wb
+    else:
+        Wt = torch.from_numpy(W).pin_memory(); ref = W
+    for (N, M) in [(2, 4), (4, 8)]:
+        for method in METHODS:
+            want = orc.find_mask(ref, N, M, method)
+            mask, masked, obj, status = tm.tm_find_mask_host(Wt, N, M, method)
+            assert status == 0
+            assert np.array_equal(mask.numpy().view(np.uint32), want["mask"])
+            got_masked = masked.view(torch.int16).numpy().view(np.uint16) if dtype == "bf16" else masked.numpy().view(np.uint32)
+            assert np.array_equal(got_masked, want["masked"].view(got_masked.dtype))
+            assert abs(obj - want["objective"]) <= 1e-6 * want["objective"]
