@@ -12,14 +12,16 @@ namespace {
 
 using tmask::DevProblem;
 
-constexpr int kMaxCtas = 1024;        // upper bound used to size workspaces (grid = min(4 * SMs, kMaxCtas))
+constexpr int kPartialSlots = 8192;   // objective partials per matrix: (CTAs x warps) of any kernel stays below this
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
 constexpr size_t kHeaderBytes = 256;  // reserved head of every workspace
 
 size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
-size_t table_bytes(int count) { return align_up(sizeof(DevProblem) * (size_t)(count > 0 ? count : 1)); }
-size_t partial_bytes(int count) { return align_up(sizeof(double) * (size_t)(count > 0 ? count : 1) * kMaxCtas * 8); }
+int at_least_one(int count) { return count > 0 ? count : 1; }
+size_t table_bytes(int count) { return align_up(sizeof(DevProblem) * (size_t)at_least_one(count)); }
+size_t entry_bytes(int count) { return align_up(tmask::tma_entry_bytes() * (size_t)at_least_one(count)); }
+size_t partial_bytes(int count) { return align_up(sizeof(double) * (size_t)at_least_one(count) * kPartialSlots); }
 
 struct DeviceState {
     bool ready = false;
@@ -77,7 +79,8 @@ DevProblem to_dev(const tm_problem& p, int M, long long item_begin) {
 
 long long items_of(const DevProblem& d, int M) { return (d.rows / M) * (long long)d.chunks; }
 
-// Validates, builds the descriptor table in the workspace and launches.  ws layout: [header | table | partials].
+// Validates, partitions the problems between the bandwidth path and the generic path, builds the
+// descriptor tables in the workspace and launches.  ws layout: [header | table | tma records | partials].
 int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes, int* status_dev,
         cudaStream_t stream, const DeviceState& dev) {
     int rc;
@@ -90,27 +93,63 @@ int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, 
         if ((rc = check_problem(probs[k], M)) != TM_OK) return rc;
     if (!ws || (uintptr_t)ws % kAlign || ws_bytes < tm_workspace_bytes(probs, count)) return TM_ERR_WORKSPACE;
 
-    std::vector<DevProblem> table((size_t)count);
-    long long total = 0;
-    for (int k = 0; k < count; ++k) { table[k] = to_dev(probs[k], M, total); total += items_of(table[k], M); }
-
-    tmask::LaunchArgs a;
-    a.count = count; a.total_items = total; a.N = N; a.M = M; a.method = method; a.stream = stream; a.status = status_dev;
     char* base = static_cast<char*>(ws);
-    a.partials = reinterpret_cast<double*>(base + kHeaderBytes + table_bytes(count));
-    const long long want = (total + tmask::generic_warps_per_cta() - 1) / tmask::generic_warps_per_cta();
-    const int cap = dev.sms * 4 < kMaxCtas ? dev.sms * 4 : kMaxCtas;
-    a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));
-    a.single = table[0];
-    if (count == 1) {
-        a.table = nullptr;
-    } else {
-        DevProblem* dtab = reinterpret_cast<DevProblem*>(base + kHeaderBytes);
-        // pageable source: the runtime stages the bytes before returning, so `table` may die here
-        if (cudaMemcpyAsync(dtab, table.data(), sizeof(DevProblem) * (size_t)count, cudaMemcpyHostToDevice, stream) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
-        a.table = dtab;
+    DevProblem* dtab = reinterpret_cast<DevProblem*>(base + kHeaderBytes);
+    char* dent = base + kHeaderBytes + table_bytes(count);
+    double* dpart = reinterpret_cast<double*>(dent + entry_bytes(count));
+
+    // group 0: generic; groups 1..4: bandwidth path by (dtype, masked output present)
+    std::vector<DevProblem> group[5];
+    for (int k = 0; k < count; ++k) {
+        DevProblem d = to_dev(probs[k], M, 0);
+        const int g = tmask::tma_eligible(d, M, method) ? 1 + 2 * d.dtype + (d.masked ? 1 : 0) : 0;
+        group[g].push_back(d);
     }
-    if (tmask::launch_generic(a) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    int used = 0;                                   // problems placed so far: offset into every workspace array
+    for (int g = 0; g < 5; ++g) {
+        const int n = (int)group[g].size();
+        if (n == 0) continue;
+        double* partials = dpart + (size_t)used * kPartialSlots;
+        if (g == 0) {
+            long long total = 0;
+            for (int k = 0; k < n; ++k) { group[g][k].item_begin = total; total += items_of(group[g][k], M); }
+            tmask::LaunchArgs a;
+            a.count = n; a.total_items = total; a.N = N; a.M = M; a.method = method; a.stream = stream; a.status = status_dev;
+            a.partials = partials;
+            const int wpc = tmask::generic_warps_per_cta();
+            const long long want = (total + wpc - 1) / wpc;
+            const int cap = dev.sms * 4 < kPartialSlots / wpc ? dev.sms * 4 : kPartialSlots / wpc;
+            a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));
+            a.single = group[g][0];
+            a.table = nullptr;
+            if (n > 1) {
+                // pageable source: the runtime stages the bytes before returning, so the vector may die here
+                if (cudaMemcpyAsync(dtab + used, group[g].data(), sizeof(DevProblem) * (size_t)n, cudaMemcpyHostToDevice, stream) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+                a.table = dtab + used;
+            }
+            if (tmask::launch_generic(a) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+        } else {
+            const size_t esz = tmask::tma_entry_bytes();
+            std::vector<char> entries(esz * (size_t)n + 128);
+            char* eh = entries.data() + ((128 - (uintptr_t)entries.data() % 128) % 128);
+            long long total = 0;
+            if (!tmask::tma_build_entries(group[g].data(), n, eh, &total)) return TM_ERR_CUDA;
+            tmask::TmaLaunch a;
+            a.entries_host = eh; a.entries_dev = nullptr; a.count = n; a.total_items = total; a.partials = partials;
+            a.status = status_dev; a.dtype = (g - 1) / 2; a.method = method; a.has_out = ((g - 1) & 1) != 0; a.stream = stream;
+            const int wpc = tmask::tma_warps_per_cta();
+            const long long want = (total + wpc - 1) / wpc;
+            const int cap = dev.sms < kPartialSlots / wpc ? dev.sms : kPartialSlots / wpc;
+            a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));
+            if (n > 1) {
+                char* de = dent + (size_t)used * esz;
+                if (cudaMemcpyAsync(de, eh, esz * (size_t)n, cudaMemcpyHostToDevice, stream) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+                a.entries_dev = de;
+            }
+            if (tmask::launch_tma(a) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+        }
+        used += n;
+    }
     return TM_OK;
 }
 
@@ -118,7 +157,7 @@ int ensure_scratch(DeviceState& d) {
     if (d.scratch) return TM_OK;
     std::lock_guard<std::mutex> lock(g_mutex);
     if (d.scratch) return TM_OK;
-    const size_t bytes = kHeaderBytes + table_bytes(1) + partial_bytes(1);
+    const size_t bytes = tm_workspace_bytes(nullptr, 1);
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
     if (cudaMemset(p, 0, kHeaderBytes) != cudaSuccess) { cudaGetLastError(); cudaFree(p); return TM_ERR_CUDA; }
@@ -159,7 +198,7 @@ size_t tm_mask_words_per_row(int64_t cols) { return cols > 0 ? (size_t)((cols + 
 size_t tm_mask_words(int64_t rows, int64_t cols) { return rows > 0 ? (size_t)rows * tm_mask_words_per_row(cols) : 0; }
 
 size_t tm_workspace_bytes(const tm_problem* /*probs_host*/, int count) {
-    return kHeaderBytes + table_bytes(count) + partial_bytes(count);
+    return kHeaderBytes + table_bytes(count) + entry_bytes(count) + partial_bytes(count);
 }
 
 int tm_find_mask(const void* W, int64_t rows, int64_t cols, int N, int M, int method,

@@ -21,4 +21,23 @@ struct LaunchArgs {
 cudaError_t launch_generic(const LaunchArgs& a);
 int generic_warps_per_cta();
 
+// Bandwidth path (TMA-staged, bit-parallel): approximate 2:4 search on 16-byte aligned matrices.
+struct TmaLaunch {
+    const void* entries_host;   // `count` records of tma_entry_bytes() each, built by tma_build_entries()
+    const void* entries_dev;    // the same records in device memory, or nullptr when count == 1
+    int count;
+    long long total_items;
+    double* partials;           // device scratch, count * ctas * tma_warps_per_cta() doubles
+    int* status;
+    int ctas;
+    int dtype, method;
+    bool has_out;               // masked_w_out present (all problems of one launch agree)
+    cudaStream_t stream;
+};
+size_t tma_entry_bytes();
+int tma_warps_per_cta();
+bool tma_eligible(const DevProblem& p, int M, int method);
+bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items);
+cudaError_t launch_tma(const TmaLaunch& a);
+
 }  // namespace tmask
