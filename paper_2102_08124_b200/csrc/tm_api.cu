@@ -137,7 +137,7 @@ int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, 
             tmask::TmaLaunch a;
             a.entries_host = eh; a.entries_dev = nullptr; a.count = n; a.total_items = total; a.partials = partials;
             a.status = status_dev; a.dtype = (g - 1) / 2; a.method = method; a.has_out = ((g - 1) & 1) != 0; a.stream = stream;
-            const int wpc = tmask::tma_warps_per_cta();
+            const int wpc = tmask::tma_warps_per_cta(a.dtype);
             const long long want = (total + wpc - 1) / wpc;
             const int cap = dev.sms < kPartialSlots / wpc ? dev.sms : kPartialSlots / wpc;
             a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));

@@ -18,8 +18,12 @@
 // Such an entry is reached by the sequential scan before its line fills up, so the rounds reproduce
 // the scan exactly; every round takes at least one entry per unfinished block, and a block never
 // lacks more than four entries.
-// Step C (one 2-for-1 swap) is needed by roughly one block in six and is done per block by
-// swap_fix_2_4().
+// Step C (one 2-for-1 swap) is needed by roughly one block in six.  After step B such a block has
+// exactly one short row r and one short column c, each holding the single entry (r,c); the swap
+// removes the lightest kept entry x = (r',c') outside row r (none of them lies in column c) and adds
+// (r,c') and (r',c).  x is lighter than the other kept entry of its row and of its column, so it is
+// one of the at most three "local minima" that swap_candidates() marks from the relation masks;
+// only those few need their magnitudes compared.
 #pragma once
 #include <cstdint>
 
@@ -66,60 +70,96 @@ TM_HD uint32_t cover_2_4(const Rel24& r) {
 }
 
 // Lines that already hold two kept entries / at least one, replicated over the line's bits.
-TM_HD void line_fill(uint32_t kept, uint32_t& row_full, uint32_t& row_has, uint32_t& col_full, uint32_t& col_has) {
+struct LineFill {
+    uint32_t row_full, row_has, col_full, col_has;
+};
+TM_HD LineFill line_fill(uint32_t kept) {
+    LineFill f;
     {
         const uint32_t a = kept, b = kept >> 1, c = kept >> 2, d = kept >> 3, t = a | b | c;
-        row_has = ((t | d) & 0x11111111u) * 15u;
-        row_full = ((maj3(a, b, c) | (d & t)) & 0x11111111u) * 15u;
+        f.row_has = ((t | d) & 0x11111111u) * 15u;
+        f.row_full = ((maj3(a, b, c) | (d & t)) & 0x11111111u) * 15u;
     }
     {
         const uint32_t a = kept, b = kept >> 4, c = kept >> 8, d = kept >> 12, t = a | b | c;
-        col_has = ((t | d) & 0x000F000Fu) * 0x1111u;
-        col_full = ((maj3(a, b, c) | (d & t)) & 0x000F000Fu) * 0x1111u;
+        f.col_has = ((t | d) & 0x000F000Fu) * 0x1111u;
+        f.col_full = ((maj3(a, b, c) | (d & t)) & 0x000F000Fu) * 0x1111u;
     }
+    return f;
+}
+TM_HD uint32_t open_candidates(uint32_t kept, const LineFill& f) { return ~(kept | f.row_full | f.col_full); }
+
+// entries of `set` that have a heavier member of `set` in their row: at least one / at least two
+TM_HD void heavier_in_row(const Rel24& r, uint32_t set, uint32_t& any, uint32_t& two) {
+    const uint32_t a = r.hr1 & rot_row<1>(set), b = r.hr2 & rot_row<2>(set), c = r.hr3 & rot_row<3>(set);
+    any = a | b | c; two = maj3(a, b, c);
+}
+TM_HD void heavier_in_col(const Rel24& r, uint32_t set, uint32_t& any, uint32_t& two) {
+    const uint32_t a = r.hc1 & rot_col<1>(set), b = r.hc2 & rot_col<2>(set), c = r.hc3 & rot_col<3>(set);
+    any = a | b | c; two = maj3(a, b, c);
 }
 
-// One round of step B.  Returns the candidates that were still open when the round began (0 = done).
-TM_HD uint32_t fill_round_2_4(const Rel24& r, uint32_t& kept) {
-    uint32_t row_full, row_has, col_full, col_has;
-    line_fill(kept, row_full, row_has, col_full, col_has);
-    const uint32_t cand = ~(kept | row_full | col_full);
-    // heavier candidates in the same row: at least one / at least two
-    const uint32_t r1 = r.hr1 & rot_row<1>(cand), r2 = r.hr2 & rot_row<2>(cand), r3 = r.hr3 & rot_row<3>(cand);
-    const uint32_t row_rej = maj3(r1, r2, r3) | ((r1 | r2 | r3) & row_has);   // a row holding one entry lacks one
-    const uint32_t c1 = r.hc1 & rot_col<1>(cand), c2 = r.hc2 & rot_col<2>(cand), c3 = r.hc3 & rot_col<3>(cand);
-    const uint32_t col_rej = maj3(c1, c2, c3) | ((c1 | c2 | c3) & col_has);
-    kept |= cand & ~(row_rej | col_rej);
-    return cand;
+// One round of step B on the candidates `cand` (= open_candidates(kept, f)): returns the entries taken.
+TM_HD uint32_t fill_accept(const Rel24& r, const LineFill& f, uint32_t cand) {
+    uint32_t ra, r2, ca, c2;
+    heavier_in_row(r, cand, ra, r2);
+    heavier_in_col(r, cand, ca, c2);
+    // a line holding one entry lacks one (no heavier candidate allowed), an empty line lacks two
+    return cand & ~(r2 | (ra & f.row_has) | c2 | (ca & f.col_has));
+}
+
+// Steps A and B for one pair of blocks, without cross-lane votes (host tests, simple kernels).
+TM_HD uint32_t cover_and_fill_2_4(const Rel24& r, LineFill& f) {
+    uint32_t kept = cover_2_4(r);
+    f = line_fill(kept);
+    for (int round = 0; round < 4; ++round) {
+        const uint32_t cand = open_candidates(kept, f);
+        if (!cand) break;
+        kept |= fill_accept(r, f, cand);
+        f = line_fill(kept);
+    }
+    return kept;
 }
 
 // Blocks (A: bit 0, B: bit 1) that still have a short row after step B, i.e. need step C.
-TM_HD uint32_t short_blocks(uint32_t kept) {
-    uint32_t row_full, row_has, col_full, col_has;
-    line_fill(kept, row_full, row_has, col_full, col_has);
-    return ((row_full & 0xFFFFu) != 0xFFFFu ? 1u : 0u) | ((row_full >> 16) != 0xFFFFu ? 2u : 0u);
+TM_HD uint32_t short_blocks(const LineFill& f) {
+    return ((f.row_full & 0xFFFFu) != 0xFFFFu ? 1u : 0u) | ((f.row_full >> 16) != 0xFFFFu ? 2u : 0u);
 }
 
-// Step C for one block: kept16 has exactly one short row r and one short column c (each holding one
-// entry, the shared entry (r,c)).  The lightest kept entry (r',c') outside row r and column c gives
-// way to (r,c') and (r',c).  key[p] = magnitude pattern of entry p.  Returns false (mask unchanged)
-// if the block does not have that shape.
-template <class KeyT>
-TM_HD bool swap_fix_2_4(const KeyT (&key)[16], uint32_t& kept16) {
-    int r = -1, c = -1, nshort = 0;
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t rowbits = (kept16 >> (4 * i)) & 0xFu, colbits = (kept16 >> i) & 0x1111u;
-        const int rc = (int)((rowbits & 1) + ((rowbits >> 1) & 1) + ((rowbits >> 2) & 1) + (rowbits >> 3));
-        const int cc = (int)((colbits & 1) + ((colbits >> 4) & 1) + ((colbits >> 8) & 1) + (colbits >> 12));
-        if (rc != 2) { r = i; nshort += (rc == 1) ? 1 : 100; }
-        if (cc != 2) { c = i; nshort += (cc == 1) ? 1 : 100; }
+// Step C, first half (bit-parallel, meaningful for blocks flagged by short_blocks): the kept entries
+// outside the short row that are lighter than the other kept entry of their row and of their column.
+TM_HD uint32_t swap_candidates(const Rel24& r, const LineFill& f, uint32_t kept) {
+    const uint32_t e = kept & f.row_full;           // rows other than the short one
+    uint32_t ra, r2, ca, c2;
+    heavier_in_row(r, e, ra, r2);
+    heavier_in_col(r, e, ca, c2);
+    return e & ra & ca;
+}
+
+// Step C, second half, for one block: `cands16` = swap_candidates of the block (1..3 entries), key(p)
+// returns the magnitude pattern of entry p.  Returns false (mask unchanged) on an unexpected shape.
+template <class KeyFn>
+TM_HD bool swap_apply_2_4(uint32_t& kept16, uint32_t cands16, KeyFn key) {
+    // the short row / column: the only ones not holding two entries
+    const uint32_t a = kept16, t = a | (a >> 1) | (a >> 2);
+    const uint32_t rfull = (maj3(a, a >> 1, a >> 2) | ((a >> 3) & t)) & 0x1111u;
+    const uint32_t u = a | (a >> 4) | (a >> 8);
+    const uint32_t cfull = (maj3(a, a >> 4, a >> 8) | ((a >> 12) & u)) & 0x000Fu;
+    const uint32_t rshort = rfull ^ 0x1111u, cshort = cfull ^ 0xFu;
+    if (!rshort || (rshort & (rshort - 1)) || !cshort || (cshort & (cshort - 1)) || !cands16) return false;
+    int x = -1; uint32_t best = 0;
+    for (int n = 0; n < 3 && cands16; ++n) {                    // ascending positions: the earliest of equals wins
+        int p = 0;
+        { uint32_t low = cands16 & (0u - cands16); while (!((low >> p) & 1)) ++p; }
+        cands16 &= cands16 - 1;
+        const uint32_t kp = key(p);
+        if (x < 0 || kp < best) { x = p; best = kp; }
     }
-    if (nshort != 2 || r < 0 || c < 0 || !((kept16 >> (4 * r + c)) & 1)) return false;
-    const uint32_t elig = kept16 & ~(0xFu << (4 * r)) & ~(0x1111u << c);
-    int x = -1; KeyT best = 0;
-    for (int p = 0; p < 16; ++p)
-        if (((elig >> p) & 1) && (x < 0 || key[p] < best)) { x = p; best = key[p]; }   // ascending p: earliest of equals
-    if (x < 0) return false;
+    if (cands16) return false;
+    int r = 0, c = 0;
+    while (!((rshort >> (4 * r)) & 1)) ++r;
+    while (!((cshort >> c) & 1)) ++c;
+    if (!((kept16 >> (4 * r + c)) & 1)) return false;
     kept16 = (kept16 & ~(1u << x)) | (1u << (4 * r + (x & 3))) | (1u << ((x & ~3) + c));
     return true;
 }

@@ -1,14 +1,21 @@
 // Bandwidth kernels of the approximate 2:4 search (TM_APPROX / TM_APPROX_COVER, M = 4).
 //
 // Every warp runs its own software pipeline over a contiguous range of work items (4 rows x 256
-// columns of one matrix): lane 0 keeps bulk-tensor (TMA) loads of the next items in flight into a
-// private ring of shared-memory stages, the 32 lanes read their two 4x4 blocks from the landed stage
-// with 128-bit shared loads, run the bit-parallel search (tm_core24.cuh) in registers, write the
-// masked weights back into the same stage and lane 0 sends it out with a TMA store.  Mask bytes
-// meet in shared memory and leave as whole 32-bit words.  No CTA-wide synchronisation exists; all
-// waits are bounded.
+// columns of one matrix).  Items are processed two at a time:
+//   1. lane 0 keeps bulk-tensor (TMA) loads of the next batch in flight into a private ring of
+//      shared-memory stages (two stage sets, used alternately);
+//   2. each lane reads its two 4x4 blocks of a landed item with 128-bit shared loads and runs steps
+//      A and B of the search bit-parallel in registers (tm_core24.cuh); the rounds of step B are
+//      warp-uniform (a vote decides whether any lane still has candidates);
+//   3. the blocks that need step C (about one in six) are queued in shared memory and fixed by as
+//      many lanes at once as there are queued blocks, each reading the few magnitudes it must compare
+//      straight from the stage;
+//   4. the lanes write the masked weights back into the stage, lane 0 sends it out with a TMA store,
+//      mask bytes meet in shared memory and leave as whole 32-bit words.
+// No CTA-wide synchronisation exists; every wait is bounded.
 #include "tm_core24.cuh"
 #include "tm_launch.h"
+#include "tm_pair_bf16.cuh"
 #include "tm_tma.cuh"
 
 #include <cstring>
@@ -17,201 +24,321 @@ namespace tmask {
 
 namespace {
 
-constexpr int kWarps = 16;                 // warps per CTA, one CTA per SM
 constexpr int kItemRows = 4;
 constexpr int kItemCols = 256;
+constexpr int kBatch = 2;                  // items per pipeline step
+constexpr int kStages = 2 * kBatch;
 
 template <int DT> struct Geometry {
     static constexpr int kElem = DT == kF32 ? 4 : 2;
-    static constexpr int kStages = DT == kF32 ? 3 : 4;
-    static constexpr int kStageBytes = kItemRows * kItemCols * kElem;
-    static constexpr int kWarpBytes = kStages * kStageBytes + 128 /* mask bytes */ + 64 /* barriers */ + 64;
+    static constexpr int kWarps = DT == kF32 ? 12 : 16;       // warps per CTA, one CTA per SM
+    static constexpr int kRowPitch = kItemCols * kElem;        // bytes between rows inside a stage
+    static constexpr int kStageBytes = kItemRows * kRowPitch;
+    // stages | mask bytes [batch][4][32] | kept [batch][32] | swap candidates [batch][32] | queue | barriers
+    static constexpr int kWarpBytes = kStages * kStageBytes + kBatch * 128 + 2 * kBatch * 128 + 128 + 64 + 64;
 };
-
-// 16 magnitudes of each of the lane's two blocks, as integers ordered like |w|
-template <int DT>
-__device__ __forceinline__ void load_keys(const unsigned char* stage, int lane, uint32_t (&raw)[4][DT == kF32 ? 8 : 4],
-                                          uint32_t (&ka)[16], uint32_t (&kb)[16]) {
-    if constexpr (DT == kBF16) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint4 v = *reinterpret_cast<const uint4*>(stage + i * (kItemCols * 2) + lane * 16);
-            raw[i][0] = v.x; raw[i][1] = v.y; raw[i][2] = v.z; raw[i][3] = v.w;
-            ka[4 * i + 0] = v.x & 0x7FFFu; ka[4 * i + 1] = (v.x >> 16) & 0x7FFFu; ka[4 * i + 2] = v.y & 0x7FFFu; ka[4 * i + 3] = (v.y >> 16) & 0x7FFFu;
-            kb[4 * i + 0] = v.z & 0x7FFFu; kb[4 * i + 1] = (v.z >> 16) & 0x7FFFu; kb[4 * i + 2] = v.w & 0x7FFFu; kb[4 * i + 3] = (v.w >> 16) & 0x7FFFu;
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint4 a = *reinterpret_cast<const uint4*>(stage + i * (kItemCols * 4) + lane * 32);
-            const uint4 b = *reinterpret_cast<const uint4*>(stage + i * (kItemCols * 4) + lane * 32 + 16);
-            raw[i][0] = a.x; raw[i][1] = a.y; raw[i][2] = a.z; raw[i][3] = a.w; raw[i][4] = b.x; raw[i][5] = b.y; raw[i][6] = b.z; raw[i][7] = b.w;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) { ka[4 * i + j] = raw[i][j] & 0x7FFFFFFFu; kb[4 * i + j] = raw[i][4 + j] & 0x7FFFFFFFu; }
-        }
-    }
-}
-
-// independent halves of the relation masks from scalar keys (one block into one half of the pair masks)
-__device__ __forceinline__ void relations_scalar(const uint32_t (&k)[16], int shift, Rel24& r) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t a = k[4 * i], b = k[4 * i + 1], c = k[4 * i + 2], d = k[4 * i + 3];
-        r.hr1 |= ((b >= a ? 1u : 0u) | (c >= b ? 2u : 0u) | (d >= c ? 4u : 0u) | (a > d ? 8u : 0u)) << (4 * i + shift);
-        r.hr2 |= ((c >= a ? 1u : 0u) | (d >= b ? 2u : 0u)) << (4 * i + shift);
-        const uint32_t e = k[i], f = k[4 + i], g = k[8 + i], h = k[12 + i];
-        r.hc1 |= ((f >= e ? 0x1u : 0u) | (g >= f ? 0x10u : 0u) | (h >= g ? 0x100u : 0u) | (e > h ? 0x1000u : 0u)) << (i + shift);
-        r.hc2 |= ((g >= e ? 0x1u : 0u) | (h >= f ? 0x10u : 0u)) << (i + shift);
-    }
-}
 
 struct alignas(128) TmaEntry {
     CUtensorMap in, out;
     DevProblem p;
     int cchunks;       // items per block row (256 columns each)
+    int brows;         // block rows
 };
 static_assert(sizeof(TmaEntry) == 384 || sizeof(TmaEntry) == 512, "descriptor records stay 128-byte aligned in tables");
 
+// Walks the work items of a table of problems in order: problem k, block row bi, column chunk cj.
+struct Cursor {
+    int k, bi, cj, cchunks, brows;
+    __device__ __forceinline__ void load(const TmaEntry* tab, int count) {
+        while (k < count && (tab[k].brows == 0 || tab[k].cchunks == 0)) ++k;   // empty matrices have no items
+        if (k < count) { cchunks = tab[k].cchunks; brows = tab[k].brows; } else { cchunks = 1; brows = 1; }
+    }
+    __device__ __forceinline__ void seek(const TmaEntry* tab, int count, long long item) {
+        k = 0;
+        while (k + 1 < count && tab[k + 1].p.item_begin <= item) ++k;
+        load(tab, count);
+        const long long local = item - tab[k < count ? k : count - 1].p.item_begin;
+        bi = (int)(local / cchunks); cj = (int)(local - (long long)bi * cchunks);
+    }
+    __device__ __forceinline__ void advance(const TmaEntry* tab, int count) {
+        if (++cj == cchunks) {
+            cj = 0;
+            if (++bi == brows) { bi = 0; ++k; load(tab, count); }
+        }
+    }
+};
+
+// ------------------------------------------------------------------------------------------
+// per-dtype front end: relation masks of the lane's two blocks; largest magnitude seen
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+template <int DT>
+__device__ __forceinline__ void front_end(const unsigned char* stage, int lane, Rel24& rel, uint32_t& worst) {
+    if constexpr (DT == kBF16) {
+        uint4 v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = *reinterpret_cast<const uint4*>(stage + i * 512 + lane * 16);
+        PairKeys pk;
+        interleave_keys(v, pk);
+        uint32_t m[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m[i] = max_u16x2(max_u16x2(pk.x[i][0], pk.x[i][1]), max_u16x2(pk.x[i][2], pk.x[i][3]));
+        worst = max_u16x2(worst, max_u16x2(max_u16x2(m[0], m[1]), max_u16x2(m[2], m[3])));
+        relations_bf16(pk, rel);
+    } else {
+        uint32_t ka[16], kb[16];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint4 a = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32);
+            const uint4 b = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32 + 16);
+            ka[4 * i] = a.x & 0x7FFFFFFFu; ka[4 * i + 1] = a.y & 0x7FFFFFFFu; ka[4 * i + 2] = a.z & 0x7FFFFFFFu; ka[4 * i + 3] = a.w & 0x7FFFFFFFu;
+            kb[4 * i] = b.x & 0x7FFFFFFFu; kb[4 * i + 1] = b.y & 0x7FFFFFFFu; kb[4 * i + 2] = b.z & 0x7FFFFFFFu; kb[4 * i + 3] = b.w & 0x7FFFFFFFu;
+        }
+        rel = Rel24{0, 0, 0, 0, 0, 0};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t (&k)[16] = h ? kb : ka;
+            const int shift = 16 * h;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t a = k[4 * i], b = k[4 * i + 1], c = k[4 * i + 2], d = k[4 * i + 3];
+                rel.hr1 |= ((b >= a ? 1u : 0u) | (c >= b ? 2u : 0u) | (d >= c ? 4u : 0u) | (a > d ? 8u : 0u)) << (4 * i + shift);
+                rel.hr2 |= ((c >= a ? 1u : 0u) | (d >= b ? 2u : 0u)) << (4 * i + shift);
+                const uint32_t e = k[i], f = k[4 + i], g = k[8 + i], hh = k[12 + i];
+                rel.hc1 |= ((f >= e ? 0x1u : 0u) | (g >= f ? 0x10u : 0u) | (hh >= g ? 0x100u : 0u) | (e > hh ? 0x1000u : 0u)) << (i + shift);
+                rel.hc2 |= ((g >= e ? 0x1u : 0u) | (hh >= f ? 0x10u : 0u)) << (i + shift);
+                worst = max(worst, max(max(a, b), max(c, d)));
+            }
+        }
+        complete_relations(rel);
+    }
+}
+
+// Step C, second half, on a block whose magnitudes sit in shared memory (natural layout).
+template <int DT>
+__device__ __forceinline__ bool swap_apply_smem(const unsigned char* blk, uint32_t& kept16, uint32_t cands16) {
+    const uint32_t a = kept16, t = a | (a >> 1) | (a >> 2);
+    const uint32_t rshort = ((maj3(a, a >> 1, a >> 2) | ((a >> 3) & t)) & 0x1111u) ^ 0x1111u;
+    const uint32_t u = a | (a >> 4) | (a >> 8);
+    const uint32_t cshort = ((maj3(a, a >> 4, a >> 8) | ((a >> 12) & u)) & 0xFu) ^ 0xFu;
+    if (__popc(rshort) != 1 || __popc(cshort) != 1 || cands16 == 0 || __popc(cands16) > 3) return false;
+    int x = -1; uint32_t best = 0;
+#pragma unroll
+    for (int n = 0; n < 3; ++n) {                                   // ascending positions: the earliest of equals wins
+        if (cands16) {
+            const int p = __ffs(cands16) - 1;
+            cands16 &= cands16 - 1;
+            uint32_t kp;
+            if constexpr (DT == kBF16) kp = *reinterpret_cast<const unsigned short*>(blk + (p >> 2) * 512 + (p & 3) * 2) & 0x7FFFu;
+            else kp = *reinterpret_cast<const uint32_t*>(blk + (p >> 2) * 1024 + (p & 3) * 4) & 0x7FFFFFFFu;
+            if (x < 0 || kp < best) { x = p; best = kp; }
+        }
+    }
+    const int r4 = __ffs(rshort) - 1, c = __ffs(cshort) - 1;        // r4 = 4 * short row
+    if (!((kept16 >> (r4 + c)) & 1)) return false;
+    kept16 = (kept16 & ~(1u << x)) | (1u << (r4 + (x & 3))) | (1u << ((x & ~3) + c));
+    return true;
+}
+
+// Masked weights back into the stage, mask bytes, objective contribution of the lane's two blocks.
+template <int DT, bool HAS_OUT>
+__device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* mrow /* [4][32] */, int lane, uint32_t kept) {
+    float s4 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if constexpr (DT == kBF16) {
+            const uint4 r = *reinterpret_cast<const uint4*>(stage + i * 512 + lane * 16);
+            const uint32_t raw[4] = {r.x, r.y, r.z, r.w};
+            uint32_t o[4], m[4];
+            lane_masks(kept, i, m);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                o[q] = raw[q] & m[q];
+                const uint32_t ab = raw[q] & m[q] & 0x7FFF7FFFu;
+                unsigned short lo, hi;
+                asm("mov.b32 {%0,%1}, %2;" : "=h"(lo), "=h"(hi) : "r"(ab));
+                asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(s4) : "h"(lo));        // fp32 accumulator + bf16 addend
+                asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(s4) : "h"(hi));
+            }
+            if constexpr (HAS_OUT) *reinterpret_cast<uint4*>(stage + i * 512 + lane * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+        } else {
+            const uint4 ra = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32);
+            const uint4 rb = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32 + 16);
+            const uint32_t raw[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+            uint32_t o[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const uint32_t bit = (kept >> (4 * i + (q & 3) + (q >> 2) * 16)) & 1u;
+                o[q] = bit ? raw[q] : 0u;
+                s4 += fabsf(__uint_as_float(o[q]));
+            }
+            if constexpr (HAS_OUT) {
+                *reinterpret_cast<uint4*>(stage + i * 1024 + lane * 32) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4*>(stage + i * 1024 + lane * 32 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+        }
+        mrow[i * 32 + lane] = (unsigned char)(((kept >> (4 * i)) & 0xFu) | ((kept >> (12 + 4 * i)) & 0xF0u));
+    }
+    return s4;
+}
+
 template <int DT, int METHOD, bool HAS_OUT>
-__global__ void __launch_bounds__(kWarps * 32, 1)
+__global__ void __launch_bounds__(Geometry<DT>::kWarps * 32, 1)
 tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict__ table, int count, long long total_items,
              double* __restrict__ partials, int* __restrict__ status_out) {
     using G = Geometry<DT>;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    unsigned char* wbase = smem_raw + (size_t)warp * G::kWarpBytes;
-    unsigned char* stages = wbase;
-    unsigned char* mbytes = wbase + G::kStages * G::kStageBytes;          // [4 rows][32 bytes]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(mbytes + 128);
+    unsigned char* stages = smem_raw + (size_t)warp * G::kWarpBytes;
+    unsigned char* mbytes = stages + kStages * G::kStageBytes;
+    uint32_t* kbuf = reinterpret_cast<uint32_t*>(mbytes + kBatch * 128);
+    uint32_t* cbuf = kbuf + kBatch * 32;
+    unsigned char* queue = reinterpret_cast<unsigned char*>(cbuf + kBatch * 32);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(queue + 128);
 
-    const long long gw = (long long)blockIdx.x * kWarps + warp, nwarps = (long long)gridDim.x * kWarps;
+    const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
     const long long per = (total_items + nwarps - 1) / nwarps;
     const long long begin = gw * per, end = min(total_items, begin + per);
+    const int n_items = (int)max(0ll, end - begin);
     const TmaEntry* tab = table ? table : &single;
 
     if (lane == 0) {
-        for (int s = 0; s < G::kStages; ++s) mbar_init(&bars[s], 1);
+        for (int s = 0; s < kStages; ++s) mbar_init(&bars[s], 1);
         fence_mbar_init();
     }
     __syncwarp();
 
-    int status = 0;
-    // producer state (lane 0): next item to request and its problem index
-    long long next = begin; int next_k = 0;
-    auto issue = [&](long long item) {
-        while (next_k + 1 < count && tab[next_k + 1].p.item_begin <= item) ++next_k;
-        const TmaEntry& e = tab[next_k];
-        const long long local = item - e.p.item_begin;
-        const int bi = (int)(local / e.cchunks), cj = (int)(local - (long long)bi * e.cchunks);
-        const int s = (int)((item - begin) % G::kStages);
-        mbar_expect_tx(&bars[s], G::kStageBytes);
-        tma_load_2d(stages + s * G::kStageBytes, &e.in, cj * kItemCols, bi * kItemRows, &bars[s]);
+    Cursor ld, cur;                        // next item to request / first item of the batch in process
+    ld.seek(tab, count, begin);
+    cur = ld;
+    int loaded = 0;
+    auto issue_next = [&](int s) {         // all lanes track the cursor, lane 0 issues the copy
+        if (lane == 0) {
+            mbar_expect_tx(&bars[s], G::kStageBytes);
+            tma_load_2d(stages + s * G::kStageBytes, &tab[ld.k].in, ld.cj * kItemCols, ld.bi * kItemRows, &bars[s]);
+        }
+        ld.advance(tab, count);
+        ++loaded;
     };
-    if (lane == 0)
-        for (int i = 0; i < G::kStages - 2 && next < end; ++i) issue(next++);
+    for (int g = 0; g < kBatch && loaded < n_items; ++g) issue_next(g);
 
-    int k = 0, acc_k = -1;
+    int status = 0, acc_k = -1;
     float facc = 0.f; double acc = 0.0;
-    uint32_t worst = 0;                                                   // largest magnitude pattern seen
+    uint32_t worst = 0;                                                  // largest magnitude pattern seen (per 16-bit lane for bf16)
+    const uint32_t lt = (1u << lane) - 1u;
+    bool alive = true;
 
-    for (long long item = begin; item < end; ++item) {
-        const int s = (int)((item - begin) % G::kStages);
-        // keep the ring full: the stage being refilled was stored from two items ago
-        if (lane == 0 && next < end) {
-            if constexpr (HAS_OUT) tma_wait_read<1>();
-            issue(next++);
-        }
-        while (k + 1 < count && tab[k + 1].p.item_begin <= item) ++k;
-        const TmaEntry& e = tab[k];
-        if (k != acc_k) {
-            if (acc_k >= 0) {
-                acc += (double)facc; facc = 0.f;
-                for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-                if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
-            }
-            acc = 0.0; acc_k = k;
-        }
-        const long long local = item - e.p.item_begin;
-        const int bi = (int)(local / e.cchunks), cj = (int)(local - (long long)bi * e.cchunks);
-        const int col0 = cj * kItemCols + lane * 8;                       // first column of the lane's two blocks
-        const uint32_t parity = (uint32_t)(((item - begin) / G::kStages) & 1);
-        if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bars[s], parity))) {
-            // a copy never landed: give the copies still in flight a bounded chance to finish, then stop
-            status |= kDevInternal;
-            if (lane == 0)
-                for (long long j = item + 1; j < next; ++j)
-                    mbar_wait_bounded(&bars[(j - begin) % G::kStages], (uint32_t)(((j - begin) / G::kStages) & 1), 1u << 16);
-            break;
-        }
-
-        unsigned char* stage = stages + s * G::kStageBytes;
-        uint32_t raw[4][DT == kF32 ? 8 : 4], ka[16], kb[16];
-        load_keys<DT>(stage, lane, raw, ka, kb);
+    for (int done = 0, batch = 0; done < n_items && alive; done += kBatch, ++batch) {
+        const int nb = min(kBatch, n_items - done), set = batch & 1;
+        const uint32_t parity = (uint32_t)((batch >> 1) & 1);
+        int qn = 0;
+        // ---- steps A and B on every item of the batch -------------------------------------------
 #pragma unroll
-        for (int p = 0; p < 16; ++p) worst = max(worst, max(ka[p], kb[p]));
-
-        Rel24 rel = {0, 0, 0, 0, 0, 0};
-        relations_scalar(ka, 0, rel);
-        relations_scalar(kb, 16, rel);
-        complete_relations(rel);
-        uint32_t kept = cover_2_4(rel);
+        for (int g = 0; g < kBatch; ++g) {
+            if (g < nb) {
+                const int s = set * kBatch + g;
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bars[s], parity))) { status |= kDevInternal; alive = false; }
+                Rel24 rel;
+                front_end<DT>(stages + s * G::kStageBytes, lane, rel, worst);
+                uint32_t k = cover_2_4(rel);
+                if constexpr (METHOD == kMethodApprox) {
+                    LineFill f = line_fill(k);
+                    uint32_t cand = open_candidates(k, f);
+                    int rounds = 0;
+                    while (__any_sync(0xFFFFFFFFu, cand != 0)) {
+                        if (++rounds > 4) { status |= kDevInternal; break; }    // a block lacks at most four entries
+                        k |= fill_accept(rel, f, cand);
+                        f = line_fill(k);
+                        cand = open_candidates(k, f);
+                    }
+                    const uint32_t sb = short_blocks(f);
+                    if (__any_sync(0xFFFFFFFFu, sb != 0)) {
+                        cbuf[g * 32 + lane] = swap_candidates(rel, f, k);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const bool need = (sb >> h) & 1;
+                            const uint32_t m = __ballot_sync(0xFFFFFFFFu, need);
+                            if (need) queue[qn + __popc(m & lt)] = (unsigned char)((g << 6) | (h << 5) | lane);
+                            qn += __popc(m);
+                        }
+                    }
+                }
+                kbuf[g * 32 + lane] = k;
+            }
+            if (g == 0) {      // refill the other stage set: its stores were issued one batch ago
+                if constexpr (HAS_OUT) { if (lane == 0 && batch > 0) tma_wait_read<0>(); }
+                for (int gg = 0; gg < kBatch; ++gg) if (loaded < n_items) issue_next((set ^ 1) * kBatch + gg);
+            }
+        }
+        __syncwarp();
+        // ---- step C on the queued blocks ---------------------------------------------------------
         if constexpr (METHOD == kMethodApprox) {
-            int rounds = 0;
-            while (__any_sync(0xFFFFFFFFu, fill_round_2_4(rel, kept) != 0)) {
-                if (++rounds > 4) { status |= kDevInternal; break; }       // a block lacks at most four entries
-            }
-            const uint32_t sb = short_blocks(kept);
-            if (sb & 1) { uint32_t h = kept & 0xFFFFu; if (!swap_fix_2_4(ka, h)) status |= kDevInternal; kept = (kept & 0xFFFF0000u) | h; }
-            if (sb & 2) { uint32_t h = kept >> 16; if (!swap_fix_2_4(kb, h)) status |= kDevInternal; kept = (kept & 0xFFFFu) | (h << 16); }
-        }
-        // blocks past the last column (zero-filled by the copy) contribute nothing
-        if (col0 >= e.p.cols) kept = 0;
-        else if (col0 + 4 >= e.p.cols) kept &= 0xFFFFu;
-
-        // objective, masked weights, mask bytes
-        float s4 = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t na = (kept >> (4 * i)) & 0xFu, nb = (kept >> (16 + 4 * i)) & 0xFu;
-            if constexpr (DT == kBF16) {
-                uint32_t out[4];
-#pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    const uint32_t bits = (v < 2 ? na >> (2 * v) : nb >> (2 * (v - 2))) & 3u;
-                    const uint32_t m = ((bits & 1u) ? 0x0000FFFFu : 0u) | ((bits & 2u) ? 0xFFFF0000u : 0u);
-                    out[v] = raw[i][v] & m;
-                    s4 += __uint_as_float((out[v] << 16) & 0x7FFFFFFFu) + __uint_as_float(out[v] & 0x7FFF0000u);
-                }
-                if constexpr (HAS_OUT)
-                    *reinterpret_cast<uint4*>(stage + i * (kItemCols * 2) + lane * 16) = make_uint4(out[0], out[1], out[2], out[3]);
-            } else {
-                uint32_t out[8];
-#pragma unroll
-                for (int v = 0; v < 8; ++v) {
-                    const uint32_t bit = (v < 4 ? na >> v : nb >> (v - 4)) & 1u;
-                    out[v] = bit ? raw[i][v] : 0u;
-                    s4 += __uint_as_float(out[v] & 0x7FFFFFFFu);
-                }
-                if constexpr (HAS_OUT) {
-                    *reinterpret_cast<uint4*>(stage + i * (kItemCols * 4) + lane * 32) = make_uint4(out[0], out[1], out[2], out[3]);
-                    *reinterpret_cast<uint4*>(stage + i * (kItemCols * 4) + lane * 32 + 16) = make_uint4(out[4], out[5], out[6], out[7]);
+            for (int q0 = 0; q0 < qn; q0 += 32) {
+                if (q0 + lane < qn) {
+                    const uint32_t e = queue[q0 + lane];
+                    const int g = e >> 6, h = (e >> 5) & 1, ln = e & 31;
+                    unsigned short* kh = reinterpret_cast<unsigned short*>(kbuf + g * 32 + ln) + h;
+                    uint32_t k16 = *kh;
+                    const uint32_t c16 = reinterpret_cast<const unsigned short*>(cbuf + g * 32 + ln)[h];
+                    const unsigned char* blk = stages + (set * kBatch + g) * G::kStageBytes + ln * (8 * G::kElem) + h * (4 * G::kElem);
+                    if (!swap_apply_smem<DT>(blk, k16, c16)) status |= kDevInternal;
+                    *kh = (unsigned short)k16;
                 }
             }
-            mbytes[i * 32 + lane] = (unsigned char)(na | (nb << 4));
+            __syncwarp();
         }
-        facc += s4;
+        // ---- outputs ---------------------------------------------------------------------------
+        Cursor out = cur;
+#pragma unroll
+        for (int g = 0; g < kBatch; ++g) {
+            if (g < nb) {
+                if (out.k != acc_k) {                                   // a new matrix starts: flush the objective partial
+                    if (acc_k >= 0) {
+                        acc += (double)facc;
+                        for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+                        if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
+                    }
+                    acc = 0.0; facc = 0.f; acc_k = out.k;
+                }
+                uint32_t k = kbuf[g * 32 + lane];
+                // blocks past the last column (zero-filled by the copy) contribute nothing
+                const int col0 = out.cj * kItemCols + lane * 8;
+                const int cols = (int)tab[out.k].p.cols;
+                if (col0 >= cols) k = 0;
+                else if (col0 + 4 >= cols) k &= 0xFFFFu;
+                facc += back_end<DT, HAS_OUT>(stages + (set * kBatch + g) * G::kStageBytes, mbytes + g * 128, lane, k);
+                out.advance(tab, count);
+            }
+        }
         if constexpr (HAS_OUT) fence_proxy_async_smem();
         __syncwarp();
-        if constexpr (HAS_OUT) {
-            if (lane == 0) { tma_store_2d(&e.out, cj * kItemCols, bi * kItemRows, stage); tma_commit(); }
+        out = cur;
+#pragma unroll
+        for (int g = 0; g < kBatch; ++g) {
+            if (g < nb) {
+                const TmaEntry& e = tab[out.k];
+                if constexpr (HAS_OUT) {
+                    if (lane == 0) tma_store_2d(&e.out, out.cj * kItemCols, out.bi * kItemRows, stages + (set * kBatch + g) * G::kStageBytes);
+                }
+                const int row = lane >> 3, word = out.cj * 8 + (lane & 7);
+                const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + g * 128 + row * 32 + (lane & 7) * 4);
+                if (word < e.p.wpr) e.p.mask[((long long)out.bi * kItemRows + row) * e.p.wpr + word] = w;
+                out.advance(tab, count);
+            }
         }
-        {   // 4 rows x 8 words of mask
-            const int row = lane >> 3, word = cj * 8 + (lane & 7);
-            const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + row * 32 + (lane & 7) * 4);
-            if (word < e.p.wpr) e.p.mask[((long long)bi * kItemRows + row) * e.p.wpr + word] = w;
-        }
+        if constexpr (HAS_OUT) { if (lane == 0) tma_commit(); }
+        cur = out;
+        if ((batch & 31) == 31) { acc += (double)facc; facc = 0.f; }       // keep the fp32 partial short
         __syncwarp();
-        if (((item - begin) & 63) == 63) { acc += (double)facc; facc = 0.f; }   // keep the fp32 partial short
+    }
+    if (!alive && lane == 0) {
+        // a copy never landed: give the copies still in flight a bounded chance to finish before the stages die
+        for (int s = 0; s < kStages; ++s) { mbar_wait_bounded(&bars[s], 0, 1u << 14); mbar_wait_bounded(&bars[s], 1, 1u << 14); }
     }
     if (lane == 0) tma_wait_all<0>();
     if (acc_k >= 0) {
@@ -219,7 +346,8 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
         if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
     }
-    if (worst >= (DT == kF32 ? 0x7F800000u : 0x7F80u)) status |= kDevNonFinite;
+    if constexpr (DT == kF32) { if (worst >= 0x7F800000u) status |= kDevNonFinite; }
+    else { if ((worst & 0xFFFFu) >= 0x7F80u || (worst >> 16) >= 0x7F80u) status |= kDevNonFinite; }
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(0xFFFFFFFFu, status, o);
     if (lane == 0 && status && status_out) atomicOr(status_out, status);
 }
@@ -270,7 +398,7 @@ bool encode_map(CUtensorMap* m, const void* base, int dtype, long long rows, lon
 template <int DT, int METHOD, bool HAS_OUT>
 cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntry* table) {
     using G = Geometry<DT>;
-    const size_t smem = (size_t)kWarps * G::kWarpBytes;
+    const size_t smem = (size_t)G::kWarps * G::kWarpBytes;
     auto kern = tma24_kernel<DT, METHOD, HAS_OUT>;
     static bool configured = false;        // per instantiation
     if (!configured) {
@@ -278,21 +406,22 @@ cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntr
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<a.ctas, kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status);
+    kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status);
     return cudaGetLastError();
 }
 
 }  // namespace
 
 size_t tma_entry_bytes() { return sizeof(TmaEntry); }
-int tma_warps_per_cta() { return kWarps; }
+int tma_warps_per_cta(int dtype) { return dtype == kF32 ? Geometry<kF32>::kWarps : Geometry<kBF16>::kWarps; }
 
 bool tma_eligible(const DevProblem& p, int M, int method) {
     if (M != 4 || (method != kMethodApprox && method != kMethodCover)) return false;
     const size_t elem = p.dtype == kF32 ? 4 : 2;
     if ((uintptr_t)p.W % 16 || ((size_t)p.ld * elem) % 16) return false;
     if (p.masked && (uintptr_t)p.masked % 16) return false;
-    if (p.rows >= (1ll << 31) || p.cols >= (1ll << 31) || (size_t)p.ld * elem >= (1ull << 40)) return false;
+    if (p.rows >= (1ll << 31) || p.cols >= (1ll << 31) - kItemCols || (size_t)p.ld * elem >= (1ull << 40)) return false;
+    if ((p.rows / kItemRows) * ((p.cols + kItemCols - 1) / kItemCols) >= (1ll << 30)) return false;
     return encode_fn() != nullptr;
 }
 
@@ -301,11 +430,13 @@ bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, l
     TmaEntry* e = static_cast<TmaEntry*>(entries_host);
     long long total = 0;
     for (int k = 0; k < count; ++k) {
+        memset(&e[k], 0, sizeof(TmaEntry));
         e[k].p = probs[k];
         e[k].cchunks = (int)((probs[k].cols + kItemCols - 1) / kItemCols);
+        e[k].brows = (int)(probs[k].rows / kItemRows);
         e[k].p.item_begin = total;
-        total += (probs[k].rows / kItemRows) * (long long)e[k].cchunks;
-        if (probs[k].rows == 0 || probs[k].cols == 0) { memset(&e[k].in, 0, sizeof(CUtensorMap)); memset(&e[k].out, 0, sizeof(CUtensorMap)); continue; }
+        total += (long long)e[k].brows * e[k].cchunks;
+        if (probs[k].rows == 0 || probs[k].cols == 0) continue;
         if (!encode_map(&e[k].in, probs[k].W, probs[k].dtype, probs[k].rows, probs[k].cols, probs[k].ld)) return false;
         if (probs[k].masked) {
             if (!encode_map(&e[k].out, probs[k].masked, probs[k].dtype, probs[k].rows, probs[k].cols, probs[k].ld)) return false;
@@ -319,7 +450,8 @@ bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, l
 
 // All problems of one launch share dtype and the presence of masked_w_out (the caller groups them).
 cudaError_t launch_tma(const TmaLaunch& a) {
-    cudaError_t err = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * kWarps, a.stream);
+    const int wpc = tma_warps_per_cta(a.dtype);
+    cudaError_t err = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * wpc, a.stream);
     if (err != cudaSuccess) return err;
     const TmaEntry* host = static_cast<const TmaEntry*>(a.entries_host);
     const TmaEntry* table = static_cast<const TmaEntry*>(a.entries_dev);   // nullptr when count == 1
@@ -331,7 +463,7 @@ cudaError_t launch_tma(const TmaLaunch& a) {
 #undef TM_DISPATCH
         if (err != cudaSuccess) return err;
     }
-    reduce_tma_kernel<<<a.count, 256, 0, a.stream>>>(host[0], table, a.partials, (long long)a.ctas * kWarps);
+    reduce_tma_kernel<<<a.count, 256, 0, a.stream>>>(host[0], table, a.partials, (long long)a.ctas * wpc);
     return cudaGetLastError();
 }
 
