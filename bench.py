@@ -32,6 +32,9 @@ FULL_ROWS, COLS = 12288, 49152
 ROWS = FULL_ROWS
 N_KEEP, M_BLOCK = 2, 4
 BYTES_PER_WEIGHT = 2 + 2 + 1.0 / 8          # read W, write masked W, write one mask bit (bf16)
+# dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture on the 2048-row case (see profiles/), per weight
+TRAFFIC_PER_WEIGHT = (201.39e6 + 165.37e6) / (2048 * 49152)
+TRAFFIC_SOURCE = "ncu --set full on the 2048 x 49152 case, scaled by rows (profiles/tma24_kernel_approx_2_4_bf16_2048x49152_full.md)"
 METRIC = "transposable-mask weights/s (2:4 approx, bf16, 1 GPU: achieved HBM GB/s vs peak in `roofline`)"
 WORKLOAD = "%dx49152 bf16, N(0,0.02) quantised to 256 levels (frequent ties), 2:4 approximate, per-step recompute"
 
@@ -236,7 +239,8 @@ def run_gpu(args):
         "gpu_launches": 2 * args.steps,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_source": peak_src, "algorithmic_bytes_per_launch": weights * BYTES_PER_WEIGHT,
+                     "traffic": TRAFFIC_PER_WEIGHT * weights if ROWS == FULL_ROWS else None, "traffic_source": TRAFFIC_SOURCE,
+                     "peak_source": peak_src, "algorithmic_bytes_per_launch": weights * BYTES_PER_WEIGHT,
                      "frac_of_8000": achieved / 8000.0,
                      "note": "duration = CUDA-event time of one step (search kernel + its tiny partial-zeroing and reduction launches)"},
         "cpu_baseline": {"value": cpu_value, "unit": "weights/s", "cores": 1, "kind": "oracle",
