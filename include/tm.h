@@ -78,9 +78,10 @@ extern "C" {
 #define TM_ERR_NM 3         /* (N, M) is not (2, 4) or (4, 8) */
 #define TM_ERR_METHOD 4
 #define TM_ERR_DTYPE 5
-#define TM_ERR_ALIGN 6      /* W / masked_w_out row starts not aligned to one block row (M elements), mask_out not to 4 bytes */
+#define TM_ERR_ALIGN 6      /* W / masked_w_out base or row pitch not a multiple of min(16, M * element size) bytes, mask_out not of 4, objective_out not of 8 */
 #define TM_ERR_CUDA 7       /* a CUDA runtime call failed (no device, launch error, allocation failure) */
 #define TM_ERR_WORKSPACE 8  /* workspace NULL, misaligned (256 bytes) or smaller than tm_workspace_bytes() */
+#define TM_ERR_TOO_LARGE 9  /* more matrices than the built-in scratch of tm_find_mask_batched_static() can serve */
 
 /* device status bits */
 #define TM_DEV_NONFINITE 1  /* an Inf or NaN was met in W (it is ordered by its bit pattern) */
@@ -141,6 +142,31 @@ size_t tm_workspace_bytes(const tm_problem* probs_host, int count);
 int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols, int N, int M, int method,
                       uint32_t* mask_out_host, void* masked_w_out_host, double* objective_out_host,
                       int* status_out_host);
+
+/*
+ * tm_find_mask_batched_static -- no counterpart in the paper: an entry point for callers that must not
+ * allocate device memory.  Some hosts of this library (a plug-in running inside another framework's
+ * memory pool, a real-time loop that pre-allocates everything, code holding a fixed memory budget)
+ * can neither call cudaMalloc themselves nor let a library do it on their behalf, and may have no
+ * place to size a workspace up front either.  This call is tm_find_mask_batched() with the workspace
+ * replaced by a scratch array built into the library image: TM_STATIC_SCRATCH_BYTES of device memory
+ * that every GPU which loads the library holds until the process exits.  It serves at most
+ * TM_STATIC_MAX_MATRICES matrices per call (each of any size); a larger count returns
+ * TM_ERR_TOO_LARGE and launches nothing -- split the model into several calls.  Inputs and outputs
+ * are still the caller's device buffers.
+ *
+ * The call allocates nothing on the device and frees nothing.  The first call on a device looks the
+ * scratch array's device address up (once per device, with that device current); make that first call
+ * before any stream capture begins.  All calls on one device share the one array, which keeps whatever
+ * the previous call left in it: each call clears the objective partials it is about to use, but two
+ * calls that overlap on the GPU (different streams, no dependency between them) race on it and corrupt
+ * each other's objectives -- order them, or use tm_find_mask_batched() with separate workspaces.
+ * Results are bit-identical to tm_find_mask_batched() on the same inputs.
+ */
+#define TM_STATIC_MAX_MATRICES 16
+#define TM_STATIC_SCRATCH_BYTES (1064960)
+int tm_find_mask_batched_static(const tm_problem* probs_host, int count, int N, int M, int method,
+                                int* status_dev, void* cuda_stream);
 
 const char* tm_status_string(int code);
 int tm_version(void);

@@ -48,6 +48,8 @@ def load_library():
     lib.tm_device_status.argtypes = [ctypes.POINTER(i32)]; lib.tm_device_status.restype = i32
     lib.tm_find_mask_batched.argtypes = [ctypes.POINTER(tm_problem), i32, i32, i32, i32, vp, sz, vp, vp]
     lib.tm_find_mask_batched.restype = i32
+    lib.tm_find_mask_batched_static.argtypes = [ctypes.POINTER(tm_problem), i32, i32, i32, i32, vp, vp]
+    lib.tm_find_mask_batched_static.restype = i32
     lib.tm_workspace_bytes.argtypes = [ctypes.POINTER(tm_problem), i32]; lib.tm_workspace_bytes.restype = sz
     lib.tm_find_mask_host.argtypes = [vp, i32, i64, i64, i32, i32, i32, vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
     lib.tm_find_mask_host.restype = i32
@@ -187,6 +189,24 @@ def tm_find_mask_batched(Ws: Sequence, N: int, M: int, method: int, masks=None, 
         _check(lib.tm_find_mask_batched(arr, len(Ws), N, M, method, _ptr(workspace), workspace.numel(), _ptr(status),
                                         ctypes.c_void_p(s.cuda_stream)))
     return masks, maskeds, objectives, status, workspace
+
+
+TM_STATIC_MAX_MATRICES = 16
+
+
+def tm_find_mask_batched_static(Ws: Sequence, N: int, M: int, method: int, masks, maskeds, objectives, status, stream=None):
+    """tm_find_mask_batched() for callers that must not allocate device memory (a plug-in inside another
+    framework's memory pool, a pre-allocated real-time loop): the library's built-in scratch replaces the
+    workspace, at most TM_STATIC_MAX_MATRICES matrices per call.  Every output tensor is passed in (masks:
+    list of int32 [rows, wpr]; maskeds: list of tensors shaped like W, or None; objectives: float64[count];
+    status: int32[1]); this function creates no tensor.  Calls that overlap on the GPU race on the scratch."""
+    import torch
+    lib = load_library()
+    dev = Ws[0].device if len(Ws) else torch.device("cuda")
+    arr = _problem_array(Ws, masks, maskeds, objectives)
+    with torch.cuda.device(dev):
+        s = stream if stream is not None else torch.cuda.current_stream(dev)
+        _check(lib.tm_find_mask_batched_static(arr, len(Ws), N, M, method, _ptr(status), ctypes.c_void_p(s.cuda_stream)))
 
 
 def tm_find_mask_host(W, N: int, M: int, method: int, mask_out=None, masked_w_out=None, want_masked: bool = True,

@@ -190,6 +190,34 @@ int grow(void** p, size_t* have, size_t want) {
     return TM_OK;
 }
 
+// ---- built-in scratch of tm_find_mask_batched_static() ------------------------------------------
+// In host code the array's name is only a handle for the runtime, not a device address: the
+// address the kernels may use comes from cudaGetSymbolAddress(), looked up once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[TM_STATIC_SCRATCH_BYTES];
+
+struct StaticScratch {
+    bool ready = false;
+    void* ptr = nullptr;
+};
+StaticScratch g_static[kMaxDevices];
+
+int static_scratch_address(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return TM_ERR_CUDA; }
+    StaticScratch& s = g_static[dev];
+    if (!s.ready) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!s.ready) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return TM_ERR_CUDA; }
+            s.ptr = p;
+            s.ready = true;
+        }
+    }
+    *out = s.ptr;
+    return TM_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -322,6 +350,26 @@ int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols,
     return TM_OK;
 }
 
+int tm_find_mask_batched_static(const tm_problem* probs_host, int count, int N, int M, int method,
+                                int* status_dev, void* cuda_stream) {
+    int rc;
+    if ((rc = check_nm(N, M)) != TM_OK) return rc;
+    if ((rc = check_method(method)) != TM_OK) return rc;
+    if (count < 0) return TM_ERR_SHAPE;
+    if (count > TM_STATIC_MAX_MATRICES) return TM_ERR_TOO_LARGE;
+    if (count > 0 && !probs_host) return TM_ERR_NULL;
+    for (int k = 0; k < count; ++k)
+        if ((rc = check_problem(probs_host[k], M)) != TM_OK) return rc;
+    if (count == 0) return TM_OK;
+    if (tm_workspace_bytes(probs_host, TM_STATIC_MAX_MATRICES) > (size_t)TM_STATIC_SCRATCH_BYTES) return TM_ERR_WORKSPACE;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != TM_OK) return rc;
+    void* scratch = nullptr;
+    if ((rc = static_scratch_address(&scratch)) != TM_OK) return rc;
+    // every launch below clears the objective partials it uses before its kernel runs on the same stream
+    return run(probs_host, count, N, M, method, scratch, TM_STATIC_SCRATCH_BYTES, status_dev, static_cast<cudaStream_t>(cuda_stream), *d);
+}
+
 const char* tm_status_string(int code) {
     switch (code) {
     case TM_OK: return "ok";
@@ -333,6 +381,7 @@ const char* tm_status_string(int code) {
     case TM_ERR_ALIGN: return "misaligned pointer or row pitch";
     case TM_ERR_CUDA: return "CUDA runtime error (no device, launch or allocation failure)";
     case TM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case TM_ERR_TOO_LARGE: return "too many matrices for the built-in scratch (TM_STATIC_MAX_MATRICES per call)";
     default: return "unknown status";
     }
 }

@@ -49,8 +49,8 @@ def test_version_and_sizes(lib):
 
 
 def test_status_strings(lib):
-    seen = {tm.tm_status_string(c) for c in range(9)}
-    assert len(seen) == 9 and "ok" in seen
+    seen = {tm.tm_status_string(c) for c in range(10)}
+    assert len(seen) == 10 and "ok" in seen
     assert tm.tm_status_string(12345) == "unknown status"
 
 
