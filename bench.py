@@ -251,6 +251,55 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_survey(args):
+    """Secondary measurements (one JSON line per case): every named workload x method through the batched call.
+    Small workloads are L2-resident across repeats, so their GB/s is not an HBM figure; it is labelled so."""
+    import torch
+
+    import paper_2102_08124_b200 as tm
+    from paper_2102_08124_b200 import build as tm_build
+    tm_build.build()
+    torch.cuda.set_device(0)
+    peak, _ = measured_peak()
+    cases = [("config1 256x256 fp32", workloads.config1, 2, 4, ["approx", "cover", "exact"]),
+             ("config2 ResNet-50-shaped, 54 matrices fp32", workloads.config2, 2, 4, ["approx", "exact"]),
+             ("config3 BERT-large-shaped, 96 matrices bf16", workloads.config3, 2, 4, ["approx"]),
+             ("config4 8192x8192 fp32 Laplace", workloads.config4, 4, 8, ["approx", "cover", "exact"]),
+             ("config5 12288x49152 bf16 quantised", workloads.config5, 2, 4, ["approx", "cover", "exact"])]
+    methods = {"approx": tm.TM_APPROX, "cover": tm.TM_APPROX_COVER, "exact": tm.TM_EXACT}
+    for name, gen, N, M, ms in cases:
+        if args.config and not name.startswith("config%d" % args.config):
+            continue
+        mats = gen()
+        Ws = [torch.from_numpy(m.view(np.int16)).cuda().view(torch.bfloat16) if m.dtype == np.uint16 else torch.from_numpy(m).cuda() for m in mats]
+        weights = sum(int(m.size) for m in mats)
+        bpw = sum(m.size * (2 * m.itemsize + 0.125) for m in mats) / weights
+        masks, maskeds, objs, status, ws = tm.tm_find_mask_batched(Ws, N, M, tm.TM_APPROX)
+        for mname in ms:
+            meth = methods[mname]
+            def step():
+                tm.tm_find_mask_batched(Ws, N, M, meth, masks=masks, maskeds=maskeds, objectives=objs, workspace=ws, status=status)
+            for _ in range(3):
+                step()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter(); step(); torch.cuda.synchronize(); once = time.perf_counter() - t0
+            steps = max(3, min(200, int(0.5 / max(once, 1e-5))))
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                step()
+            e1.record(); torch.cuda.synchronize()
+            msec = e0.elapsed_time(e1) / steps
+            gbs = weights * bpw / (msec * 1e-3) / 1e9
+            print(json.dumps({"workload": name, "N": N, "M": M, "method": mname, "matrices": len(mats), "weights": weights,
+                              "ms_per_call": msec, "weights_per_s": weights / (msec * 1e-3), "algorithmic_GBps": gbs,
+                              "frac_of_measured_hbm": gbs / peak, "steps": steps,
+                              "resident_in_l2": bool(weights * bpw < 100e6), "status": int(status.item()),
+                              "objective_sum": float(objs.sum().item())}), flush=True)
+        del Ws, masks, maskeds, objs, ws
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -262,8 +311,12 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--skip-clocks", action="store_true", help="no nvidia-smi sampling and no extended warm-up")
+    ap.add_argument("--survey", action="store_true", help="secondary table: all named workloads and methods, one JSON line each")
+    ap.add_argument("--config", type=int, default=0, help="with --survey: only this workload (1..5)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.survey:
+        run_survey(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

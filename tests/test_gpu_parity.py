@@ -178,3 +178,87 @@ def test_host_buffer_entry_point(dtype):
             got_masked = masked.view(torch.int16).numpy().view(np.uint16) if dtype == "bf16" else masked.numpy().view(np.uint32)
             assert np.array_equal(got_masked, want["masked"].view(got_masked.dtype))
             assert abs(obj - want["objective"]) <= 1e-6 * want["objective"]
+
+
+# ----------------------------------------------------------------------------------------------
+# Full-size workloads, in the launch configuration the benchmark times
+# ----------------------------------------------------------------------------------------------
+def _check_line_sums(bits, N, M):
+    r, c = bits.shape
+    b = bits.reshape(r // M, M, c // M, M)
+    assert (b.sum(axis=1) == N).all() and (b.sum(axis=3) == N).all()
+
+
+def test_config5_full_size_sampled_strips():
+    """12288 x 49152 bf16 (the benchmark's workload): invariants on every block, bit parity on sampled row strips."""
+    W = workloads.config5()[0]
+    Wd = to_device(W)
+    mask, masked, obj = tm.tm_find_mask_bf16(Wd, 2, 4, tm.TM_APPROX)
+    torch.cuda.synchronize()
+    assert tm.tm_device_status() == 0
+    rng = np.random.Generator(np.random.PCG64(55))
+    strips = sorted(set([0, 12288 // 4 - 1] + [int(x) for x in rng.integers(0, 12288 // 4, size=22)]))
+    for s in strips:
+        rows = slice(4 * s, 4 * s + 4)
+        want = orc.find_mask(np.ascontiguousarray(W[rows]), 2, 4, orc.APPROX)
+        assert np.array_equal(to_host_bits(mask[rows]), want["mask"]), s
+        assert np.array_equal(to_host_bits(masked[rows]), want["masked"].view(np.uint16)), s
+    # properties that hold at any size: exactly two kept per line, masked = W where kept else +0, objective = sum |masked|
+    for r0 in range(0, 12288, 2048):
+        m = to_host_bits(mask[r0:r0 + 2048])
+        bits = orc.unpack_mask(m, 49152)
+        _check_line_sums(bits, 2, 4)
+        got = to_host_bits(masked[r0:r0 + 2048])
+        assert np.array_equal(got, np.where(bits == 1, W[r0:r0 + 2048], 0).astype(np.uint16))
+    total = float(workloads.bf16_bits_to_f32(to_host_bits(masked)).astype(np.float64).__abs__().sum())
+    assert abs(float(obj.item()) - total) <= 1e-6 * total
+
+
+def test_config3_full_size_whole_model():
+    """96 BERT-large-shaped bf16 matrices in one batched call; every matrix checked against the oracle."""
+    mats = workloads.config3()
+    Ws = [to_device(m) for m in mats]
+    masks, maskeds, objs, status, ws = tm.tm_find_mask_batched(Ws, 2, 4, tm.TM_APPROX)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for k, m in enumerate(mats):
+        want = orc.find_mask(m, 2, 4, orc.APPROX, threads=orc.max_threads(), want_masked=False)
+        assert np.array_equal(to_host_bits(masks[k]), want["mask"]), k
+        assert abs(float(objs[k].item()) - want["objective"]) <= 1e-6 * want["objective"], k
+    # a later simulated step: the perturbed weights give different masks, still bit-identical to the oracle
+    mats2 = workloads.config3_perturbed(mats[:4], 1)
+    Ws2 = [to_device(m) for m in mats2]
+    masks2, _, _, status2, _ = tm.tm_find_mask_batched(Ws2, 2, 4, tm.TM_APPROX)
+    torch.cuda.synchronize()
+    for k, m in enumerate(mats2):
+        want = orc.find_mask(m, 2, 4, orc.APPROX, threads=orc.max_threads(), want_masked=False)
+        assert np.array_equal(to_host_bits(masks2[k]), want["mask"]), k
+        assert not np.array_equal(to_host_bits(masks2[k]), to_host_bits(masks[k]))
+
+
+def test_config4_full_size_4_8():
+    """8192 x 8192 fp32 Laplace, 4:8: approximate mask checked everywhere, exact mask on sampled block rows,
+    exact >= approximate per block everywhere; the kept-mass gap is reported by the benchmark."""
+    W = workloads.config4()[0]
+    Wd = to_device(W)
+    am, amasked, aobj = tm.tm_find_mask(Wd, 4, 8, tm.TM_APPROX)
+    em, emasked, eobj = tm.tm_find_mask(Wd, 4, 8, tm.TM_EXACT)
+    torch.cuda.synchronize()
+    assert tm.tm_device_status() == 0
+    want = orc.find_mask(W, 4, 8, orc.APPROX, threads=orc.max_threads(), want_masked=False)
+    assert np.array_equal(to_host_bits(am), want["mask"])
+    assert abs(float(aobj.item()) - want["objective"]) <= 1e-6 * want["objective"]
+    ebits = orc.unpack_mask(to_host_bits(em), 8192)
+    abits = orc.unpack_mask(to_host_bits(am), 8192)
+    _check_line_sums(ebits, 4, 8); _check_line_sums(abits, 4, 8)
+    mag = np.abs(W.astype(np.float64))
+    eb = (mag * ebits).reshape(1024, 8, 1024, 8).sum(axis=(1, 3))
+    ab = (mag * abits).reshape(1024, 8, 1024, 8).sum(axis=(1, 3))
+    assert (eb >= ab * (1 - 1e-12)).all()
+    rng = np.random.Generator(np.random.PCG64(44))
+    for s in sorted(set([0, 1023] + [int(x) for x in rng.integers(0, 1024, size=4)])):
+        rows = slice(8 * s, 8 * s + 8)
+        w2 = orc.find_mask(np.ascontiguousarray(W[rows]), 4, 8, orc.EXACT, threads=orc.max_threads())
+        assert np.array_equal(to_host_bits(em[rows]), w2["mask"]), s
+        assert np.array_equal(to_host_bits(emasked[rows]), w2["masked"].view(np.uint32)), s
+    assert float(eobj.item()) >= float(aobj.item())
