@@ -85,7 +85,8 @@ __device__ __forceinline__ const DevProblem& find_problem(const DevProblem* tabl
 }
 
 template <int N, int M, int METHOD>
-__global__ void __launch_bounds__(kWarpsPerCta * 32)
+// the exact 2:4 scorer is register-hungry: two CTAs per SM cap it at 128 registers (its rare wide-integer path spills)
+__global__ void __launch_bounds__(kWarpsPerCta * 32, (METHOD == kMethodExact && M == 4) ? 2 : 1)
 generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, int count, long long total_items,
                double* __restrict__ partials, int* __restrict__ status_out) {
     const int lane = threadIdx.x & 31;
@@ -127,7 +128,7 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
 
         uint64_t kept;
         if constexpr (METHOD == kMethodExact) {
-            if constexpr (M == 4) kept = exact_2_4(u);
+            if constexpr (M == 4) kept = exact_2_4(u, P.dtype == kBF16 ? 16 : 0);
             else kept = exact_ssp<N, M>(u, status);
         } else {
             kept = cover_mask<N, M>(u);

@@ -258,12 +258,76 @@ __device__ __forceinline__ uint64_t exact_2_4_scored(const uint32_t (&u)[16], in
 }
 
 __device__ __noinline__ uint64_t exact_2_4_wide(const uint32_t (&u)[16], int Emin) { return exact_2_4_scored<Wide>(u, Emin); }
+__device__ __noinline__ uint64_t exact_2_4_int64(const uint32_t (&u)[16], int Emin) { return exact_2_4_scored<long long>(u, Emin); }
 
-__device__ __forceinline__ uint64_t exact_2_4(const uint32_t (&u)[16]) {
+// Fast scorer.  A row keeps one of six column pairs {a,b} (index b(b-1)/2 + a, the order of
+// kRowChoice).  value(row i, pair) = (q_a + q_b) * 2^16 + (nibble << 4i): the mask code rides in the
+// low 16 bits, so one integer maximum implements "larger sum, then larger code".  The 90 patterns
+// split by what rows 0,1 leave for rows 2,3:
+//   both rows take the same pair k        -> rows 2,3 both take the complementary pair      (6 cases)
+//   they take complementary pairs         -> rows 2,3 take any complementary pairs          (1 case, 6 x 6)
+//   they share column c and skip column d -> rows 2,3 share d and skip c                    (12 cases, 2 x 2)
+// so 19 sums of a best upper half and a best lower half cover everything.
+__host__ __device__ constexpr int pair_index(int a, int b) { return a < b ? b * (b - 1) / 2 + a : a * (a - 1) / 2 + b; }
+// the n-th (n = 0, 1) column that is neither c nor d
+__host__ __device__ constexpr int other_column(int c, int d, int n) {
+    int x = 0;
+    for (int k = 0; k < 4; ++k)
+        if (k != c && k != d) { if (n == 0) { x = k; break; } --n; }
+    return x;
+}
+
+template <int C, int D>
+__device__ __forceinline__ unsigned long long shared_column_case(const unsigned long long (&v)[4][6]) {
+    constexpr int a = other_column(C, D, 0), b = other_column(C, D, 1);
+    constexpr int ca = pair_index(C, a), cb = pair_index(C, b), da = pair_index(D, a), db = pair_index(D, b);
+    const unsigned long long up = max(v[0][ca] + v[1][cb], v[0][cb] + v[1][ca]);
+    const unsigned long long lo = max(v[2][da] + v[3][db], v[2][db] + v[3][da]);
+    return up + lo;
+}
+
+__device__ __forceinline__ uint64_t exact_2_4_classes(const uint32_t (&u)[16], int Emin, int drop_bits) {
+    unsigned long long v[4][6];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        unsigned long long q[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t sig; int E; split_float(u[i * 4 + j], sig, E);
+            q[j] = sig ? ((unsigned long long)(sig >> drop_bits) << (E - Emin + 16)) : 0ull;
+        }
+#pragma unroll
+        for (int b = 1; b < 4; ++b)
+#pragma unroll
+            for (int a = 0; a < b; ++a)
+                v[i][pair_index(a, b)] = q[a] + q[b] + ((unsigned long long)((1u << a) | (1u << b)) << (4 * i));
+    }
+    unsigned long long best = 0;
+    // same pair twice / complementary pairs
+    unsigned long long up_c = 0, lo_c = 0;
+#pragma unroll
+    for (int k = 0; k < 6; ++k) {
+        best = max(best, v[0][k] + v[1][k] + v[2][5 - k] + v[3][5 - k]);
+        up_c = max(up_c, v[0][k] + v[1][5 - k]);
+        lo_c = max(lo_c, v[2][k] + v[3][5 - k]);
+    }
+    best = max(best, up_c + lo_c);
+    // shared column c, skipped column d
+    best = max(best, max(max(shared_column_case<0, 1>(v), shared_column_case<0, 2>(v)), shared_column_case<0, 3>(v)));
+    best = max(best, max(max(shared_column_case<1, 0>(v), shared_column_case<1, 2>(v)), shared_column_case<1, 3>(v)));
+    best = max(best, max(max(shared_column_case<2, 0>(v), shared_column_case<2, 1>(v)), shared_column_case<2, 3>(v)));
+    best = max(best, max(max(shared_column_case<3, 0>(v), shared_column_case<3, 1>(v)), shared_column_case<3, 2>(v)));
+    return best & 0xFFFFull;
+}
+
+// drop_bits: low significand bits known to be zero in every entry (16 for widened bf16 inputs)
+__device__ __forceinline__ uint64_t exact_2_4(const uint32_t (&u)[16], int drop_bits) {
     int Emin, Emax;
     if (!exponent_range<16>(u, Emin, Emax)) { Emin = 1; Emax = 1; }     // all zero: every sum is 0, the largest code wins
-    // 24 significand bits + spread + 3 bits for eight terms must stay below 2^62
-    if (Emax - Emin <= 34) return exact_2_4_scored<long long>(u, Emin);
+    const int spread = Emax - Emin;
+    // (24 - drop) significand bits + spread + 3 bits for eight terms + 16 code bits must stay below 2^63
+    if (spread <= 19 + drop_bits) return exact_2_4_classes(u, Emin, drop_bits);
+    if (spread <= 34) return exact_2_4_int64(u, Emin);
     return exact_2_4_wide(u, Emin);
 }
 
