@@ -10,9 +10,9 @@
 //                   neither set finds both degrees full).
 //   complete_mask   this library's completion: greedy fill heavy -> light, then 2-for-1 swaps.
 //   exact_2_4       the optimum of Eq. 1 for M = 4 by scoring all 90 valid patterns.
-//   exact_ssp       the optimum for any M <= 8 by successive shortest paths on the flow network of
+//   exact_ssp       the optimum for any M <= 8 by shortest augmenting paths on the flow network of
 //                   Fig. 3 (rows supply M-N units, columns demand M-N, unit-capacity coefficient
-//                   edges; a unit on (i,j) prunes W_ij).
+//                   edges; a unit on (i,j) prunes W_ij), started from a row-feasible pseudo-flow.
 //
 // Exact arithmetic.  |w_p| = sig_p * 2^(E_p - 150); with Emin the smallest exponent among the
 // block's non-zero entries, q_p = sig_p << (E_p - Emin) is an integer proportional to |w_p|.  When
@@ -332,7 +332,7 @@ __device__ __forceinline__ uint64_t exact_2_4(const uint32_t (&u)[16], int drop_
 }
 
 // ------------------------------------------------------------------------------------------
-// Exact, any M <= 8: successive shortest paths on the network of Fig. 3
+// Exact, any M <= 8: min-cost flow on the network of Fig. 3
 // ------------------------------------------------------------------------------------------
 // Cost of the coefficient edge of entry p: q_p * 2^64 + 2^p (the tie rule folded into the cost:
 // minimising the pruned cost maximises (sum of kept |w|, code)).
@@ -360,55 +360,77 @@ template <> struct CostOps<CostWide> {
     }
 };
 
+// Min-cost flow by repairing a pseudo-flow: start from the state in which every row prunes its M-N
+// lightest entries (row supplies met, optimality conditions met with row potentials at the cost of the
+// row's (M-N)-th lightest entry), then repair the column imbalances -- a handful of units instead of
+// M(M-N) -- by shortest paths from over-subscribed to under-subscribed columns (Dijkstra on reduced
+// costs, which stay non-negative).  Costs are the exact integers of Fig. 3's coefficient edges with
+// the tie rule folded in, so the result is the unique optimum whatever path is taken among equals.
 template <class C, int N, int M>
-__device__ __noinline__ uint64_t exact_ssp_run(const uint32_t (&u)[M * M], int Emin, int& status) {
+__device__ __noinline__ uint64_t exact_flow_run(const uint32_t (&u)[M * M], int Emin, int& status) {
     using Ops = CostOps<C>;
-    C cost[M * M];
+    constexpr int P = M - N;
+    C cost[M * M], pot[2 * M];
     for (int p = 0; p < M * M; ++p) {
         uint32_t sig; int E; split_float(u[p], sig, E);
         cost[p] = Ops::edge(sig, sig ? E - Emin : 0, p);
     }
     uint64_t pruned = 0;
-    int supply[M], demand[M];
-    for (int i = 0; i < M; ++i) { supply[i] = M - N; demand[i] = M - N; }
-    for (int unit = 0; unit < M * (M - N); ++unit) {
-        // Bellman-Ford over the residual graph; nodes 0..M-1 rows, M..2M-1 columns
-        C dist[2 * M]; int pre[2 * M]; unsigned reach = 0;
-        for (int i = 0; i < M; ++i) if (supply[i] > 0) { dist[i] = Ops::zero(); pre[i] = -1; reach |= 1u << i; }
-        bool changed = true;
-        for (int round = 0; round < 2 * M + 1 && changed; ++round) {
-            changed = false;
-            for (int i = 0; i < M; ++i) {
-                if (!((reach >> i) & 1)) continue;
-                for (int j = 0; j < M; ++j) {
-                    if ((pruned >> (i * M + j)) & 1) continue;          // forward arc: prune (i,j)
-                    const C d = Ops::add(dist[i], cost[i * M + j]);
-                    if (!((reach >> (M + j)) & 1) || Ops::less(d, dist[M + j])) { dist[M + j] = d; pre[M + j] = i; reach |= 1u << (M + j); changed = true; }
-                }
-            }
-            for (int j = 0; j < M; ++j) {
-                if (!((reach >> (M + j)) & 1)) continue;
+    int load[M];
+    for (int j = 0; j < M; ++j) { load[j] = 0; pot[M + j] = Ops::zero(); }
+    for (int i = 0; i < M; ++i) {
+        for (int j = 0; j < M; ++j) {
+            int heavier = 0;
+            for (int k = 0; k < M; ++k)
+                heavier += (k != j) && (u[i * M + k] > u[i * M + j] || (u[i * M + k] == u[i * M + j] && k > j));
+            if (heavier >= N) { pruned |= 1ull << (i * M + j); load[j]++; }
+            if (heavier == N) pot[i] = Ops::neg(cost[i * M + j]);      // reduced cost c + pot[row] - pot[col]: <= 0 pruned, >= 0 kept
+        }
+    }
+    for (int unit = 0; unit <= M * P; ++unit) {
+        unsigned reach = 0, done = 0;
+        C dist[2 * M]; int pre[2 * M];
+        for (int j = 0; j < M; ++j)
+            if (load[j] > P) { dist[M + j] = Ops::zero(); pre[M + j] = -1; reach |= 1u << (M + j); }
+        if (!reach) break;                                              // every column holds exactly M-N pruned entries
+        if (unit == M * P) { status |= kDevInternal; break; }
+        int target = -1;
+        for (int step = 0; step < 2 * M; ++step) {
+            int v = -1;
+            for (int n = 0; n < 2 * M; ++n)
+                if (((reach & ~done) >> n) & 1) { if (v < 0 || Ops::less(dist[n], dist[v])) v = n; }
+            if (v < 0) break;
+            done |= 1u << v;
+            if (v >= M && load[v - M] < P) { target = v; break; }
+            if (v >= M) {                                               // column: un-prune one of its pruned entries
+                const int j = v - M;
                 for (int i = 0; i < M; ++i) {
-                    if (!((pruned >> (i * M + j)) & 1)) continue;       // backward arc: un-prune (i,j)
-                    const C d = Ops::add(dist[M + j], Ops::neg(cost[i * M + j]));
-                    if (!((reach >> i) & 1) || Ops::less(d, dist[i])) { dist[i] = d; pre[i] = M + j; reach |= 1u << i; changed = true; }
+                    if (!((pruned >> (i * M + j)) & 1) || ((done >> i) & 1)) continue;
+                    const C nd = Ops::add(dist[v], Ops::add(Ops::add(pot[v], Ops::neg(pot[i])), Ops::neg(cost[i * M + j])));
+                    if (!((reach >> i) & 1) || Ops::less(nd, dist[i])) { dist[i] = nd; pre[i] = v; reach |= 1u << i; }
+                }
+            } else {                                                    // row: prune one more of its kept entries
+                const int i = v;
+                for (int j = 0; j < M; ++j) {
+                    if (((pruned >> (i * M + j)) & 1) || ((done >> (M + j)) & 1)) continue;
+                    const C nd = Ops::add(dist[v], Ops::add(Ops::add(pot[i], Ops::neg(pot[M + j])), cost[i * M + j]));
+                    if (!((reach >> (M + j)) & 1) || Ops::less(nd, dist[M + j])) { dist[M + j] = nd; pre[M + j] = i; reach |= 1u << (M + j); }
                 }
             }
         }
-        if (changed) status |= kDevInternal;                           // a negative cycle cannot exist
-        int sink = -1;
-        for (int j = 0; j < M; ++j)
-            if (demand[j] > 0 && ((reach >> (M + j)) & 1) && (sink < 0 || Ops::less(dist[M + j], dist[M + sink]))) sink = j;
-        if (sink < 0) { status |= kDevInternal; break; }
-        int v = M + sink, steps = 0;
-        demand[sink]--;
-        while (pre[v] >= 0 && steps++ < 2 * M + 2) {                     // walk back, toggling arcs
+        if (target < 0) { status |= kDevInternal; break; }
+        const C D = dist[target];
+        for (int n = 0; n < 2 * M; ++n)
+            pot[n] = Ops::add(pot[n], (((done >> n) & 1) && Ops::less(dist[n], D)) ? dist[n] : D);
+        int v = target, steps = 0;
+        load[target - M]++;
+        while (pre[v] >= 0 && steps++ < 2 * M + 2) {
             const int w = pre[v];
-            if (v >= M) pruned |= 1ull << (w * M + (v - M));            // row w -> column v-M
-            else pruned &= ~(1ull << (v * M + (w - M)));                // column w-M -> row v
+            if (v >= M) pruned |= 1ull << (w * M + (v - M));           // row w -> column v-M
+            else pruned &= ~(1ull << (v * M + (w - M)));               // column w-M -> row v
             v = w;
         }
-        if (v < M && pre[v] < 0) supply[v]--; else status |= kDevInternal;
+        if (v >= M && pre[v] < 0) load[v - M]--; else { status |= kDevInternal; break; }
     }
     const uint64_t all = (M == 8) ? ~0ull : ((1ull << (M * M)) - 1);
     return ~pruned & all;
@@ -418,9 +440,10 @@ template <int N, int M>
 __device__ __forceinline__ uint64_t exact_ssp(const uint32_t (&u)[M * M], int& status) {
     int Emin, Emax;
     if (!exponent_range<M * M>(u, Emin, Emax)) { Emin = 1; Emax = 1; }
-    // path costs add at most M*M signed terms: 24 + spread + 6 bits must stay below 2^62
-    if (Emax - Emin <= 31) return exact_ssp_run<Cost128, N, M>(u, Emin, status);
-    return exact_ssp_run<CostWide, N, M>(u, Emin, status);
+    // 128-bit costs: 64 tie bits + 24 significand bits + spread; paths (<= 2M arcs) and potentials (<= M(M-N)
+    // updates) add 4 + 5 bits, the sign one more
+    if (Emax - Emin <= 26) return exact_flow_run<Cost128, N, M>(u, Emin, status);
+    return exact_flow_run<CostWide, N, M>(u, Emin, status);
 }
 
 }  // namespace tmask
