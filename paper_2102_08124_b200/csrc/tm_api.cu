@@ -133,11 +133,11 @@ int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, 
             std::vector<char> entries(esz * (size_t)n + 128);
             char* eh = entries.data() + ((128 - (uintptr_t)entries.data() % 128) % 128);
             long long total = 0;
-            if (!tmask::tma_build_entries(group[g].data(), n, eh, &total)) return TM_ERR_CUDA;
+            if (!tmask::tma_build_entries(group[g].data(), n, eh, &total, M)) return TM_ERR_CUDA;
             tmask::TmaLaunch a;
             a.entries_host = eh; a.entries_dev = nullptr; a.count = n; a.total_items = total; a.partials = partials;
-            a.status = status_dev; a.dtype = (g - 1) / 2; a.method = method; a.has_out = ((g - 1) & 1) != 0; a.stream = stream;
-            const int wpc = tmask::tma_warps_per_cta(a.dtype);
+            a.status = status_dev; a.dtype = (g - 1) / 2; a.method = method; a.M = M; a.has_out = ((g - 1) & 1) != 0; a.stream = stream;
+            const int wpc = tmask::tma_warps_per_cta(a.dtype, M);
             const long long want = (total + wpc - 1) / wpc;
             const int cap = dev.sms < kPartialSlots / wpc ? dev.sms : kPartialSlots / wpc;
             a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));

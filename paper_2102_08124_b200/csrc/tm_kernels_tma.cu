@@ -17,6 +17,7 @@
 #include "tm_launch.h"
 #include "tm_pair_bf16.cuh"
 #include "tm_tma.cuh"
+#include "tm_tma_items.cuh"
 
 #include <cstring>
 
@@ -36,36 +37,6 @@ template <int DT> struct Geometry {
     static constexpr int kStageBytes = kItemRows * kRowPitch;
     // stages | mask bytes [batch][4][32] | kept [batch][32] | swap candidates [batch][32] | queue | barriers
     static constexpr int kWarpBytes = kStages * kStageBytes + kBatch * 128 + 2 * kBatch * 128 + 128 + 64 + 64;
-};
-
-struct alignas(128) TmaEntry {
-    CUtensorMap in, out;
-    DevProblem p;
-    int cchunks;       // items per block row (256 columns each)
-    int brows;         // block rows
-};
-static_assert(sizeof(TmaEntry) == 384 || sizeof(TmaEntry) == 512, "descriptor records stay 128-byte aligned in tables");
-
-// Walks the work items of a table of problems in order: problem k, block row bi, column chunk cj.
-struct Cursor {
-    int k, bi, cj, cchunks, brows;
-    __device__ __forceinline__ void load(const TmaEntry* tab, int count) {
-        while (k < count && (tab[k].brows == 0 || tab[k].cchunks == 0)) ++k;   // empty matrices have no items
-        if (k < count) { cchunks = tab[k].cchunks; brows = tab[k].brows; } else { cchunks = 1; brows = 1; }
-    }
-    __device__ __forceinline__ void seek(const TmaEntry* tab, int count, long long item) {
-        k = 0;
-        while (k + 1 < count && tab[k + 1].p.item_begin <= item) ++k;
-        load(tab, count);
-        const long long local = item - tab[k < count ? k : count - 1].p.item_begin;
-        bi = (int)(local / cchunks); cj = (int)(local - (long long)bi * cchunks);
-    }
-    __device__ __forceinline__ void advance(const TmaEntry* tab, int count) {
-        if (++cj == cchunks) {
-            cj = 0;
-            if (++bi == brows) { bi = 0; ++k; load(tab, count); }
-        }
-    }
 };
 
 // ------------------------------------------------------------------------------------------
@@ -368,33 +339,6 @@ reduce_tma_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __res
     if (threadIdx.x == 0 && P.objective) *P.objective = sm[0];
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess) { cudaGetLastError(); p = nullptr; }
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-bool encode_map(CUtensorMap* m, const void* base, int dtype, long long rows, long long cols, long long ld) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)ld * (dtype == kF32 ? 4 : 2)};
-    const cuuint32_t box[2] = {(cuuint32_t)kItemCols, (cuuint32_t)kItemRows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(m, dtype == kF32 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), dims, strides,
-              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int DT, int METHOD, bool HAS_OUT>
 cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntry* table) {
     using G = Geometry<DT>;
@@ -413,44 +357,33 @@ cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntr
 }  // namespace
 
 size_t tma_entry_bytes() { return sizeof(TmaEntry); }
-int tma_warps_per_cta(int dtype) { return dtype == kF32 ? Geometry<kF32>::kWarps : Geometry<kBF16>::kWarps; }
+int tma_warps_per_cta(int dtype, int M) { return M == 8 ? tma48_warps_per_cta(dtype) : (dtype == kF32 ? Geometry<kF32>::kWarps : Geometry<kBF16>::kWarps); }
 
 bool tma_eligible(const DevProblem& p, int M, int method) {
-    if (M != 4 || (method != kMethodApprox && method != kMethodCover)) return false;
+    if ((M != 4 && M != 8) || (method != kMethodApprox && method != kMethodCover)) return false;
     const size_t elem = p.dtype == kF32 ? 4 : 2;
     if ((uintptr_t)p.W % 16 || ((size_t)p.ld * elem) % 16) return false;
     if (p.masked && (uintptr_t)p.masked % 16) return false;
     if (p.rows >= (1ll << 31) || p.cols >= (1ll << 31) - kItemCols || (size_t)p.ld * elem >= (1ull << 40)) return false;
-    if ((p.rows / kItemRows) * ((p.cols + kItemCols - 1) / kItemCols) >= (1ll << 30)) return false;
+    if ((p.rows / M) * ((p.cols + kItemCols - 1) / kItemCols) >= (1ll << 30)) return false;
     return encode_fn() != nullptr;
 }
 
-// Fills `entries_host` (count TmaEntry records) for problems that all passed tma_eligible().
-bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items) {
-    TmaEntry* e = static_cast<TmaEntry*>(entries_host);
-    long long total = 0;
-    for (int k = 0; k < count; ++k) {
-        memset(&e[k], 0, sizeof(TmaEntry));
-        e[k].p = probs[k];
-        e[k].cchunks = (int)((probs[k].cols + kItemCols - 1) / kItemCols);
-        e[k].brows = (int)(probs[k].rows / kItemRows);
-        e[k].p.item_begin = total;
-        total += (long long)e[k].brows * e[k].cchunks;
-        if (probs[k].rows == 0 || probs[k].cols == 0) continue;
-        if (!encode_map(&e[k].in, probs[k].W, probs[k].dtype, probs[k].rows, probs[k].cols, probs[k].ld)) return false;
-        if (probs[k].masked) {
-            if (!encode_map(&e[k].out, probs[k].masked, probs[k].dtype, probs[k].rows, probs[k].cols, probs[k].ld)) return false;
-        } else {
-            e[k].out = e[k].in;
-        }
-    }
-    *total_items = total;
-    return true;
+// Fills `entries_host` (count TmaEntry records) for problems that all passed tma_eligible(); an item is M rows x 256 columns.
+bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M) {
+    return build_entries(probs, count, static_cast<TmaEntry*>(entries_host), total_items, M, kItemCols);
+}
+
+cudaError_t tma_reduce(const void* entries_host, const void* entries_dev, int count, const double* partials, long long stride, cudaStream_t stream) {
+    const TmaEntry* host = static_cast<const TmaEntry*>(entries_host);
+    reduce_tma_kernel<<<count, 256, 0, stream>>>(host[0], static_cast<const TmaEntry*>(entries_dev), partials, stride);
+    return cudaGetLastError();
 }
 
 // All problems of one launch share dtype and the presence of masked_w_out (the caller groups them).
 cudaError_t launch_tma(const TmaLaunch& a) {
-    const int wpc = tma_warps_per_cta(a.dtype);
+    if (a.M == 8) return launch_tma48(a);
+    const int wpc = tma_warps_per_cta(a.dtype, 4);
     cudaError_t err = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * wpc, a.stream);
     if (err != cudaSuccess) return err;
     const TmaEntry* host = static_cast<const TmaEntry*>(a.entries_host);

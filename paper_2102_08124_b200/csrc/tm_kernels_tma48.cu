@@ -1,0 +1,394 @@
+// Bandwidth kernels of the approximate 4:8 search (TM_APPROX / TM_APPROX_COVER, M = 8).
+//
+// Same pipeline idea as the 2:4 kernels: every warp walks a contiguous range of work items (8 rows x
+// 256 columns of one matrix) with bulk-tensor (TMA) loads running ahead into a private ring of
+// shared-memory stages and TMA stores draining it; a lane owns one 8x8 block of the item.
+// The search itself is the bit-parallel core of tm_core48.cuh on 64-bit sets:
+//   front end  the 448 row/column comparisons of the block, collected into relation masks
+//              (bf16: two comparisons per 32-bit subtraction on packed magnitudes; fp32: scalar);
+//   step A     two bit-sliced counts;
+//   step B     warp-uniform rounds (a vote decides whether any lane still has candidates);
+//   step C     per lane: candidates from the relation masks, then the few magnitudes that must be
+//              compared are read back from the stage;
+//   back end   masked weights written into the stage and stored by TMA, mask bytes through shared
+//              memory as whole words, objective in fp32 per lane / fp64 across.
+#include "tm_core48.cuh"
+#include "tm_launch.h"
+#include "tm_pair_bf16.cuh"
+#include "tm_tma.cuh"
+#include "tm_tma_items.cuh"
+
+namespace tmask {
+
+namespace {
+
+constexpr int kRows8 = 8;
+constexpr int kCols8 = 256;
+
+template <int DT> struct Geo48 {
+    static constexpr int kElem = DT == kF32 ? 4 : 2;
+    static constexpr int kWarps = DT == kF32 ? 12 : 16;
+    static constexpr int kStages = DT == kF32 ? 2 : 3;
+    static constexpr int kRowPitch = kCols8 * kElem;
+    static constexpr int kStageBytes = kRows8 * kRowPitch;
+    static constexpr int kWarpBytes = kStages * kStageBytes + 256 /* mask bytes [8][32] */ + 64 /* barriers */ + 64;
+};
+
+__device__ __forceinline__ uint32_t max_u16x2_(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+// p[b] carries the decisions destined for bit 7-b of every byte (see gather8); only bits 0..3 wanted
+__device__ __forceinline__ uint32_t gather4_low(uint32_t p7, uint32_t p6, uint32_t p5, uint32_t p4) {
+    return bitsel(bitsel(p7 >> 7, p6 >> 6, 0x01010101u), bitsel(p5 >> 5, p4 >> 4, 0x04040404u), 0x03030303u);
+}
+
+// ---- bf16: packed comparisons ----------------------------------------------------------------
+// blk: row 0 of the lane's block inside the stage (row pitch 512 bytes)
+__device__ __forceinline__ void relations48_bf16(const unsigned char* blk, Rel48& rel, uint32_t& worst) {
+    uint32_t R[8][4];                              // R[i][c] = (|x_i,2c|, |x_i,2c+1|)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint4 v = *reinterpret_cast<const uint4*>(blk + i * 512);
+        R[i][0] = v.x & 0x7FFF7FFFu; R[i][1] = v.y & 0x7FFF7FFFu; R[i][2] = v.z & 0x7FFF7FFFu; R[i][3] = v.w & 0x7FFF7FFFu;
+        worst = max_u16x2_(worst, max_u16x2_(max_u16x2_(R[i][0], R[i][1]), max_u16x2_(R[i][2], R[i][3])));
+    }
+    // column relations hc[k]: bit (i,j) <- rows (i, i+k mod 8) of column j.  One subtraction decides two
+    // adjacent columns; byte permutes line the decisions up as (byte = row, top bit), a select tree packs them.
+#pragma unroll
+    for (int k = 1; k <= 4; ++k) {
+        uint32_t word[2] = {0, 0};
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            if (k == 4 && w == 1) continue;        // rows 4..7 of hc[4] follow by antisymmetry
+            uint32_t cw[8];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t d[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int i = 4 * w + r;
+                    d[r] = (i + k <= 7) ? later_heavier(R[(i + k) & 7][c], R[i][c]) : earlier_heavier(R[(i + k) & 7][c], R[i][c]);
+                }
+                const uint32_t q0 = prmt(d[0], d[1], 0x7351), q1 = prmt(d[2], d[3], 0x7351);
+                cw[2 * c] = prmt(q0, q1, 0x5410);
+                cw[2 * c + 1] = prmt(q0, q1, 0x7632);
+            }
+            const uint32_t p[8] = {cw[7], cw[6], cw[5], cw[4], cw[3], cw[2], cw[1], cw[0]};
+            word[w] = gather8(p);
+        }
+        rel.hc[k] = (u64)word[0] | ((u64)word[1] << 32);
+    }
+    // row relations hr[k]: rows 2i', 2i'+1 are paired, Y[i'][j] = (|x_2i',j|, |x_2i'+1,j|)
+    uint32_t Y[4][8];
+#pragma unroll
+    for (int ip = 0; ip < 4; ++ip)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            Y[ip][2 * c] = prmt(R[2 * ip][c], R[2 * ip + 1][c], 0x5410);
+            Y[ip][2 * c + 1] = prmt(R[2 * ip][c], R[2 * ip + 1][c], 0x7632);
+        }
+#pragma unroll
+    for (int k = 1; k <= 4; ++k) {
+        uint32_t word[2];
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            uint32_t pj[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (k == 4 && j >= 4) { pj[j] = 0; continue; }
+                const uint32_t d0 = (j + k <= 7) ? later_heavier(Y[2 * w][(j + k) & 7], Y[2 * w][j]) : earlier_heavier(Y[2 * w][(j + k) & 7], Y[2 * w][j]);
+                const uint32_t d1 = (j + k <= 7) ? later_heavier(Y[2 * w + 1][(j + k) & 7], Y[2 * w + 1][j]) : earlier_heavier(Y[2 * w + 1][(j + k) & 7], Y[2 * w + 1][j]);
+                pj[j] = prmt(d0, d1, 0x7531);      // bytes = rows 4w .. 4w+3 of column j
+            }
+            if (k == 4) {
+                word[w] = gather4_low(pj[0], pj[1], pj[2], pj[3]);
+            } else {
+                const uint32_t p[8] = {pj[7], pj[6], pj[5], pj[4], pj[3], pj[2], pj[1], pj[0]};
+                word[w] = gather8(p);
+            }
+        }
+        rel.hr[k] = (u64)word[0] | ((u64)word[1] << 32);
+    }
+    complete_relations8(rel);
+}
+
+// ---- fp32: scalar comparisons ------------------------------------------------------------------
+__device__ __forceinline__ void relations48_f32(const unsigned char* blk, Rel48& rel, uint32_t& worst) {
+    uint32_t u[64];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint4 a = *reinterpret_cast<const uint4*>(blk + i * 1024), b = *reinterpret_cast<const uint4*>(blk + i * 1024 + 16);
+        u[8 * i] = a.x & 0x7FFFFFFFu; u[8 * i + 1] = a.y & 0x7FFFFFFFu; u[8 * i + 2] = a.z & 0x7FFFFFFFu; u[8 * i + 3] = a.w & 0x7FFFFFFFu;
+        u[8 * i + 4] = b.x & 0x7FFFFFFFu; u[8 * i + 5] = b.y & 0x7FFFFFFFu; u[8 * i + 6] = b.z & 0x7FFFFFFFu; u[8 * i + 7] = b.w & 0x7FFFFFFFu;
+    }
+#pragma unroll
+    for (int p = 0; p < 64; ++p) worst = max(worst, u[p]);
+#pragma unroll
+    for (int k = 1; k <= 4; ++k) {
+        uint32_t rw[2] = {0, 0}, cw[2] = {0, 0};
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int bit = 8 * (i & 3) + j;
+                if (!(k == 4 && j >= 4)) {
+                    const int jj = (j + k) & 7;          // later position: ties count as heavier
+                    const bool h = (j + k <= 7) ? (u[8 * i + jj] >= u[8 * i + j]) : (u[8 * i + jj] > u[8 * i + j]);
+                    rw[i >> 2] |= (h ? 1u : 0u) << bit;
+                }
+                if (!(k == 4 && i >= 4)) {
+                    const int ii = (i + k) & 7;
+                    const bool h = (i + k <= 7) ? (u[8 * ii + j] >= u[8 * i + j]) : (u[8 * ii + j] > u[8 * i + j]);
+                    cw[i >> 2] |= (h ? 1u : 0u) << bit;
+                }
+            }
+        rel.hr[k] = (u64)rw[0] | ((u64)rw[1] << 32);
+        rel.hc[k] = (u64)cw[0] | ((u64)cw[1] << 32);
+    }
+    complete_relations8(rel);
+}
+
+// magnitude pattern of entry p of the lane's block, read back from the stage
+template <int DT>
+__device__ __forceinline__ uint32_t key_at(const unsigned char* blk, int p) {
+    if constexpr (DT == kBF16) return *reinterpret_cast<const unsigned short*>(blk + (p >> 3) * 512 + (p & 7) * 2) & 0x7FFFu;
+    else return *reinterpret_cast<const uint32_t*>(blk + (p >> 3) * 1024 + (p & 7) * 4) & 0x7FFFFFFFu;
+}
+
+// Step C, scalar half (see swap_apply8): set bits are visited in ascending position.
+template <int DT>
+__device__ __forceinline__ bool swap_apply8_smem(const unsigned char* blk, u64& kept, u64 cands, u64 free_a, u64 free_b) {
+    if (!cands) return false;
+    int x = -1; uint32_t best = 0;
+    for (int n = 0; n < 64 && cands; ++n) {
+        const int p = __ffsll((long long)cands) - 1;
+        cands &= cands - 1;
+        const uint32_t kp = key_at<DT>(blk, p);
+        if (x < 0 || kp < best) { x = p; best = kp; }
+    }
+    const int r2 = x >> 3, c2 = x & 7;
+    u64 ca = free_a & (0x0101010101010101ull << c2), cb = free_b & (0xFFull << (8 * r2));
+    int a = -1, b = -1; uint32_t ka = 0, kb = 0;
+    for (int n = 0; n < 8 && ca; ++n) {
+        const int e = __ffsll((long long)ca) - 1; ca &= ca - 1;
+        const uint32_t k = key_at<DT>(blk, e);
+        if (a < 0 || k >= ka) { a = e; ka = k; }
+    }
+    for (int n = 0; n < 8 && cb; ++n) {
+        const int e = __ffsll((long long)cb) - 1; cb &= cb - 1;
+        const uint32_t k = key_at<DT>(blk, e);
+        if (b < 0 || k >= kb) { b = e; kb = k; }
+    }
+    if (a < 0 || b < 0) return false;
+    kept = (kept & ~(1ull << x)) | (1ull << a) | (1ull << b);
+    return true;
+}
+
+// Masked weights back into the stage, mask bytes, objective contribution of the lane's block.
+template <int DT, bool HAS_OUT>
+__device__ __forceinline__ float back_end48(unsigned char* blk, unsigned char* mrow /* [8][32] */, int lane, u64 kept) {
+    float s8 = 0.f;
+    const uint32_t kw[2] = {(uint32_t)kept, (uint32_t)(kept >> 32)};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t word = kw[i >> 2];
+        const int base = 8 * (i & 3);
+        if constexpr (DT == kBF16) {
+            const uint4 r = *reinterpret_cast<const uint4*>(blk + i * 512);
+            const uint32_t raw[4] = {r.x, r.y, r.z, r.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                // keep bits of columns 2c, 2c+1 -> top bit of a byte each -> 16-bit lane masks
+                const uint32_t sa = word << (31 - (base + 2 * c)), sb = word << (30 - (base + 2 * c));
+                const uint32_t m = prmt(sa, sb, 0xFFBB);
+                o[c] = raw[c] & m;
+                const uint32_t ab = raw[c] & m & 0x7FFF7FFFu;
+                unsigned short lo, hi;
+                asm("mov.b32 {%0,%1}, %2;" : "=h"(lo), "=h"(hi) : "r"(ab));
+                asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(s8) : "h"(lo));
+                asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(s8) : "h"(hi));
+            }
+            if constexpr (HAS_OUT) *reinterpret_cast<uint4*>(blk + i * 512) = make_uint4(o[0], o[1], o[2], o[3]);
+        } else {
+            const uint4 ra = *reinterpret_cast<const uint4*>(blk + i * 1024), rb = *reinterpret_cast<const uint4*>(blk + i * 1024 + 16);
+            const uint32_t raw[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+            uint32_t o[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                o[q] = ((word >> (base + q)) & 1u) ? raw[q] : 0u;
+                s8 += fabsf(__uint_as_float(o[q]));
+            }
+            if constexpr (HAS_OUT) {
+                *reinterpret_cast<uint4*>(blk + i * 1024) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4*>(blk + i * 1024 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+        }
+        mrow[i * 32 + lane] = (unsigned char)(word >> base);
+    }
+    return s8;
+}
+
+template <int DT, int METHOD, bool HAS_OUT>
+__global__ void __launch_bounds__(Geo48<DT>::kWarps * 32, 1)
+tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict__ table, int count, long long total_items,
+             double* __restrict__ partials, int* __restrict__ status_out) {
+    using G = Geo48<DT>;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned char* stages = smem_raw + (size_t)warp * G::kWarpBytes;
+    unsigned char* mbytes = stages + G::kStages * G::kStageBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(mbytes + 256);
+
+    const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
+    const long long per = (total_items + nwarps - 1) / nwarps;
+    const long long begin = gw * per, end = min(total_items, begin + per);
+    const int n_items = (int)max(0ll, end - begin);
+    const TmaEntry* tab = table ? table : &single;
+
+    if (lane == 0) {
+        for (int s = 0; s < G::kStages; ++s) mbar_init(&bars[s], 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+
+    Cursor ld, cur;
+    ld.seek(tab, count, begin);
+    cur = ld;
+    int loaded = 0;
+    auto issue_next = [&]() {              // all lanes track the cursor, lane 0 issues the copy
+        const int s = loaded % G::kStages;
+        if (lane == 0) {
+            mbar_expect_tx(&bars[s], G::kStageBytes);
+            tma_load_2d(stages + s * G::kStageBytes, &tab[ld.k].in, ld.cj * kCols8, ld.bi * kRows8, &bars[s]);
+        }
+        ld.advance(tab, count);
+        ++loaded;
+    };
+    for (int g = 0; g < G::kStages - 1 && loaded < n_items; ++g) issue_next();
+
+    int status = 0, acc_k = -1;
+    float facc = 0.f; double acc = 0.0;
+    uint32_t worst = 0;
+
+    for (int it = 0; it < n_items; ++it) {
+        const int s = it % G::kStages;
+        const uint32_t parity = (uint32_t)((it / G::kStages) & 1);
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bars[s], parity))) {
+            status |= kDevInternal;
+            if (lane == 0)                 // give the copies still in flight a bounded chance to land before the stages die
+                for (int j = it + 1; j < loaded; ++j) mbar_wait_bounded(&bars[j % G::kStages], (uint32_t)((j / G::kStages) & 1), 1u << 14);
+            break;
+        }
+        unsigned char* stage = stages + s * G::kStageBytes;
+        unsigned char* blk = stage + lane * (8 * G::kElem);
+
+        Rel48 rel;
+        if constexpr (DT == kBF16) relations48_bf16(blk, rel, worst); else relations48_f32(blk, rel, worst);
+        u64 kept = cover_4_8(rel);
+        if constexpr (METHOD == kMethodApprox) {
+            Lack48 L = line_lack(kept);
+            u64 cand = open_candidates8(kept, L);
+            int rounds = 0;
+            while (__any_sync(0xFFFFFFFFu, cand != 0)) {
+                if (++rounds > 16) { status |= kDevInternal; break; }      // a block lacks at most sixteen entries
+                kept |= fill_accept8(rel, L, cand);
+                L = line_lack(kept);
+                cand = open_candidates8(kept, L);
+            }
+            int swaps = 0;
+            while (__any_sync(0xFFFFFFFFu, L.row_short != 0)) {
+                if (++swaps > 5) { status |= kDevInternal; break; }       // at most N*N/4 = 4 swaps per block
+                if (L.row_short) {
+                    u64 fa, fb;
+                    const u64 c = swap_candidates8(rel, L, kept, fa, fb);
+                    if (!swap_apply8_smem<DT>(blk, kept, c, fa, fb)) { status |= kDevInternal; L.row_short = 0; }
+                    else L = line_lack(kept);
+                }
+            }
+        }
+        const TmaEntry& e = tab[cur.k];
+        if (cur.cj * kCols8 + lane * 8 >= (int)e.p.cols) kept = 0;       // blocks past the last column (zero-filled by the copy)
+
+        if (cur.k != acc_k) {                                              // a new matrix starts: flush the objective partial
+            if (acc_k >= 0) {
+                acc += (double)facc;
+                for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+                if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
+            }
+            acc = 0.0; facc = 0.f; acc_k = cur.k;
+        }
+        facc += back_end48<DT, HAS_OUT>(blk, mbytes, lane, kept);
+        if constexpr (HAS_OUT) fence_proxy_async_smem();
+        __syncwarp();
+        if constexpr (HAS_OUT) {
+            if (lane == 0) { tma_store_2d(&e.out, cur.cj * kCols8, cur.bi * kRows8, stage); tma_commit(); }
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {                                      // 8 rows x 8 words of mask
+            const int idx = lane + 32 * h, row = idx >> 3, word = cur.cj * 8 + (idx & 7);
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + row * 32 + (idx & 7) * 4);
+            if (word < e.p.wpr) e.p.mask[((long long)cur.bi * kRows8 + row) * e.p.wpr + word] = w;
+        }
+        // refill: the stage of the previous item is free once its store has been read
+        if (loaded < n_items) {
+            if constexpr (HAS_OUT) { if (lane == 0) tma_wait_read<1>(); }
+            __syncwarp();
+            issue_next();
+        }
+        cur.advance(tab, count);
+        if ((it & 15) == 15) { acc += (double)facc; facc = 0.f; }           // keep the fp32 partial short
+        __syncwarp();
+    }
+    if (lane == 0) tma_wait_all<0>();
+    if (acc_k >= 0) {
+        acc += (double)facc;
+        for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
+    }
+    if constexpr (DT == kF32) { if (worst >= 0x7F800000u) status |= kDevNonFinite; }
+    else { if ((worst & 0xFFFFu) >= 0x7F80u || (worst >> 16) >= 0x7F80u) status |= kDevNonFinite; }
+    for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(0xFFFFFFFFu, status, o);
+    if (lane == 0 && status && status_out) atomicOr(status_out, status);
+}
+
+template <int DT, int METHOD, bool HAS_OUT>
+cudaError_t launch_one48(const TmaLaunch& a, const TmaEntry& single, const TmaEntry* table) {
+    using G = Geo48<DT>;
+    const size_t smem = (size_t)G::kWarps * G::kWarpBytes;
+    auto kern = tma48_kernel<DT, METHOD, HAS_OUT>;
+    static bool configured = false;        // per instantiation
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int tma48_warps_per_cta(int dtype) { return dtype == kF32 ? Geo48<kF32>::kWarps : Geo48<kBF16>::kWarps; }
+
+cudaError_t launch_tma48(const TmaLaunch& a) {
+    const int wpc = tma48_warps_per_cta(a.dtype);
+    cudaError_t err = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * wpc, a.stream);
+    if (err != cudaSuccess) return err;
+    const TmaEntry* host = static_cast<const TmaEntry*>(a.entries_host);
+    const TmaEntry* table = static_cast<const TmaEntry*>(a.entries_dev);
+    if (a.total_items > 0) {
+#define TM_DISPATCH(DT, METHOD)                                                                                   \
+    err = a.has_out ? launch_one48<DT, METHOD, true>(a, host[0], table) : launch_one48<DT, METHOD, false>(a, host[0], table)
+        if (a.dtype == kF32) { if (a.method == kMethodApprox) TM_DISPATCH(kF32, kMethodApprox); else TM_DISPATCH(kF32, kMethodCover); }
+        else { if (a.method == kMethodApprox) TM_DISPATCH(kBF16, kMethodApprox); else TM_DISPATCH(kBF16, kMethodCover); }
+#undef TM_DISPATCH
+        if (err != cudaSuccess) return err;
+    }
+    return tma_reduce(a.entries_host, a.entries_dev, a.count, a.partials, (long long)a.ctas * wpc, a.stream);
+}
+
+}  // namespace tmask

@@ -30,14 +30,18 @@ struct TmaLaunch {
     double* partials;           // device scratch, count * ctas * tma_warps_per_cta(dtype) doubles
     int* status;
     int ctas;
-    int dtype, method;
+    int dtype, method, M;
     bool has_out;               // masked_w_out present (all problems of one launch agree)
     cudaStream_t stream;
 };
 size_t tma_entry_bytes();
-int tma_warps_per_cta(int dtype);
+int tma_warps_per_cta(int dtype, int M);
 bool tma_eligible(const DevProblem& p, int M, int method);
-bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items);
+bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M);
+cudaError_t tma_reduce(const void* entries_host, const void* entries_dev, int count, const double* partials, long long stride, cudaStream_t stream);
+// 4:8 variant (tm_kernels_tma48.cu), reached through launch_tma()
+int tma48_warps_per_cta(int dtype);
+cudaError_t launch_tma48(const TmaLaunch& a);
 cudaError_t launch_tma(const TmaLaunch& a);
 
 }  // namespace tmask

@@ -1,0 +1,91 @@
+// Work-item bookkeeping shared by the bandwidth kernels: one descriptor record per matrix (tensor maps
+// for loads and stores plus the problem), a cursor that walks the items of a table of matrices in
+// order, and the host-side construction of the records.  An item is M rows x 256 columns.
+#pragma once
+#include <cstring>
+
+#include "tm_device.cuh"
+#include "tm_tma.cuh"
+
+namespace tmask {
+
+struct alignas(128) TmaEntry {
+    CUtensorMap in, out;
+    DevProblem p;
+    int cchunks;       // items per block row (256 columns each)
+    int brows;         // block rows
+};
+static_assert(sizeof(TmaEntry) == 384 || sizeof(TmaEntry) == 512, "descriptor records stay 128-byte aligned in tables");
+
+// Walks the work items of a table of problems in order: problem k, block row bi, column chunk cj.
+struct Cursor {
+    int k, bi, cj, cchunks, brows;
+    __device__ __forceinline__ void load(const TmaEntry* tab, int count) {
+        while (k < count && (tab[k].brows == 0 || tab[k].cchunks == 0)) ++k;   // empty matrices have no items
+        if (k < count) { cchunks = tab[k].cchunks; brows = tab[k].brows; } else { cchunks = 1; brows = 1; }
+    }
+    __device__ __forceinline__ void seek(const TmaEntry* tab, int count, long long item) {
+        k = 0;
+        while (k + 1 < count && tab[k + 1].p.item_begin <= item) ++k;
+        load(tab, count);
+        const long long local = item - tab[k < count ? k : count - 1].p.item_begin;
+        bi = (int)(local / cchunks); cj = (int)(local - (long long)bi * cchunks);
+    }
+    __device__ __forceinline__ void advance(const TmaEntry* tab, int count) {
+        if (++cj == cchunks) {
+            cj = 0;
+            if (++bi == brows) { bi = 0; ++k; load(tab, count); }
+        }
+    }
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) { cudaGetLastError(); p = nullptr; }
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+inline bool encode_map(CUtensorMap* m, const void* base, int dtype, long long rows, long long cols, long long ld, int box_rows, int box_cols) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * (dtype == kF32 ? 4 : 2)};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, dtype == kF32 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), dims, strides,
+              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+
+inline bool build_entries(const DevProblem* probs, int count, TmaEntry* e, long long* total_items, int item_rows, int item_cols) {
+    long long total = 0;
+    for (int k = 0; k < count; ++k) {
+        memset(&e[k], 0, sizeof(TmaEntry));
+        e[k].p = probs[k];
+        e[k].cchunks = (int)((probs[k].cols + item_cols - 1) / item_cols);
+        e[k].brows = (int)(probs[k].rows / item_rows);
+        e[k].p.item_begin = total;
+        total += (long long)e[k].brows * e[k].cchunks;
+        if (probs[k].rows == 0 || probs[k].cols == 0) continue;
+        if (!encode_map(&e[k].in, probs[k].W, probs[k].dtype, probs[k].rows, probs[k].cols, probs[k].ld, item_rows, item_cols)) return false;
+        if (probs[k].masked) {
+            if (!encode_map(&e[k].out, probs[k].masked, probs[k].dtype, probs[k].rows, probs[k].cols, probs[k].ld, item_rows, item_cols)) return false;
+        } else {
+            e[k].out = e[k].in;
+        }
+    }
+    *total_items = total;
+    return true;
+}
+
+}  // namespace tmask
