@@ -265,7 +265,10 @@ def run_survey(args):
              ("config2 ResNet-50-shaped, 54 matrices fp32", workloads.config2, 2, 4, ["approx", "exact"]),
              ("config3 BERT-large-shaped, 96 matrices bf16", workloads.config3, 2, 4, ["approx"]),
              ("config4 8192x8192 fp32 Laplace", workloads.config4, 4, 8, ["approx", "cover", "exact"]),
-             ("config5 12288x49152 bf16 quantised", workloads.config5, 2, 4, ["approx", "cover", "exact"])]
+             ("config5 12288x49152 bf16 quantised", workloads.config5, 2, 4, ["approx", "cover", "exact"]),
+             # two more large cases, so that every (dtype, N:M) pair of the bandwidth kernels has an HBM-sized measurement
+             ("config6 (extra) 8192x8192 fp32 Laplace, 2:4", workloads.config4, 2, 4, ["approx", "cover"]),
+             ("config7 (extra) 12288x49152 bf16 quantised, 4:8", workloads.config5, 4, 8, ["approx", "cover"])]
     methods = {"approx": tm.TM_APPROX, "cover": tm.TM_APPROX_COVER, "exact": tm.TM_EXACT}
     for name, gen, N, M, ms in cases:
         if args.config and not name.startswith("config%d" % args.config):
@@ -274,11 +277,12 @@ def run_survey(args):
         Ws = [torch.from_numpy(m.view(np.int16)).cuda().view(torch.bfloat16) if m.dtype == np.uint16 else torch.from_numpy(m).cuda() for m in mats]
         weights = sum(int(m.size) for m in mats)
         bpw = sum(m.size * (2 * m.itemsize + 0.125) for m in mats) / weights
-        masks, maskeds, objs, status, ws = tm.tm_find_mask_batched(Ws, N, M, tm.TM_APPROX)
+        batch = tm.TmBatch(Ws)                    # descriptors marshalled once, as a training loop would
+        objs, status = batch.objectives, batch.status
         for mname in ms:
             meth = methods[mname]
             def step():
-                tm.tm_find_mask_batched(Ws, N, M, meth, masks=masks, maskeds=maskeds, objectives=objs, workspace=ws, status=status)
+                batch.run(N, M, meth)
             for _ in range(3):
                 step()
             torch.cuda.synchronize()
@@ -296,7 +300,7 @@ def run_survey(args):
                               "frac_of_measured_hbm": gbs / peak, "steps": steps,
                               "resident_in_l2": bool(weights * bpw < 100e6), "status": int(status.item()),
                               "objective_sum": float(objs.sum().item())}), flush=True)
-        del Ws, masks, maskeds, objs, ws
+        del Ws, batch, objs, status
         torch.cuda.empty_cache()
 
 

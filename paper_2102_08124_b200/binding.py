@@ -150,6 +150,50 @@ def _problem_array(Ws: Sequence, masks, maskeds, objectives):
     return arr
 
 
+class TmBatch:
+    """A list of matrices with their output tensors, marshalled once into the C descriptor array.
+
+    Filling the descriptors costs a few microseconds per matrix in Python; a training loop that re-derives the
+    masks of the same weight buffers every few iterations prepares the batch once and calls run() each time."""
+
+    def __init__(self, Ws: Sequence, masks=None, maskeds=None, objectives=None, workspace=None, status=None, want_masked: bool = True):
+        import torch
+        if len(Ws) == 0:
+            raise TmError(2, "empty batch")
+        dev = Ws[0].device
+        for W in Ws:
+            if not (W.is_cuda and W.dim() == 2 and (W.shape[1] <= 1 or W.stride(1) == 1) and W.device == dev):
+                raise TmError(2, "every W must be a 2-D CUDA tensor with unit column stride on one device")
+        if masks is None:
+            masks = [torch.empty((W.shape[0], tm_mask_words_per_row(W.shape[1])), dtype=torch.int32, device=dev) for W in Ws]
+        if maskeds is None and want_masked:
+            maskeds = [torch.empty_strided(W.shape, W.stride(), dtype=W.dtype, device=dev) for W in Ws]
+        if maskeds is not None:
+            for W, Y in zip(Ws, maskeds):                      # the ABI has one leading dimension per matrix
+                if Y is not None and (Y.shape != W.shape or Y.stride() != W.stride() or Y.dtype != W.dtype):
+                    raise TmError(2, "masked_w_out must have the shape, strides and dtype of W")
+        if objectives is None:
+            objectives = torch.empty((len(Ws),), dtype=torch.float64, device=dev)
+        if status is None:
+            status = torch.zeros((1,), dtype=torch.int32, device=dev)
+        if workspace is None:
+            workspace = torch.empty((tm_workspace_bytes(len(Ws)),), dtype=torch.uint8, device=dev)
+        self.Ws, self.masks, self.maskeds, self.objectives, self.status, self.workspace = list(Ws), masks, maskeds, objectives, status, workspace
+        self.device = dev
+        self.count = len(Ws)
+        self._arr = _problem_array(Ws, masks, maskeds, objectives)
+        self._lib = load_library()
+
+    def run(self, N: int, M: int, method: int, stream=None):
+        """tm_find_mask_batched on the prepared descriptors; asynchronous on `stream` or torch's current stream."""
+        import torch
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        with torch.cuda.device(self.device):
+            _check(self._lib.tm_find_mask_batched(self._arr, self.count, N, M, method, _ptr(self.workspace), self.workspace.numel(),
+                                                  _ptr(self.status), ctypes.c_void_p(s.cuda_stream)))
+        return self.masks, self.maskeds, self.objectives, self.status
+
+
 def tm_workspace_bytes(count: int) -> int:
     return int(load_library().tm_workspace_bytes(None, count))
 

@@ -133,6 +133,19 @@ def test_batched_mixed_dtypes_and_strides(method):
     _batched_parity(mats[:4], 2, 4, method, strided=True)
 
 
+def test_prepared_batch_object():
+    mats = [workloads.normal_f32(32, 264, 0.05, 61), workloads.normal_bf16(16, 520, 0.02, 62)]
+    batch = tm.TmBatch([to_device(m) for m in mats])
+    for method in (tm.TM_APPROX, tm.TM_EXACT, tm.TM_APPROX):          # the same descriptors serve repeated calls
+        masks, maskeds, objs, status = batch.run(2, 4, method)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for k, m in enumerate(mats):
+            want = orc.find_mask(m, 2, 4, method)
+            assert np.array_equal(to_host_bits(masks[k]), want["mask"]), k
+            assert abs(float(objs[k].item()) - want["objective"]) <= 1e-6 * want["objective"], k
+
+
 def test_batched_4_8():
     mats = [workloads.laplace_f32(32, 264, 0.05, 31), workloads.normal_bf16(16, 520, 0.02, 32)]
     for method in METHODS:
