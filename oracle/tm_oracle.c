@@ -416,6 +416,111 @@ int tmo_find_mask(const void* W, int dtype, int64_t rows, int64_t cols, int64_t 
     return TMO_OK;
 }
 
+/* ------------------------------------------------------------------------- */
+/* Neighbouring operations of Section 5 ("Structured sparsity without full training") */
+/* ------------------------------------------------------------------------- */
+static float bits_to_float(uint32_t b) { union { uint32_t b; float f; } c; c.b = b; return c.f; }
+static uint32_t float_to_bits(float f) { union { uint32_t b; float f; } c; c.f = f; return c.b; }
+/* raw value of element idx widened to fp32 (bf16 exactly) */
+static float elem_value(const void* W, int dtype, int64_t idx) {
+    if (dtype == TMO_F32) return ((const float*)W)[idx];
+    return bits_to_float(((uint32_t)((const uint16_t*)W)[idx]) << 16);
+}
+/* fp32 -> bf16, round to nearest even; NaN stays NaN */
+static uint16_t float_to_bf16(float f) {
+    uint32_t u = float_to_bits(f);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x40u);
+    return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+}
+
+/* 1-D N:M magnitude pruning (Section 5, "we prune [the] weights with the lowest magnitude" in every group of M
+ * contiguous weights of a row).  N = KEPT per group; order (|w|, position in the group), the later of equals is
+ * the heavier one.  violations = pruned entries that are non-zero ("pattern-violations": active weights the
+ * pattern removes).  absorb_mean ("mean absorption"): the mean of the group's pruned weights is added to every
+ * kept weight: mu = (sum of the pruned weights in position order, fp64) / (their number); kept' = fp64(kept + mu)
+ * rounded to fp32 (and then to bf16, nearest even, for bf16 tensors).  objective = sum of kept |w| (before absorption). */
+int tmo_nm_mask_1d(const void* W, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int M, int absorb_mean,
+                   uint32_t* mask_out, void* masked_w_out, double* objective_out, int64_t* violations_out) {
+    if (M < 1 || M > TMO_MAXM || N < 0 || N > M || rows < 0 || cols < 0 || cols % M || ld < cols) return TMO_ERR_ARG;
+    if (dtype != TMO_F32 && dtype != TMO_BF16) return TMO_ERR_ARG;
+    int64_t wpr = (cols + 31) / 32, viol = 0;
+    double total = 0.0, comp = 0.0;
+    if (mask_out) memset(mask_out, 0, (size_t)(rows * wpr) * sizeof(uint32_t));
+    for (int64_t r = 0; r < rows; ++r) for (int64_t g = 0; g < cols / M; ++g) {
+        uint32_t u[TMO_MAXM]; int kept[TMO_MAXM];
+        for (int j = 0; j < M; ++j) u[j] = mag_bits(W, dtype, r * ld + g * M + j);
+        for (int j = 0; j < M; ++j) {               /* kept iff fewer than N entries of the group are heavier */
+            int heavier = 0;
+            for (int k = 0; k < M; ++k) if (k != j && lighter(u, j, k)) heavier++;
+            kept[j] = heavier < N;
+        }
+        double psum = 0.0; int pcnt = 0;
+        for (int j = 0; j < M; ++j) if (!kept[j]) { psum += (double)elem_value(W, dtype, r * ld + g * M + j); pcnt++; viol += (u[j] != 0); }
+        double mu = (absorb_mean && pcnt) ? psum / (double)pcnt : 0.0;
+        for (int j = 0; j < M; ++j) {
+            int64_t c = g * M + j, idx = r * ld + c;
+            if (kept[j] && mask_out) mask_out[r * wpr + c / 32] |= 1u << (c % 32);
+            if (kept[j]) { double x = (double)bits_to_float(u[j]), t = total + x; comp += (total >= x) ? ((total - t) + x) : ((x - t) + total); total = t; }
+            if (masked_w_out) {
+                if (dtype == TMO_F32) {
+                    uint32_t raw = ((const uint32_t*)W)[idx];
+                    ((uint32_t*)masked_w_out)[idx] = !kept[j] ? 0u : (absorb_mean ? float_to_bits((float)((double)bits_to_float(raw) + mu)) : raw);
+                } else {
+                    uint16_t raw = ((const uint16_t*)W)[idx];
+                    ((uint16_t*)masked_w_out)[idx] = !kept[j] ? (uint16_t)0 :
+                        (absorb_mean ? float_to_bf16((float)((double)bits_to_float((uint32_t)raw << 16) + mu)) : raw);
+                }
+            }
+        }
+    }
+    if (objective_out) *objective_out = total + comp;
+    if (violations_out) *violations_out = viol;
+    return TMO_OK;
+}
+
+/* Pattern-violations of an arbitrary packed mask: entries whose mask bit is 0 although the weight is non-zero. */
+int tmo_mask_violations(const void* W, int dtype, int64_t rows, int64_t cols, int64_t ld, const uint32_t* mask, int64_t* violations_out) {
+    if (rows < 0 || cols < 0 || ld < cols || (dtype != TMO_F32 && dtype != TMO_BF16)) return TMO_ERR_ARG;
+    int64_t wpr = (cols + 31) / 32, viol = 0;
+    for (int64_t r = 0; r < rows; ++r) for (int64_t c = 0; c < cols; ++c)
+        if (!((mask[r * wpr + c / 32] >> (c % 32)) & 1u) && mag_bits(W, dtype, r * ld + c) != 0) viol++;
+    *violations_out = viol;
+    return TMO_OK;
+}
+
+/* 2:4 operand compression for W and its transpose from one transposable mask (Section 1 and Fig. 2: the same
+ * mask serves Y = W X and dL/dX = W^T dL/dY).  Row form: for every row and every group of 4 columns the two kept
+ * values in column order -> values[rows][cols/2]; their column indices inside the group, idx0 | idx1 << 2, as a
+ * nibble -> meta[rows][ceil(cols/32)] (group g of a row: bits 4*(g%8) of word g/8).  Column form: the same for
+ * W^T (groups of 4 rows of a column) -> values_t[cols][rows/2], meta_t[cols][ceil(rows/32)].
+ * A group that does not hold exactly two kept entries gets zeros and is counted in bad_groups. */
+int tmo_compress_2_4(const void* W, int dtype, int64_t rows, int64_t cols, int64_t ld, const uint32_t* mask,
+                     void* values, uint32_t* meta, void* values_t, uint32_t* meta_t, int64_t* bad_groups) {
+    if (rows < 0 || cols < 0 || rows % 4 || cols % 4 || ld < cols || (dtype != TMO_F32 && dtype != TMO_BF16)) return TMO_ERR_ARG;
+    int64_t wpr = (cols + 31) / 32, wpr_t = (rows + 31) / 32, bad = 0;
+    size_t es = dtype == TMO_F32 ? 4 : 2;
+    memset(meta, 0, (size_t)(rows * wpr) * 4); memset(meta_t, 0, (size_t)(cols * wpr_t) * 4);
+    memset(values, 0, (size_t)(rows * (cols / 2)) * es); memset(values_t, 0, (size_t)(cols * (rows / 2)) * es);
+#define TMO_BIT(r, c) ((mask[(r) * wpr + (c) / 32] >> ((c) % 32)) & 1u)
+    for (int64_t r = 0; r < rows; ++r) for (int64_t g = 0; g < cols / 4; ++g) {
+        int idx[4], n = 0;
+        for (int j = 0; j < 4; ++j) if (TMO_BIT(r, g * 4 + j)) idx[n++] = j;
+        if (n != 2) { bad++; continue; }
+        for (int k = 0; k < 2; ++k) memcpy((char*)values + (size_t)(r * (cols / 2) + g * 2 + k) * es, (const char*)W + (size_t)(r * ld + g * 4 + idx[k]) * es, es);
+        meta[r * wpr + g / 8] |= (uint32_t)(idx[0] | (idx[1] << 2)) << (4 * (g % 8));
+    }
+    for (int64_t c = 0; c < cols; ++c) for (int64_t g = 0; g < rows / 4; ++g) {
+        int idx[4], n = 0;
+        for (int i = 0; i < 4; ++i) if (TMO_BIT(g * 4 + i, c)) idx[n++] = i;
+        if (n != 2) { bad++; continue; }
+        for (int k = 0; k < 2; ++k) memcpy((char*)values_t + (size_t)(c * (rows / 2) + g * 2 + k) * es, (const char*)W + (size_t)((g * 4 + idx[k]) * ld + c) * es, es);
+        meta_t[c * wpr_t + g / 8] |= (uint32_t)(idx[0] | (idx[1] << 2)) << (4 * (g % 8));
+    }
+#undef TMO_BIT
+    if (bad_groups) *bad_groups = bad;
+    return TMO_OK;
+}
+
 int tmo_max_threads(void) {
 #ifdef _OPENMP
     return omp_get_max_threads();

@@ -44,6 +44,9 @@ def _load():
         lib.tmo_block_exact_enum.argtypes = [vp, i32, i32, vp, vp]
         lib.tmo_block_exact_bruteforce.argtypes = [vp, i32, i32, vp, vp]
         lib.tmo_block_exact_mcf.argtypes = [vp, i32, i32, vp, vp, vp, vp]
+        lib.tmo_nm_mask_1d.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, vp, vp, vp, vp]
+        lib.tmo_mask_violations.argtypes = [vp, i32, i64, i64, i64, vp, vp]
+        lib.tmo_compress_2_4.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp]
         lib.tmo_max_threads.restype = i32
         _lib = lib
     return _lib
@@ -134,6 +137,42 @@ def find_mask(W, N, M, method, threads: int = 1, want_masked: bool = True):
     if rc != 0:
         raise ValueError("tmo_find_mask rejected its arguments")
     return dict(mask=mask, masked=masked, objective=obj.value, nonfinite=bad.value)
+
+
+def nm_mask_1d(W, N, M, absorb_mean: bool = False):
+    """1-D N:M magnitude pruning along rows (N kept per group of M).  -> dict(mask, masked, objective, violations)."""
+    W = np.ascontiguousarray(W)
+    dtype = F32 if W.dtype == np.float32 else BF16
+    rows, cols = W.shape
+    mask = np.zeros((rows, (cols + 31) // 32), np.uint32); masked = np.empty_like(W)
+    obj = ctypes.c_double(0.0); viol = ctypes.c_int64(0)
+    rc = _load().tmo_nm_mask_1d(_ptr(W), dtype, rows, cols, cols, N, M, int(absorb_mean), _ptr(mask), _ptr(masked),
+                                ctypes.byref(obj), ctypes.byref(viol))
+    if rc != 0:
+        raise ValueError("tmo_nm_mask_1d rejected its arguments")
+    return dict(mask=mask, masked=masked, objective=obj.value, violations=viol.value)
+
+
+def mask_violations(W, mask) -> int:
+    W = np.ascontiguousarray(W); mask = np.ascontiguousarray(mask, dtype=np.uint32)
+    viol = ctypes.c_int64(0)
+    rc = _load().tmo_mask_violations(_ptr(W), F32 if W.dtype == np.float32 else BF16, W.shape[0], W.shape[1], W.shape[1], _ptr(mask), ctypes.byref(viol))
+    assert rc == 0
+    return viol.value
+
+
+def compress_2_4(W, mask):
+    """-> dict(values[rows, cols/2], meta[rows, wpr], values_t[cols, rows/2], meta_t[cols, wpr_t], bad_groups)."""
+    W = np.ascontiguousarray(W); mask = np.ascontiguousarray(mask, dtype=np.uint32)
+    rows, cols = W.shape
+    values = np.zeros((rows, cols // 2), W.dtype); values_t = np.zeros((cols, rows // 2), W.dtype)
+    meta = np.zeros((rows, (cols + 31) // 32), np.uint32); meta_t = np.zeros((cols, (rows + 31) // 32), np.uint32)
+    bad = ctypes.c_int64(0)
+    rc = _load().tmo_compress_2_4(_ptr(W), F32 if W.dtype == np.float32 else BF16, rows, cols, cols, _ptr(mask), _ptr(values), _ptr(meta),
+                                  _ptr(values_t), _ptr(meta_t), ctypes.byref(bad))
+    if rc != 0:
+        raise ValueError("tmo_compress_2_4 rejected its arguments")
+    return dict(values=values, meta=meta, values_t=values_t, meta_t=meta_t, bad_groups=bad.value)
 
 
 def unpack_mask(mask: np.ndarray, cols: int) -> np.ndarray:
