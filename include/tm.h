@@ -86,6 +86,7 @@ extern "C" {
 /* device status bits */
 #define TM_DEV_NONFINITE 1  /* an Inf or NaN was met in W (it is ordered by its bit pattern) */
 #define TM_DEV_INTERNAL 2   /* an iteration cap was hit (cannot happen; outputs fall back to a valid mask) */
+#define TM_DEV_BADMASK 4    /* tm_compress_2_4: a group of four did not hold exactly two kept entries (zeros were emitted) */
 
 typedef struct tm_problem {
     const void* W;          /* device, dtype, rows x ld */
@@ -167,6 +168,41 @@ int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols,
 #define TM_STATIC_SCRATCH_BYTES (1064960)
 int tm_find_mask_batched_static(const tm_problem* probs_host, int count, int N, int M, int method,
                                 int* status_dev, void* cuda_stream);
+
+/*
+ * Neighbouring operations.  They share one small device workspace of tm_aux_workspace_bytes() bytes
+ * (256-byte aligned, caller-owned, one per stream), run asynchronously on cuda_stream and never allocate.
+ *
+ * tm_nm_mask_1d -- Section 5, "Structured sparsity without full training": the plain (non-transposable) N:M
+ * pattern along rows: in every group of M contiguous weights of a row the M-N of lowest magnitude are pruned
+ * (the paper counts the pruned ones; here, as everywhere in this header, N counts the KEPT ones).  Order by
+ * (|w|, position), the later of equals being the heavier.  M in {2, 4, 8}, 0 <= N <= M, cols % M == 0.
+ * prob_host: one descriptor (host pointer); mask_out, masked_w_out, objective_out as for tm_find_mask.
+ * violations_out (device, may be NULL): the paper's "pattern-violations", the number of non-zero weights the
+ * pattern removes.  flags & TM_NM1D_ABSORB_MEAN ("mean absorption"): every kept weight receives the mean of
+ * its group's pruned weights: mu = (their sum in position order, fp64) / (their number), kept' = kept + mu in
+ * fp64, rounded once to fp32 (and from there to bf16, nearest even, for bf16 tensors).  The paper leaves open
+ * whether the mean is taken over the pruned or spread over the kept entries; for N = M/2 both agree.
+ *
+ * tm_mask_violations -- the same count for an arbitrary packed mask (layout of mask_out): weights that are
+ * non-zero although their mask bit is 0.
+ *
+ * tm_compress_2_4 -- Section 1 and Fig. 2: the transposable mask lets the same 2:4 pattern serve Y = W X and
+ * dL/dX = W^T dL/dY; this call prepares both operands from one read of W.  values[rows][cols/2]: for every
+ * row and every group of four columns the two kept weights in column order; meta[rows][wpr(cols)]: their
+ * column indices inside the group as a nibble idx0 | idx1 << 2, group g of the row in bits 4*(g%8) of word g/8.
+ * values_t[cols][rows/2], meta_t[cols][wpr(rows)]: the same for W^T (groups of four rows of a column).
+ * rows % 4 == cols % 4 == 0; W rows aligned to one block row.  A group without exactly two kept entries gets zeros
+ * and raises TM_DEV_BADMASK in *status_dev.  This is this library's plain layout, not a vendor library's.
+ */
+#define TM_NM1D_ABSORB_MEAN 1
+size_t tm_aux_workspace_bytes(void);
+int tm_nm_mask_1d(const tm_problem* prob_host, int N, int M, int flags, unsigned long long* violations_out,
+                  void* workspace_dev, size_t workspace_bytes, int* status_dev, void* cuda_stream);
+int tm_mask_violations(const void* W, int dtype, int64_t rows, int64_t cols, int64_t ld, const uint32_t* mask,
+                       unsigned long long* violations_out, void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
+int tm_compress_2_4(const void* W, int dtype, int64_t rows, int64_t cols, int64_t ld, const uint32_t* mask,
+                    void* values, uint32_t* meta, void* values_t, uint32_t* meta_t, int* status_dev, void* cuda_stream);
 
 const char* tm_status_string(int code);
 int tm_version(void);

@@ -9,7 +9,8 @@ from typing import Optional, Sequence
 
 TM_EXACT, TM_APPROX, TM_APPROX_COVER = 0, 1, 2
 TM_F32, TM_BF16 = 0, 1
-TM_DEV_NONFINITE, TM_DEV_INTERNAL = 1, 2
+TM_DEV_NONFINITE, TM_DEV_INTERNAL, TM_DEV_BADMASK = 1, 2, 4
+TM_NM1D_ABSORB_MEAN = 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libtm.so")
@@ -53,6 +54,11 @@ def load_library():
     lib.tm_workspace_bytes.argtypes = [ctypes.POINTER(tm_problem), i32]; lib.tm_workspace_bytes.restype = sz
     lib.tm_find_mask_host.argtypes = [vp, i32, i64, i64, i32, i32, i32, vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
     lib.tm_find_mask_host.restype = i32
+    u64p = ctypes.c_void_p
+    lib.tm_aux_workspace_bytes.restype = sz
+    lib.tm_nm_mask_1d.argtypes = [ctypes.POINTER(tm_problem), i32, i32, i32, u64p, vp, sz, vp, vp]; lib.tm_nm_mask_1d.restype = i32
+    lib.tm_mask_violations.argtypes = [vp, i32, i64, i64, i64, vp, u64p, vp, sz, vp]; lib.tm_mask_violations.restype = i32
+    lib.tm_compress_2_4.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp]; lib.tm_compress_2_4.restype = i32
     lib.tm_status_string.argtypes = [i32]; lib.tm_status_string.restype = ctypes.c_char_p
     lib.tm_version.restype = i32
     _lib = lib
@@ -251,6 +257,82 @@ def tm_find_mask_batched_static(Ws: Sequence, N: int, M: int, method: int, masks
     with torch.cuda.device(dev):
         s = stream if stream is not None else torch.cuda.current_stream(dev)
         _check(lib.tm_find_mask_batched_static(arr, len(Ws), N, M, method, _ptr(status), ctypes.c_void_p(s.cuda_stream)))
+
+
+def tm_aux_workspace_bytes() -> int:
+    return int(load_library().tm_aux_workspace_bytes())
+
+
+def _aux_workspace(dev, workspace):
+    import torch
+    if workspace is None:
+        workspace = torch.empty((tm_aux_workspace_bytes(),), dtype=torch.uint8, device=dev)
+    return workspace
+
+
+def _stream_ptr(dev, stream):
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream(dev)
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def tm_nm_mask_1d(W, N: int, M: int, absorb_mean: bool = False, mask_out=None, masked_w_out=None, objective_out=None,
+                  violations_out=None, status=None, workspace=None, stream=None, want_masked: bool = True):
+    """1-D N:M magnitude pruning along rows (N kept per group of M).  Returns (mask, masked, objective[1],
+    violations int64[1], status int32[1]); asynchronous on `stream` or torch's current stream."""
+    import torch
+    lib = load_library()
+    if not (W.is_cuda and W.dim() == 2 and (W.shape[1] <= 1 or W.stride(1) == 1)):
+        raise TmError(2, "W must be a 2-D CUDA tensor with unit column stride")
+    dev = W.device
+    if mask_out is None:
+        mask_out = torch.empty((W.shape[0], tm_mask_words_per_row(W.shape[1])), dtype=torch.int32, device=dev)
+    if masked_w_out is None and want_masked:
+        masked_w_out = torch.empty_strided(W.shape, W.stride(), dtype=W.dtype, device=dev)
+    if objective_out is None:
+        objective_out = torch.empty((1,), dtype=torch.float64, device=dev)
+    if violations_out is None:
+        violations_out = torch.zeros((1,), dtype=torch.int64, device=dev)
+    if status is None:
+        status = torch.zeros((1,), dtype=torch.int32, device=dev)
+    workspace = _aux_workspace(dev, workspace)
+    arr = _problem_array([W], [mask_out], [masked_w_out] if masked_w_out is not None else None, objective_out)
+    with torch.cuda.device(dev):
+        _check(lib.tm_nm_mask_1d(arr, N, M, TM_NM1D_ABSORB_MEAN if absorb_mean else 0, _ptr(violations_out), _ptr(workspace), workspace.numel(),
+                                 _ptr(status), _stream_ptr(dev, stream)))
+    return mask_out, masked_w_out, objective_out, violations_out, status
+
+
+def tm_mask_violations(W, mask, violations_out=None, workspace=None, stream=None):
+    """Non-zero weights whose bit in the packed mask is 0.  Returns int64[1] (device)."""
+    import torch
+    lib = load_library()
+    dev = W.device
+    if violations_out is None:
+        violations_out = torch.zeros((1,), dtype=torch.int64, device=dev)
+    workspace = _aux_workspace(dev, workspace)
+    with torch.cuda.device(dev):
+        _check(lib.tm_mask_violations(_ptr(W), _dtype_code(W), W.shape[0], W.shape[1], W.stride(0) if W.shape[0] > 1 else W.shape[1], _ptr(mask),
+                                      _ptr(violations_out), _ptr(workspace), workspace.numel(), _stream_ptr(dev, stream)))
+    return violations_out
+
+
+def tm_compress_2_4(W, mask, values=None, meta=None, values_t=None, meta_t=None, status=None, stream=None):
+    """2:4 compressed operands of W and W^T from one transposable mask.  Returns (values [rows, cols/2],
+    meta int32 [rows, wpr(cols)], values_t [cols, rows/2], meta_t int32 [cols, wpr(rows)], status int32[1])."""
+    import torch
+    lib = load_library()
+    dev = W.device
+    rows, cols = W.shape
+    if values is None: values = torch.empty((rows, cols // 2), dtype=W.dtype, device=dev)
+    if values_t is None: values_t = torch.empty((cols, rows // 2), dtype=W.dtype, device=dev)
+    if meta is None: meta = torch.empty((rows, tm_mask_words_per_row(cols)), dtype=torch.int32, device=dev)
+    if meta_t is None: meta_t = torch.empty((cols, tm_mask_words_per_row(rows)), dtype=torch.int32, device=dev)
+    if status is None: status = torch.zeros((1,), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib.tm_compress_2_4(_ptr(W), _dtype_code(W), rows, cols, W.stride(0) if rows > 1 else cols, _ptr(mask), _ptr(values), _ptr(meta),
+                                   _ptr(values_t), _ptr(meta_t), _ptr(status), _stream_ptr(dev, stream)))
+    return values, meta, values_t, meta_t, status
 
 
 def tm_find_mask_host(W, N: int, M: int, method: int, mask_out=None, masked_w_out=None, want_masked: bool = True,

@@ -370,6 +370,90 @@ int tm_find_mask_batched_static(const tm_problem* probs_host, int count, int N, 
     return run(probs_host, count, N, M, method, scratch, TM_STATIC_SCRATCH_BYTES, status_dev, static_cast<cudaStream_t>(cuda_stream), *d);
 }
 
+size_t tm_aux_workspace_bytes(void) { return kHeaderBytes + 2 * sizeof(double) * (size_t)tmask::aux_partial_slots(); }
+
+namespace {
+int check_aux_matrix(const void* W, int dtype, int64_t rows, int64_t cols, int64_t ld, int M) {
+    if (dtype != TM_F32 && dtype != TM_BF16) return TM_ERR_DTYPE;
+    if (rows < 0 || cols < 0 || cols % M || ld < cols) return TM_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return TM_OK;
+    if (!W) return TM_ERR_NULL;
+    const size_t elem = dtype == TM_F32 ? 4 : 2;
+    const size_t vec = (size_t)M * elem < 16 ? (size_t)M * elem : 16;
+    if ((uintptr_t)W % vec || ((size_t)ld * elem) % vec) return TM_ERR_ALIGN;
+    return TM_OK;
+}
+int check_aux_workspace(void* ws, size_t bytes) {
+    return (!ws || (uintptr_t)ws % kAlign || bytes < tm_aux_workspace_bytes()) ? TM_ERR_WORKSPACE : TM_OK;
+}
+}  // namespace
+
+int tm_nm_mask_1d(const tm_problem* prob_host, int N, int M, int flags, unsigned long long* violations_out,
+                  void* workspace_dev, size_t workspace_bytes, int* status_dev, void* cuda_stream) {
+    if (!prob_host) return TM_ERR_NULL;
+    if ((M != 2 && M != 4 && M != 8) || N < 0 || N > M) return TM_ERR_NM;
+    const tm_problem& p = *prob_host;
+    int rc;
+    if ((rc = check_aux_matrix(p.W, p.dtype, p.rows, p.cols, p.ld, M)) != TM_OK) return rc;
+    if (p.rows > 0 && p.cols > 0) {
+        if (!p.mask_out) return TM_ERR_NULL;
+        const size_t elem = p.dtype == TM_F32 ? 4 : 2, vec = (size_t)M * elem < 16 ? (size_t)M * elem : 16;
+        if ((uintptr_t)p.mask_out % 4 || (p.masked_w_out && (uintptr_t)p.masked_w_out % vec) || (p.objective_out && (uintptr_t)p.objective_out % 8) ||
+            (violations_out && (uintptr_t)violations_out % 8)) return TM_ERR_ALIGN;
+    }
+    if ((rc = check_aux_workspace(workspace_dev, workspace_bytes)) != TM_OK) return rc;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != TM_OK) return rc;
+    tmask::AuxProblem a;
+    a.W = p.W; a.mask = p.mask_out; a.masked = p.masked_w_out; a.rows = p.rows; a.cols = p.cols; a.ld = p.ld; a.dtype = p.dtype;
+    a.wpr = (int)((p.cols + 31) / 32);
+    char* base = static_cast<char*>(workspace_dev) + kHeaderBytes;
+    double* op = reinterpret_cast<double*>(base);
+    unsigned long long* vp = reinterpret_cast<unsigned long long*>(base + sizeof(double) * (size_t)tmask::aux_partial_slots());
+    if (tmask::launch_nm1d(a, N, M, flags, false, op, vp, p.objective_out, violations_out, status_dev, d->sms,
+                           static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    return TM_OK;
+}
+
+int tm_mask_violations(const void* W, int dtype, int64_t rows, int64_t cols, int64_t ld, const uint32_t* mask,
+                       unsigned long long* violations_out, void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
+    int rc;
+    if ((rc = check_aux_matrix(W, dtype, rows, cols, ld, 1)) != TM_OK) return rc;
+    if (!violations_out || (rows > 0 && cols > 0 && !mask)) return TM_ERR_NULL;
+    if ((uintptr_t)mask % 4 || (uintptr_t)violations_out % 8) return TM_ERR_ALIGN;
+    if ((rc = check_aux_workspace(workspace_dev, workspace_bytes)) != TM_OK) return rc;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != TM_OK) return rc;
+    tmask::AuxProblem a;
+    a.W = W; a.mask = const_cast<uint32_t*>(mask); a.masked = nullptr; a.rows = rows; a.cols = cols; a.ld = ld; a.dtype = dtype;
+    a.wpr = (int)((cols + 31) / 32);
+    char* base = static_cast<char*>(workspace_dev) + kHeaderBytes;
+    double* op = reinterpret_cast<double*>(base);
+    unsigned long long* vp = reinterpret_cast<unsigned long long*>(base + sizeof(double) * (size_t)tmask::aux_partial_slots());
+    if (tmask::launch_nm1d(a, 0, 8, 0, true, op, vp, nullptr, violations_out, nullptr, d->sms,
+                           static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    return TM_OK;
+}
+
+int tm_compress_2_4(const void* W, int dtype, int64_t rows, int64_t cols, int64_t ld, const uint32_t* mask,
+                    void* values, uint32_t* meta, void* values_t, uint32_t* meta_t, int* status_dev, void* cuda_stream) {
+    int rc;
+    if (rows % 4) return TM_ERR_SHAPE;
+    if ((rc = check_aux_matrix(W, dtype, rows, cols, ld, 4)) != TM_OK) return rc;
+    if (rows == 0 || cols == 0) return TM_OK;
+    if (!mask || !values || !meta || !values_t || !meta_t) return TM_ERR_NULL;
+    if ((uintptr_t)mask % 4 || (uintptr_t)meta % 4 || (uintptr_t)meta_t % 4 || (uintptr_t)values % 8 || (uintptr_t)values_t % 4) return TM_ERR_ALIGN;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != TM_OK) return rc;
+    tmask::AuxProblem a;
+    a.W = W; a.mask = const_cast<uint32_t*>(mask); a.masked = nullptr; a.rows = rows; a.cols = cols; a.ld = ld; a.dtype = dtype;
+    a.wpr = (int)((cols + 31) / 32);
+    if (tmask::launch_compress24(a, values, meta, values_t, meta_t, status_dev, d->sms, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        cudaGetLastError(); return TM_ERR_CUDA;
+    }
+    return TM_OK;
+}
+
 const char* tm_status_string(int code) {
     switch (code) {
     case TM_OK: return "ok";

@@ -12,6 +12,7 @@ constexpr int kF32 = 0;
 constexpr int kBF16 = 1;
 constexpr int kDevNonFinite = 1;
 constexpr int kDevInternal = 2;
+constexpr int kDevBadMask = 4;
 
 // One matrix of a (possibly batched) call, as the kernels see it.
 struct DevProblem {
@@ -25,6 +26,16 @@ struct DevProblem {
     int wpr;             // mask words per row
     int bcols;           // blocks per block row
     int chunks;          // work items per block row
+};
+
+// One matrix of the neighbouring operations (1-D pruning, violation count, 2:4 compression).
+struct AuxProblem {
+    const void* W;
+    uint32_t* mask;      // output of the 1-D pruning, input of the other two
+    void* masked;        // may be null
+    long long rows, cols, ld;
+    int dtype;
+    int wpr;
 };
 
 // Magnitudes travel as the fp32 bit pattern of |w| (bf16 widened exactly): for finite values the

@@ -1,0 +1,296 @@
+// Neighbouring operations of the mask search (Section 5 of the paper and the operand preparation the
+// transposable mask exists for):
+//   nm1d_kernel        1-D N:M magnitude pruning along rows, with the pattern-violation count and the
+//                      optional mean absorption, fused with the packed mask / masked weights / objective;
+//   violations_kernel  pattern-violations of an arbitrary packed mask;
+//   compress24_kernel  2:4 compressed values + 2-bit indices for W and for W^T from one transposable mask,
+//                      one read of W (the transposed half goes through a shared-memory tile).
+// All three stream the matrix once with vector loads; they are bound by HBM bandwidth.
+#include <type_traits>
+
+#include "tm_launch.h"
+
+namespace tmask {
+
+namespace {
+
+constexpr int kAuxWarps = 8;
+constexpr int kUnit = 8;                      // elements per thread and step: one mask byte
+
+__device__ __forceinline__ float bf16_to_float(uint32_t h) { return __uint_as_float(h << 16); }
+// fp32 -> bf16, round to nearest even; NaN stays NaN
+__device__ __forceinline__ uint32_t float_to_bf16_bits(float f) {
+    const uint32_t u = __float_as_uint(f);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (u >> 16) | 0x40u;
+    return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
+}
+
+// raw element bits of one unit (8 elements from column c0 of row r); elements past `cols` read as 0
+template <int DT>
+__device__ __forceinline__ void load_unit(const AuxProblem& P, long long r, long long c0, uint32_t (&raw)[kUnit]) {
+    const int valid = (int)min((long long)kUnit, P.cols - c0);
+    if constexpr (DT == kF32) {
+        const uint32_t* p = reinterpret_cast<const uint32_t*>(P.W) + r * P.ld + c0;
+        if (valid == kUnit && ((uintptr_t)p & 15) == 0) {
+            const uint4 a = __ldg(reinterpret_cast<const uint4*>(p)), b = __ldg(reinterpret_cast<const uint4*>(p) + 1);
+            raw[0] = a.x; raw[1] = a.y; raw[2] = a.z; raw[3] = a.w; raw[4] = b.x; raw[5] = b.y; raw[6] = b.z; raw[7] = b.w;
+        } else {
+#pragma unroll
+            for (int j = 0; j < kUnit; ++j) raw[j] = j < valid ? __ldg(p + j) : 0u;
+        }
+    } else {
+        const uint16_t* p = reinterpret_cast<const uint16_t*>(P.W) + r * P.ld + c0;
+        if (valid == kUnit && ((uintptr_t)p & 15) == 0) {
+            const uint4 a = __ldg(reinterpret_cast<const uint4*>(p));
+            const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { raw[2 * j] = w[j] & 0xFFFFu; raw[2 * j + 1] = w[j] >> 16; }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kUnit; ++j) raw[j] = j < valid ? (uint32_t)__ldg(p + j) : 0u;
+        }
+    }
+}
+template <int DT>
+__device__ __forceinline__ void store_unit(const AuxProblem& P, long long r, long long c0, const uint32_t (&out)[kUnit]) {
+    const int valid = (int)min((long long)kUnit, P.cols - c0);
+    if constexpr (DT == kF32) {
+        uint32_t* p = reinterpret_cast<uint32_t*>(P.masked) + r * P.ld + c0;
+        if (valid == kUnit && ((uintptr_t)p & 15) == 0) {
+            reinterpret_cast<uint4*>(p)[0] = make_uint4(out[0], out[1], out[2], out[3]);
+            reinterpret_cast<uint4*>(p)[1] = make_uint4(out[4], out[5], out[6], out[7]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < kUnit; ++j) if (j < valid) p[j] = out[j];
+        }
+    } else {
+        uint16_t* p = reinterpret_cast<uint16_t*>(P.masked) + r * P.ld + c0;
+        if (valid == kUnit && ((uintptr_t)p & 15) == 0) {
+            *reinterpret_cast<uint4*>(p) = make_uint4(out[0] | (out[1] << 16), out[2] | (out[3] << 16), out[4] | (out[5] << 16), out[6] | (out[7] << 16));
+        } else {
+#pragma unroll
+            for (int j = 0; j < kUnit; ++j) if (j < valid) p[j] = (uint16_t)out[j];
+        }
+    }
+}
+
+template <int DT> __device__ __forceinline__ uint32_t magnitude(uint32_t raw) { return DT == kF32 ? (raw & 0x7FFFFFFFu) : (raw & 0x7FFFu); }
+template <int DT> __device__ __forceinline__ float value_of(uint32_t raw) { return DT == kF32 ? __uint_as_float(raw) : bf16_to_float(raw); }
+
+// MODE 0: 1-D N:M pruning (N kept per group of M).  MODE 1: violations of a given mask.
+template <int DT, int M, int MODE>
+__global__ void __launch_bounds__(kAuxWarps * 32)
+nm1d_kernel(const AuxProblem P, int N, int flags, double* __restrict__ obj_partials, unsigned long long* __restrict__ viol_partials,
+            int* __restrict__ status_out) {
+    const int lane = threadIdx.x & 31;
+    const long long gw = (long long)blockIdx.x * kAuxWarps + (threadIdx.x >> 5), nwarps = (long long)gridDim.x * kAuxWarps;
+    const long long units = (P.cols + kUnit - 1) / kUnit, chunks = (units + 31) / 32, total = P.rows * chunks;
+    const long long per = (total + nwarps - 1) / nwarps, begin = gw * per, end = min(total, begin + per);
+    double acc = 0.0; unsigned long long viol = 0; bool bad = false;
+    for (long long item = begin; item < end; ++item) {
+        const long long r = item / chunks, chunk = item - r * chunks, unit = chunk * 32 + lane, c0 = unit * kUnit;
+        const bool active = c0 < P.cols;
+        uint32_t raw[kUnit], mag[kUnit];
+        if (active) load_unit<DT>(P, r, c0, raw);
+        else {
+#pragma unroll
+            for (int j = 0; j < kUnit; ++j) raw[j] = 0;
+        }
+#pragma unroll
+        for (int j = 0; j < kUnit; ++j) { mag[j] = magnitude<DT>(raw[j]); bad |= mag[j] >= (DT == kF32 ? 0x7F800000u : 0x7F80u); }
+        uint32_t keep = 0;
+        if constexpr (MODE == 0) {
+#pragma unroll
+            for (int j = 0; j < kUnit; ++j) {          // kept iff fewer than N entries of the group are heavier
+                int heavier = 0;
+#pragma unroll
+                for (int k = (j / M) * M; k < (j / M) * M + M; ++k)
+                    if (k != j) heavier += (k > j) ? (mag[k] >= mag[j]) : (mag[k] > mag[j]);
+                keep |= (heavier < N ? 1u : 0u) << j;
+            }
+            const int valid = active ? (int)min((long long)kUnit, P.cols - c0) : 0;
+            keep &= (1u << valid) - 1u;
+            float s = 0.f;
+            uint32_t out[kUnit];
+#pragma unroll
+            for (int j = 0; j < kUnit; ++j) {
+                const bool k = (keep >> j) & 1u;
+                out[j] = k ? raw[j] : 0u;
+                s += k ? __uint_as_float(DT == kF32 ? mag[j] : (mag[j] << 16)) : 0.f;
+                viol += (!k && j < valid && mag[j] != 0) ? 1ull : 0ull;
+            }
+            acc += (double)s;
+            if (flags & 1) {                             // mean absorption, fp64, one rounding to fp32 (then to bf16)
+#pragma unroll
+                for (int g = 0; g < kUnit / M; ++g) {
+                    double psum = 0.0; int pcnt = 0;
+#pragma unroll
+                    for (int j = g * M; j < g * M + M; ++j) if (!((keep >> j) & 1u)) { psum += (double)value_of<DT>(raw[j]); ++pcnt; }
+                    const double mu = pcnt ? psum / (double)pcnt : 0.0;
+#pragma unroll
+                    for (int j = g * M; j < g * M + M; ++j)
+                        if ((keep >> j) & 1u) {
+                            const float v = (float)((double)value_of<DT>(raw[j]) + mu);
+                            out[j] = DT == kF32 ? __float_as_uint(v) : float_to_bf16_bits(v);
+                        }
+                }
+            }
+            if (P.masked && active) store_unit<DT>(P, r, c0, out);
+            // four lanes share a mask word
+            uint32_t bits = keep << (8 * (lane & 3));
+            bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, 1);
+            bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, 2);
+            const long long word = chunk * 8 + (lane >> 2);
+            if ((lane & 3) == 0 && word < P.wpr) P.mask[r * P.wpr + word] = bits;
+        } else {
+            const long long word = unit >> 2;
+            const uint32_t m = (active && word < P.wpr) ? (__ldg(P.mask + r * P.wpr + word) >> (8 * (unit & 3))) & 0xFFu : 0xFFu;
+#pragma unroll
+            for (int j = 0; j < kUnit; ++j) viol += (!((m >> j) & 1u) && mag[j] != 0) ? 1ull : 0ull;
+        }
+    }
+    for (int o = 16; o; o >>= 1) { acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o); viol += __shfl_xor_sync(0xFFFFFFFFu, viol, o); }
+    if (lane == 0) { obj_partials[gw] = acc; viol_partials[gw] = viol; }
+    if (__any_sync(0xFFFFFFFFu, bad) && lane == 0 && status_out) atomicOr(status_out, kDevNonFinite);
+}
+
+__global__ void __launch_bounds__(256)
+aux_reduce_kernel(const double* __restrict__ obj_partials, const unsigned long long* __restrict__ viol_partials, int n,
+                  double* objective_out, unsigned long long* violations_out) {
+    __shared__ double so[256]; __shared__ unsigned long long sv[256];
+    double a = 0.0; unsigned long long v = 0;
+    for (int i = threadIdx.x; i < n; i += 256) { a += obj_partials[i]; v += viol_partials[i]; }
+    so[threadIdx.x] = a; sv[threadIdx.x] = v;
+    __syncthreads();
+    for (int o = 128; o; o >>= 1) {
+        if ((int)threadIdx.x < o) { so[threadIdx.x] += so[threadIdx.x + o]; sv[threadIdx.x] += sv[threadIdx.x + o]; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) { if (objective_out) *objective_out = so[0]; if (violations_out) *violations_out = sv[0]; }
+}
+
+// ---- 2:4 compression ---------------------------------------------------------------------------
+// CTA tile: 32 rows x 128 columns = 8 x 32 blocks of 4x4; warp = block row, lane = block column.
+template <int DT>
+__global__ void __launch_bounds__(256)
+compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __restrict__ meta, void* __restrict__ values_t,
+                  uint32_t* __restrict__ meta_t, int* __restrict__ status_out) {
+    using elem_t = typename std::conditional<DT == kF32, uint32_t, uint16_t>::type;
+    __shared__ elem_t tile_t[128][16 + 2];              // [column of the tile][value index along rows]
+    __shared__ uint32_t tile_mt[128];                   // transposed metadata word of every column
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long tiles_c = (P.cols + 127) / 128, tiles_r = (P.rows + 31) / 32;
+    const long long wpr_t = (P.rows + 31) / 32, half_c = P.cols / 2, half_r = P.rows / 2;
+    bool bad = false;
+    for (long long t = blockIdx.x; t < tiles_r * tiles_c; t += gridDim.x) {
+        const long long tr = t / tiles_c, tc = t - tr * tiles_c;
+        const long long r0 = tr * 32 + warp * 4, c0 = tc * 128 + lane * 4;
+        const bool active = r0 < P.rows && c0 < P.cols;
+        if (threadIdx.x < 128) tile_mt[threadIdx.x] = 0;
+        __syncthreads();
+        uint32_t v[4][4] = {}, mbits = 0;                // mbits bit 4i+j = mask of (row i, column j)
+        if (active) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if constexpr (DT == kF32) {
+                    const uint4 a = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(P.W) + (r0 + i) * P.ld + c0));
+                    v[i][0] = a.x; v[i][1] = a.y; v[i][2] = a.z; v[i][3] = a.w;
+                } else {
+                    const uint2 a = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(P.W) + (r0 + i) * P.ld + c0));
+                    v[i][0] = a.x & 0xFFFFu; v[i][1] = a.x >> 16; v[i][2] = a.y & 0xFFFFu; v[i][3] = a.y >> 16;
+                }
+                mbits |= ((__ldg(P.mask + (r0 + i) * P.wpr + (c0 >> 5)) >> (c0 & 31)) & 0xFu) << (4 * i);
+            }
+        }
+        // row form: two kept values per row, in column order, and their indices
+        uint32_t row_nibbles = 0;                        // nibble i = metadata of row i
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t m = (mbits >> (4 * i)) & 0xFu;
+            uint32_t a = 0, b = 0, nib = 0;
+            if (__popc(m) == 2) {
+                const int i0 = __ffs(m) - 1, i1 = 31 - __clz(m);
+                a = i0 == 0 ? v[i][0] : (i0 == 1 ? v[i][1] : v[i][2]);
+                b = i1 == 1 ? v[i][1] : (i1 == 2 ? v[i][2] : v[i][3]);
+                nib = (uint32_t)(i0 | (i1 << 2));
+            } else if (active) bad = true;
+            row_nibbles |= nib << (4 * i);
+            if (active) {
+                if constexpr (DT == kF32) *reinterpret_cast<uint2*>(reinterpret_cast<uint32_t*>(values) + (r0 + i) * half_c + (c0 >> 1)) = make_uint2(a, b);
+                else *reinterpret_cast<uint32_t*>(reinterpret_cast<uint16_t*>(values) + (r0 + i) * half_c + (c0 >> 1)) = a | (b << 16);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {                    // eight lanes share a metadata word of a row
+            uint32_t w = ((row_nibbles >> (4 * i)) & 0xFu) << (4 * (lane & 7));
+            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 1); w |= __shfl_xor_sync(0xFFFFFFFFu, w, 2); w |= __shfl_xor_sync(0xFFFFFFFFu, w, 4);
+            if ((lane & 7) == 0 && active) meta[(r0 + i) * P.wpr + (c0 >> 5)] = w;
+        }
+        // column form through the shared tile: column c of the tile gets its two kept values of this block row
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t m = ((mbits >> j) & 1u) | (((mbits >> (4 + j)) & 1u) << 1) | (((mbits >> (8 + j)) & 1u) << 2) | (((mbits >> (12 + j)) & 1u) << 3);
+            uint32_t a = 0, b = 0, nib = 0;
+            if (__popc(m) == 2) {
+                const int i0 = __ffs(m) - 1, i1 = 31 - __clz(m);
+                a = i0 == 0 ? v[0][j] : (i0 == 1 ? v[1][j] : v[2][j]);
+                b = i1 == 1 ? v[1][j] : (i1 == 2 ? v[2][j] : v[3][j]);
+                nib = (uint32_t)(i0 | (i1 << 2));
+            } else if (active) bad = true;
+            tile_t[lane * 4 + j][warp * 2] = (elem_t)a;
+            tile_t[lane * 4 + j][warp * 2 + 1] = (elem_t)b;
+            if (nib) atomicOr(&tile_mt[lane * 4 + j], nib << (4 * warp));
+        }
+        __syncthreads();
+        {   // 128 columns x 16 values: two threads per column, eight values each
+            const int c = threadIdx.x >> 1, h = threadIdx.x & 1;
+            const long long col = tc * 128 + c, vr0 = tr * 16 + h * 8;      // first value index along the transposed row
+            if (col < P.cols) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (vr0 + k < half_r) reinterpret_cast<elem_t*>(values_t)[col * half_r + vr0 + k] = tile_t[c][h * 8 + k];
+                if (h == 0) meta_t[col * wpr_t + tr] = tile_mt[c];
+            }
+        }
+        __syncthreads();
+    }
+    if (bad && status_out) atomicOr(status_out, kDevBadMask);
+}
+
+}  // namespace
+
+int aux_partial_slots() { return 8192; }
+
+static int aux_grid(long long items, int sms) {
+    const long long want = (items + kAuxWarps - 1) / kAuxWarps;
+    const long long cap = (long long)sms * 8 < 1024 ? (long long)sms * 8 : 1024;
+    return (int)(want < 1 ? 1 : (want > cap ? cap : want));
+}
+
+cudaError_t launch_nm1d(const AuxProblem& P, int N, int M, int flags, bool violations_only, double* obj_partials,
+                        unsigned long long* viol_partials, double* objective_out, unsigned long long* violations_out,
+                        int* status, int sms, cudaStream_t stream) {
+    const long long units = (P.cols + kUnit - 1) / kUnit, items = P.rows * ((units + 31) / 32);
+    const int grid = aux_grid(items, sms);
+#define TM_NM1D(DT, MM, MODE) nm1d_kernel<DT, MM, MODE><<<grid, kAuxWarps * 32, 0, stream>>>(P, N, flags, obj_partials, viol_partials, status)
+    if (violations_only) { if (P.dtype == kF32) TM_NM1D(kF32, 8, 1); else TM_NM1D(kBF16, 8, 1); }
+    else if (P.dtype == kF32) { if (M == 2) TM_NM1D(kF32, 2, 0); else if (M == 4) TM_NM1D(kF32, 4, 0); else TM_NM1D(kF32, 8, 0); }
+    else { if (M == 2) TM_NM1D(kBF16, 2, 0); else if (M == 4) TM_NM1D(kBF16, 4, 0); else TM_NM1D(kBF16, 8, 0); }
+#undef TM_NM1D
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    aux_reduce_kernel<<<1, 256, 0, stream>>>(obj_partials, viol_partials, grid * kAuxWarps, objective_out, violations_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_compress24(const AuxProblem& P, void* values, uint32_t* meta, void* values_t, uint32_t* meta_t, int* status,
+                              int sms, cudaStream_t stream) {
+    const long long tiles = ((P.rows + 31) / 32) * ((P.cols + 127) / 128);
+    if (tiles == 0) return cudaSuccess;
+    const int grid = (int)(tiles < (long long)sms * 8 ? tiles : (long long)sms * 8);
+    if (P.dtype == kF32) compress24_kernel<kF32><<<grid, 256, 0, stream>>>(P, values, meta, values_t, meta_t, status);
+    else compress24_kernel<kBF16><<<grid, 256, 0, stream>>>(P, values, meta, values_t, meta_t, status);
+    return cudaGetLastError();
+}
+
+}  // namespace tmask

@@ -44,4 +44,13 @@ int tma48_warps_per_cta(int dtype);
 cudaError_t launch_tma48(const TmaLaunch& a);
 cudaError_t launch_tma(const TmaLaunch& a);
 
+
+// Neighbouring operations (tm_kernels_aux.cu)
+int aux_partial_slots();
+cudaError_t launch_nm1d(const AuxProblem& P, int N, int M, int flags, bool violations_only, double* obj_partials,
+                        unsigned long long* viol_partials, double* objective_out, unsigned long long* violations_out,
+                        int* status, int sms, cudaStream_t stream);
+cudaError_t launch_compress24(const AuxProblem& P, void* values, uint32_t* meta, void* values_t, uint32_t* meta_t, int* status,
+                              int sms, cudaStream_t stream);
+
 }  // namespace tmask

@@ -1,0 +1,90 @@
+"""GPU parity of the neighbouring operations (1-D N:M pruning with violation count and mean absorption, mask
+violations, 2:4 operand compression) against the CPU oracle: everything bit-exact, objective within 1e-6."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2102_08124_b200 as tm
+import workloads
+from oracle import tm_oracle as orc
+from tests.gpu_util import to_device, to_host_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(dtype, rows, cols, seed, ties=False):
+    if ties:
+        W = np.random.Generator(np.random.PCG64(seed)).integers(-2, 3, size=(rows, cols)).astype(np.float32)
+    else:
+        W = workloads.normal_f32(rows, cols, 0.02, seed)
+        W[np.random.Generator(np.random.PCG64(seed + 1)).random(W.shape) < 0.3] = 0.0      # an "unstructured sparse" tensor
+    return workloads.f32_to_bf16_bits(W) if dtype == "bf16" else W
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N,M", [(2, 4), (4, 8), (1, 4), (1, 2), (3, 4), (2, 8), (6, 8), (0, 4), (4, 4)])
+@pytest.mark.parametrize("absorb", [False, True])
+def test_nm_1d(dtype, N, M, absorb):
+    for rows, cols, seed, ties in [(7, 8 * 33 + M, 3, False), (16, 1024, 4, True), (1, M, 5, False), (5, 2048 + 8, 6, False)]:
+        W = _case(dtype, rows, cols - cols % M, seed, ties)
+        want = orc.nm_mask_1d(W, N, M, absorb_mean=absorb)
+        mask, masked, obj, viol, status = tm.tm_nm_mask_1d(to_device(W), N, M, absorb_mean=absorb)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert np.array_equal(to_host_bits(mask), want["mask"])
+        assert np.array_equal(to_host_bits(masked), want["masked"].view(np.uint16 if dtype == "bf16" else np.uint32))
+        assert int(viol.item()) == want["violations"]
+        assert abs(float(obj.item()) - want["objective"]) <= 1e-6 * abs(want["objective"]) + 1e-300
+
+
+def test_nm_1d_strided_rows_and_unaligned_pitch():
+    base = to_device(_case("bf16", 12, 100, 7))                  # 200-byte pitch: rows are only 8-byte aligned
+    W = base[:, :92]                                             # a strided view
+    want = orc.nm_mask_1d(np.ascontiguousarray(to_host_bits(W.contiguous())), 2, 4)
+    mask, masked, obj, viol, status = tm.tm_nm_mask_1d(W, 2, 4)
+    torch.cuda.synchronize()
+    assert np.array_equal(to_host_bits(mask), want["mask"])
+    assert np.array_equal(to_host_bits(masked.contiguous()), want["masked"])
+    assert int(viol.item()) == want["violations"]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_mask_violations(dtype):
+    W = _case(dtype, 40, 520, 11)
+    Wd = to_device(W)
+    for N, M in [(2, 4), (4, 8)]:
+        res = orc.find_mask(W, N, M, orc.APPROX)
+        got = tm.tm_mask_violations(Wd, torch.from_numpy(res["mask"].view(np.int32)).cuda())
+        torch.cuda.synchronize()
+        assert int(got.item()) == orc.mask_violations(W, res["mask"])
+    zero = torch.zeros((40, 17), dtype=torch.int32, device="cuda")
+    assert int(tm.tm_mask_violations(Wd, zero).item()) == int((workloads.bf16_bits_to_f32(W) != 0).sum() if dtype == "bf16" else (W != 0).sum())
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_compress_2_4(dtype):
+    for rows, cols, seed in [(4, 4, 21), (36, 132, 22), (64, 512, 23), (100, 260, 24)]:
+        W = _case(dtype, rows, cols, seed) if dtype == "f32" or cols % 8 == 0 or True else None
+        Wd = to_device(W)
+        fn = tm.tm_find_mask_bf16 if dtype == "bf16" else tm.tm_find_mask
+        mask, _, _ = fn(Wd, 2, 4, tm.TM_APPROX)
+        values, meta, values_t, meta_t, status = tm.tm_compress_2_4(Wd, mask)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        want = orc.compress_2_4(W, to_host_bits(mask))
+        assert want["bad_groups"] == 0
+        assert np.array_equal(to_host_bits(values), want["values"].view(np.uint16 if dtype == "bf16" else np.uint32))
+        assert np.array_equal(to_host_bits(meta), want["meta"])
+        assert np.array_equal(to_host_bits(values_t), want["values_t"].view(np.uint16 if dtype == "bf16" else np.uint32))
+        assert np.array_equal(to_host_bits(meta_t), want["meta_t"])
+    # a mask that is not transposable is flagged, and the bad groups come out as zeros like the oracle's
+    W = _case("f32", 16, 64, 31); Wd = to_device(W)
+    one_d, _, _, _, _ = tm.tm_nm_mask_1d(Wd, 2, 4)
+    values, meta, values_t, meta_t, status = tm.tm_compress_2_4(Wd, one_d)
+    torch.cuda.synchronize()
+    assert int(status.item()) == tm.TM_DEV_BADMASK
+    want = orc.compress_2_4(W, to_host_bits(one_d))
+    assert np.array_equal(to_host_bits(values_t), want["values_t"].view(np.uint32)) and np.array_equal(to_host_bits(meta_t), want["meta_t"])
+    assert np.array_equal(to_host_bits(values), want["values"].view(np.uint32))
