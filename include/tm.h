@@ -25,7 +25,8 @@
  *                           paper's Lemma, W(P) <= 2 W*, speaks about).
  *
  * Conventions the paper leaves open
- *   - N counts KEPT entries per block row / column (Eq. 1).  Supported (N, M): (2, 4) and (4, 8).
+ *   - N counts KEPT entries per block row / column (Eq. 1).  Supported (N, M): (2, 4) and (4, 8) on every
+ *     path; (1, 4), (3, 4), (2, 8) and (6, 8) through the generic kernels.
  *   - Order of magnitudes: by the bit pattern of |w| (sign cleared, so -0 == +0), ties broken by the
  *     row-major position p = i*M + j inside the block; the earlier position is the lighter one.
  *     Algorithm 1's degree test is read as "fewer than M-N pruned edges at the node".
@@ -75,7 +76,7 @@ extern "C" {
 #define TM_OK 0
 #define TM_ERR_NULL 1       /* a required pointer is NULL */
 #define TM_ERR_SHAPE 2      /* negative size, rows or cols not a multiple of M, ld < cols, count < 0 */
-#define TM_ERR_NM 3         /* (N, M) is not (2, 4) or (4, 8) */
+#define TM_ERR_NM 3         /* unsupported (N, M) */
 #define TM_ERR_METHOD 4
 #define TM_ERR_DTYPE 5
 #define TM_ERR_ALIGN 6      /* W / masked_w_out base or row pitch not a multiple of min(16, M * element size) bytes, mask_out not of 4, objective_out not of 8 */

@@ -51,7 +51,10 @@ int current_device(DeviceState** st) {
     return TM_OK;
 }
 
-int check_nm(int N, int M) { return ((N == 2 && M == 4) || (N == 4 && M == 8)) ? TM_OK : TM_ERR_NM; }
+int check_nm(int N, int M) {
+    const bool ok = (M == 4 && (N == 1 || N == 2 || N == 3)) || (M == 8 && (N == 2 || N == 4 || N == 6));
+    return ok ? TM_OK : TM_ERR_NM;
+}
 int check_method(int m) { return (m == TM_EXACT || m == TM_APPROX || m == TM_APPROX_COVER) ? TM_OK : TM_ERR_METHOD; }
 
 int check_problem(const tm_problem& p, int M) {
@@ -102,7 +105,7 @@ int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, 
     std::vector<DevProblem> group[5];
     for (int k = 0; k < count; ++k) {
         DevProblem d = to_dev(probs[k], M, 0);
-        const int g = tmask::tma_eligible(d, M, method) ? 1 + 2 * d.dtype + (d.masked ? 1 : 0) : 0;
+        const int g = tmask::tma_eligible(d, N, M, method) ? 1 + 2 * d.dtype + (d.masked ? 1 : 0) : 0;
         group[g].push_back(d);
     }
     int used = 0;                                   // problems placed so far: offset into every workspace array
@@ -459,7 +462,7 @@ const char* tm_status_string(int code) {
     case TM_OK: return "ok";
     case TM_ERR_NULL: return "a required pointer is NULL";
     case TM_ERR_SHAPE: return "bad shape: sizes must be non-negative multiples of M and ld >= cols";
-    case TM_ERR_NM: return "unsupported (N, M): only (2, 4) and (4, 8)";
+    case TM_ERR_NM: return "unsupported (N, M)";
     case TM_ERR_METHOD: return "unknown method";
     case TM_ERR_DTYPE: return "unknown dtype";
     case TM_ERR_ALIGN: return "misaligned pointer or row pitch";

@@ -86,7 +86,7 @@ __device__ __forceinline__ const DevProblem& find_problem(const DevProblem* tabl
 
 template <int N, int M, int METHOD>
 // the exact 2:4 scorer is register-hungry: two CTAs per SM cap it at 128 registers (its rare wide-integer path spills)
-__global__ void __launch_bounds__(kWarpsPerCta * 32, (METHOD == kMethodExact && M == 4) ? 2 : 1)
+__global__ void __launch_bounds__(kWarpsPerCta * 32, (METHOD == kMethodExact && M == 4 && N == 2) ? 2 : 1)
 generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, int count, long long total_items,
                double* __restrict__ partials, int* __restrict__ status_out) {
     const int lane = threadIdx.x & 31;
@@ -128,7 +128,7 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
 
         uint64_t kept;
         if constexpr (METHOD == kMethodExact) {
-            if constexpr (M == 4) kept = exact_2_4(u, P.dtype == kBF16 ? 16 : 0);
+            if constexpr (M == 4 && N == 2) kept = exact_2_4(u, P.dtype == kBF16 ? 16 : 0);
             else kept = exact_ssp<N, M>(u, status);
         } else {
             kept = cover_mask<N, M>(u);
@@ -212,7 +212,8 @@ cudaError_t launch_generic(const LaunchArgs& a) {
     cudaError_t e = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * kWarpsPerCta, a.stream);
     if (e != cudaSuccess) return e;
     if (a.total_items > 0) {
-        e = (a.M == 4) ? launch_nm<2, 4>(a) : launch_nm<4, 8>(a);
+        if (a.M == 4) e = a.N == 2 ? launch_nm<2, 4>(a) : (a.N == 1 ? launch_nm<1, 4>(a) : launch_nm<3, 4>(a));
+        else e = a.N == 4 ? launch_nm<4, 8>(a) : (a.N == 2 ? launch_nm<2, 8>(a) : launch_nm<6, 8>(a));
         if (e != cudaSuccess) return e;
     }
     reduce_kernel<<<a.count, 256, 0, a.stream>>>(a.single, a.table, a.partials, (long long)a.ctas * kWarpsPerCta);

@@ -359,8 +359,8 @@ cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntr
 size_t tma_entry_bytes() { return sizeof(TmaEntry); }
 int tma_warps_per_cta(int dtype, int M) { return M == 8 ? tma48_warps_per_cta(dtype) : (dtype == kF32 ? Geometry<kF32>::kWarps : Geometry<kBF16>::kWarps); }
 
-bool tma_eligible(const DevProblem& p, int M, int method) {
-    if ((M != 4 && M != 8) || (method != kMethodApprox && method != kMethodCover)) return false;
+bool tma_eligible(const DevProblem& p, int N, int M, int method) {
+    if (!((N == 2 && M == 4) || (N == 4 && M == 8)) || (method != kMethodApprox && method != kMethodCover)) return false;
     const size_t elem = p.dtype == kF32 ? 4 : 2;
     if ((uintptr_t)p.W % 16 || ((size_t)p.ld * elem) % 16) return false;
     if (p.masked && (uintptr_t)p.masked % 16) return false;

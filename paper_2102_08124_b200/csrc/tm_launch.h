@@ -36,7 +36,7 @@ struct TmaLaunch {
 };
 size_t tma_entry_bytes();
 int tma_warps_per_cta(int dtype, int M);
-bool tma_eligible(const DevProblem& p, int M, int method);
+bool tma_eligible(const DevProblem& p, int N, int M, int method);
 bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M);
 cudaError_t tma_reduce(const void* entries_host, const void* entries_dev, int count, const double* partials, long long stride, cudaStream_t stream);
 // 4:8 variant (tm_kernels_tma48.cu), reached through launch_tma()

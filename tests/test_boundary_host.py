@@ -58,7 +58,7 @@ A = 0x10000  # a fake, well-aligned, never dereferenced device address
 
 
 @pytest.mark.parametrize("args,code", [
-    (dict(N=2, M=5), 3), (dict(N=3, M=4), 3), (dict(N=4, M=4), 3), (dict(N=2, M=8), 3), (dict(N=0, M=0), 3),
+    (dict(N=2, M=5), 3), (dict(N=0, M=4), 3), (dict(N=4, M=4), 3), (dict(N=3, M=8), 3), (dict(N=0, M=0), 3), (dict(N=1, M=2), 3),
     (dict(method=3), 4), (dict(method=-1), 4),
     (dict(rows=-4), 2), (dict(rows=6), 2), (dict(cols=6), 2), (dict(rows=4, cols=4, N=4, M=8), 2),
     (dict(W=0), 1), (dict(mask=0), 1),

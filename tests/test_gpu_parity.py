@@ -29,6 +29,17 @@ def test_small_ragged_shapes(N, M, method, dtype):
 
 
 @pytest.mark.parametrize("method", METHODS)
+@pytest.mark.parametrize("N,M", [(1, 4), (3, 4), (2, 8), (6, 8)])
+def test_other_n_m_pairs(N, M, method):
+    """Transposable masks with N != M/2 kept entries per line (generic kernels)."""
+    W = workloads.normal_f32(3 * M, 40 * M, 0.02, 70 + N + M)
+    assert_parity(W, N, M, method)
+    assert_parity(workloads.f32_to_bf16_bits(W), N, M, method)
+    rng = np.random.Generator(np.random.PCG64(71))
+    assert_parity(rng.integers(-2, 3, size=(2 * M, 36 * M)).astype(np.float32), N, M, method)
+
+
+@pytest.mark.parametrize("method", METHODS)
 def test_config1(method):
     assert_parity(workloads.config1()[0], 2, 4, method)
 
