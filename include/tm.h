@@ -134,6 +134,22 @@ int tm_find_mask_batched(const tm_problem* probs_host, int count, int N, int M, 
 size_t tm_workspace_bytes(const tm_problem* probs_host, int count);
 
 /*
+ * tm_plan_create / tm_plan_run / tm_plan_destroy -- tm_find_mask_batched() split for training loops that
+ * re-derive the masks of the same buffers every few iterations (Section 4.1, "Sparse Training from
+ * scratch": the mask is refreshed every 40 iterations).  tm_plan_create validates the descriptors, builds the
+ * tensor maps and copies the descriptor tables into the workspace once (synchronising stream 0; it allocates
+ * host memory for the plan, nothing on the device).  tm_plan_run then only clears the objective partials and
+ * launches the kernels on cuda_stream: it touches no host memory asynchronously, so it can be recorded by a
+ * stream capture and replayed.  The workspace belongs to the plan until tm_plan_destroy; the matrices must stay
+ * where they were (same pointers, shapes, pitches).  Results equal tm_find_mask_batched()'s bit for bit.
+ */
+typedef struct tm_plan tm_plan;
+int tm_plan_create(const tm_problem* probs_host, int count, int N, int M, int method, void* workspace_dev, size_t workspace_bytes,
+                   tm_plan** plan_out);
+int tm_plan_run(const tm_plan* plan, int* status_dev, void* cuda_stream);
+void tm_plan_destroy(tm_plan* plan);
+
+/*
  * tm_find_mask_host -- the search on HOST buffers (Eq. 1 / Algorithm 1 as above): copies W to the
  * current device in row strips, runs the kernels and copies mask, masked weights and objective back,
  * overlapping the three on separate streams; returns when the outputs are in host memory.
@@ -195,8 +211,14 @@ int tm_find_mask_batched_static(const tm_problem* probs_host, int count, int N, 
  * values_t[cols][rows/2], meta_t[cols][wpr(rows)]: the same for W^T (groups of four rows of a column).
  * rows % 4 == cols % 4 == 0; W rows aligned to one block row.  A group without exactly two kept entries gets zeros
  * and raises TM_DEV_BADMASK in *status_dev.  This is this library's plain layout, not a vendor library's.
+ *
+ * tm_mask_hamming -- number of differing bits of two packed masks of `words` 32-bit words: how much of the
+ * mask a refresh changed (Section 4.1 refreshes the mask every 40 iterations; Section 1 recalls that frequent
+ * mask changes are what the straight-through training of dense copies has to keep in check).
  */
 #define TM_NM1D_ABSORB_MEAN 1
+int tm_mask_hamming(const uint32_t* mask_a, const uint32_t* mask_b, int64_t words, unsigned long long* distance_out,
+                    void* workspace_dev, size_t workspace_bytes, void* cuda_stream);
 size_t tm_aux_workspace_bytes(void);
 int tm_nm_mask_1d(const tm_problem* prob_host, int N, int M, int flags, unsigned long long* violations_out,
                   void* workspace_dev, size_t workspace_bytes, int* status_dev, void* cuda_stream);

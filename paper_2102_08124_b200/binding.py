@@ -54,11 +54,15 @@ def load_library():
     lib.tm_workspace_bytes.argtypes = [ctypes.POINTER(tm_problem), i32]; lib.tm_workspace_bytes.restype = sz
     lib.tm_find_mask_host.argtypes = [vp, i32, i64, i64, i32, i32, i32, vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
     lib.tm_find_mask_host.restype = i32
+    lib.tm_plan_create.argtypes = [ctypes.POINTER(tm_problem), i32, i32, i32, i32, vp, sz, ctypes.POINTER(vp)]; lib.tm_plan_create.restype = i32
+    lib.tm_plan_run.argtypes = [vp, vp, vp]; lib.tm_plan_run.restype = i32
+    lib.tm_plan_destroy.argtypes = [vp]; lib.tm_plan_destroy.restype = None
     u64p = ctypes.c_void_p
     lib.tm_aux_workspace_bytes.restype = sz
     lib.tm_nm_mask_1d.argtypes = [ctypes.POINTER(tm_problem), i32, i32, i32, u64p, vp, sz, vp, vp]; lib.tm_nm_mask_1d.restype = i32
     lib.tm_mask_violations.argtypes = [vp, i32, i64, i64, i64, vp, u64p, vp, sz, vp]; lib.tm_mask_violations.restype = i32
     lib.tm_compress_2_4.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp]; lib.tm_compress_2_4.restype = i32
+    lib.tm_mask_hamming.argtypes = [vp, vp, i64, u64p, vp, sz, vp]; lib.tm_mask_hamming.restype = i32
     lib.tm_status_string.argtypes = [i32]; lib.tm_status_string.restype = ctypes.c_char_p
     lib.tm_version.restype = i32
     _lib = lib
@@ -200,6 +204,47 @@ class TmBatch:
         return self.masks, self.maskeds, self.objectives, self.status
 
 
+class TmPlan:
+    """Handle of a prepared batched search (see tm_plan_create in include/tm.h); owns its tensors."""
+
+    def __init__(self, handle, batch, N, M, method):
+        self._handle, self.batch, self.N, self.M, self.method = handle, batch, N, M, method
+
+    def __del__(self):
+        try:
+            tm_plan_destroy(self)
+        except Exception:
+            pass
+
+
+def tm_plan_create(Ws: Sequence, N: int, M: int, method: int, masks=None, maskeds=None, objectives=None, workspace=None,
+                   status=None, want_masked: bool = True) -> TmPlan:
+    """Validates and prepares a batched search once: descriptors, tensor maps and device tables.  tm_plan_run() then
+    only launches kernels (it can be captured into a CUDA graph)."""
+    import torch
+    batch = TmBatch(Ws, masks, maskeds, objectives, workspace, status, want_masked)
+    h = ctypes.c_void_p()
+    with torch.cuda.device(batch.device):
+        _check(batch._lib.tm_plan_create(batch._arr, batch.count, N, M, method, _ptr(batch.workspace), batch.workspace.numel(), ctypes.byref(h)))
+    return TmPlan(h, batch, N, M, method)
+
+
+def tm_plan_run(plan: TmPlan, status=None, stream=None):
+    """Launches the prepared search on `stream` (or torch's current stream).  Returns (masks, maskeds, objectives, status)."""
+    import torch
+    b = plan.batch
+    st = status if status is not None else b.status
+    with torch.cuda.device(b.device):
+        _check(b._lib.tm_plan_run(plan._handle, _ptr(st), _stream_ptr(b.device, stream)))
+    return b.masks, b.maskeds, b.objectives, st
+
+
+def tm_plan_destroy(plan: TmPlan):
+    if plan._handle is not None and plan._handle.value:
+        plan.batch._lib.tm_plan_destroy(plan._handle)
+        plan._handle = None
+
+
 def tm_workspace_bytes(count: int) -> int:
     return int(load_library().tm_workspace_bytes(None, count))
 
@@ -315,6 +360,22 @@ def tm_mask_violations(W, mask, violations_out=None, workspace=None, stream=None
         _check(lib.tm_mask_violations(_ptr(W), _dtype_code(W), W.shape[0], W.shape[1], W.stride(0) if W.shape[0] > 1 else W.shape[1], _ptr(mask),
                                       _ptr(violations_out), _ptr(workspace), workspace.numel(), _stream_ptr(dev, stream)))
     return violations_out
+
+
+def tm_mask_hamming(mask_a, mask_b, distance_out=None, workspace=None, stream=None):
+    """Number of differing bits of two packed masks (same shape).  Returns int64[1] (device)."""
+    import torch
+    lib = load_library()
+    dev = mask_a.device
+    if mask_a.shape != mask_b.shape or not (mask_a.is_contiguous() and mask_b.is_contiguous()):
+        raise TmError(2, "masks must be contiguous and of one shape")
+    if distance_out is None:
+        distance_out = torch.zeros((1,), dtype=torch.int64, device=dev)
+    workspace = _aux_workspace(dev, workspace)
+    with torch.cuda.device(dev):
+        _check(lib.tm_mask_hamming(_ptr(mask_a), _ptr(mask_b), mask_a.numel(), _ptr(distance_out), _ptr(workspace), workspace.numel(),
+                                   _stream_ptr(dev, stream)))
+    return distance_out
 
 
 def tm_compress_2_4(W, mask, values=None, meta=None, values_t=None, meta_t=None, status=None, stream=None):

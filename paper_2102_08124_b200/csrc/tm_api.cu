@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <new>
 #include <vector>
 
 #include "../../include/tm.h"
@@ -82,10 +83,24 @@ DevProblem to_dev(const tm_problem& p, int M, long long item_begin) {
 
 long long items_of(const DevProblem& d, int M) { return (d.rows / M) * (long long)d.chunks; }
 
-// Validates, partitions the problems between the bandwidth path and the generic path, builds the
-// descriptor tables in the workspace and launches.  ws layout: [header | table | tma records | partials].
-int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes, int* status_dev,
-        cudaStream_t stream, const DeviceState& dev) {
+// A validated call, partitioned between the bandwidth path and the generic path, with every launch
+// argument worked out.  ws layout: [header | table | tma records | partials].
+struct PlanGroup {
+    bool tma = false;
+    int n = 0, used = 0;                     // matrices of the group, offset of the group in every workspace array
+    std::vector<DevProblem> probs;           // generic path: the device table's host image
+    std::vector<char> entry_store;           // bandwidth path: descriptor records (128-byte aligned inside)
+    char* entries = nullptr;
+    tmask::LaunchArgs generic;
+    tmask::TmaLaunch bandwidth;
+};
+struct Plan {
+    int device = -1, N = 0, M = 0, method = 0, count = 0;
+    void* ws = nullptr;
+    std::vector<PlanGroup> groups;
+};
+
+int validate_call(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes) {
     int rc;
     if ((rc = check_nm(N, M)) != TM_OK) return rc;
     if ((rc = check_method(method)) != TM_OK) return rc;
@@ -95,6 +110,14 @@ int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, 
     for (int k = 0; k < count; ++k)
         if ((rc = check_problem(probs[k], M)) != TM_OK) return rc;
     if (!ws || (uintptr_t)ws % kAlign || ws_bytes < tm_workspace_bytes(probs, count)) return TM_ERR_WORKSPACE;
+    return TM_OK;
+}
+
+int build_plan(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes, const DeviceState& dev, Plan& plan) {
+    const int rc = validate_call(probs, count, N, M, method, ws, ws_bytes);
+    if (rc != TM_OK) return rc;
+    plan.N = N; plan.M = M; plan.method = method; plan.count = count; plan.ws = ws;
+    if (count == 0) return TM_OK;
 
     char* base = static_cast<char*>(ws);
     DevProblem* dtab = reinterpret_cast<DevProblem*>(base + kHeaderBytes);
@@ -108,52 +131,78 @@ int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, 
         const int g = tmask::tma_eligible(d, N, M, method) ? 1 + 2 * d.dtype + (d.masked ? 1 : 0) : 0;
         group[g].push_back(d);
     }
-    int used = 0;                                   // problems placed so far: offset into every workspace array
+    int used = 0;
     for (int g = 0; g < 5; ++g) {
         const int n = (int)group[g].size();
         if (n == 0) continue;
+        plan.groups.emplace_back();
+        PlanGroup& pg = plan.groups.back();
+        pg.tma = g != 0; pg.n = n; pg.used = used;
         double* partials = dpart + (size_t)used * kPartialSlots;
         if (g == 0) {
+            pg.probs = group[g];
             long long total = 0;
-            for (int k = 0; k < n; ++k) { group[g][k].item_begin = total; total += items_of(group[g][k], M); }
-            tmask::LaunchArgs a;
-            a.count = n; a.total_items = total; a.N = N; a.M = M; a.method = method; a.stream = stream; a.status = status_dev;
+            for (int k = 0; k < n; ++k) { pg.probs[k].item_begin = total; total += items_of(pg.probs[k], M); }
+            tmask::LaunchArgs& a = pg.generic;
+            a.count = n; a.total_items = total; a.N = N; a.M = M; a.method = method; a.stream = nullptr; a.status = nullptr;
             a.partials = partials;
             const int wpc = tmask::generic_warps_per_cta();
             const long long want = (total + wpc - 1) / wpc;
             const int cap = dev.sms * 4 < kPartialSlots / wpc ? dev.sms * 4 : kPartialSlots / wpc;
             a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));
-            a.single = group[g][0];
-            a.table = nullptr;
-            if (n > 1) {
-                // pageable source: the runtime stages the bytes before returning, so the vector may die here
-                if (cudaMemcpyAsync(dtab + used, group[g].data(), sizeof(DevProblem) * (size_t)n, cudaMemcpyHostToDevice, stream) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
-                a.table = dtab + used;
-            }
-            if (tmask::launch_generic(a) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+            a.single = pg.probs[0];
+            a.table = n > 1 ? dtab + used : nullptr;
         } else {
             const size_t esz = tmask::tma_entry_bytes();
-            std::vector<char> entries(esz * (size_t)n + 128);
-            char* eh = entries.data() + ((128 - (uintptr_t)entries.data() % 128) % 128);
+            pg.entry_store.resize(esz * (size_t)n + 128);
+            pg.entries = pg.entry_store.data() + ((128 - (uintptr_t)pg.entry_store.data() % 128) % 128);
             long long total = 0;
-            if (!tmask::tma_build_entries(group[g].data(), n, eh, &total, M)) return TM_ERR_CUDA;
-            tmask::TmaLaunch a;
-            a.entries_host = eh; a.entries_dev = nullptr; a.count = n; a.total_items = total; a.partials = partials;
-            a.status = status_dev; a.dtype = (g - 1) / 2; a.method = method; a.M = M; a.has_out = ((g - 1) & 1) != 0; a.stream = stream;
+            if (!tmask::tma_build_entries(group[g].data(), n, pg.entries, &total, M)) return TM_ERR_CUDA;
+            tmask::TmaLaunch& a = pg.bandwidth;
+            a.entries_host = pg.entries; a.count = n; a.total_items = total; a.partials = partials;
+            a.status = nullptr; a.dtype = (g - 1) / 2; a.method = method; a.M = M; a.has_out = ((g - 1) & 1) != 0; a.stream = nullptr;
             const int wpc = tmask::tma_warps_per_cta(a.dtype, M);
             const long long want = (total + wpc - 1) / wpc;
             const int cap = dev.sms < kPartialSlots / wpc ? dev.sms : kPartialSlots / wpc;
             a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));
-            if (n > 1) {
-                char* de = dent + (size_t)used * esz;
-                if (cudaMemcpyAsync(de, eh, esz * (size_t)n, cudaMemcpyHostToDevice, stream) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
-                a.entries_dev = de;
-            }
-            if (tmask::launch_tma(a) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+            a.entries_dev = n > 1 ? dent + (size_t)used * esz : nullptr;
         }
         used += n;
     }
     return TM_OK;
+}
+
+// Copies the descriptor tables of multi-matrix groups into the workspace (pageable sources: the runtime
+// stages the bytes before cudaMemcpyAsync returns, so the plan may die right after).
+int upload_plan(const Plan& plan, cudaStream_t stream) {
+    for (const PlanGroup& pg : plan.groups) {
+        if (pg.n <= 1) continue;
+        cudaError_t e = pg.tma
+            ? cudaMemcpyAsync(const_cast<void*>(pg.bandwidth.entries_dev), pg.entries, tmask::tma_entry_bytes() * (size_t)pg.n, cudaMemcpyHostToDevice, stream)
+            : cudaMemcpyAsync(const_cast<DevProblem*>(pg.generic.table), pg.probs.data(), sizeof(DevProblem) * (size_t)pg.n, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    }
+    return TM_OK;
+}
+
+// Kernel launches (and the clearing of their partials) only: nothing here touches host memory asynchronously.
+int launch_plan(const Plan& plan, int* status_dev, cudaStream_t stream) {
+    for (const PlanGroup& pg : plan.groups) {
+        cudaError_t e;
+        if (pg.tma) { tmask::TmaLaunch a = pg.bandwidth; a.status = status_dev; a.stream = stream; e = tmask::launch_tma(a); }
+        else { tmask::LaunchArgs a = pg.generic; a.status = status_dev; a.stream = stream; e = tmask::launch_generic(a); }
+        if (e != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    }
+    return TM_OK;
+}
+
+int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes, int* status_dev,
+        cudaStream_t stream, const DeviceState& dev) {
+    Plan plan;
+    int rc = build_plan(probs, count, N, M, method, ws, ws_bytes, dev, plan);
+    if (rc != TM_OK) return rc;
+    if ((rc = upload_plan(plan, stream)) != TM_OK) return rc;
+    return launch_plan(plan, status_dev, stream);
 }
 
 int ensure_scratch(DeviceState& d) {
@@ -373,6 +422,36 @@ int tm_find_mask_batched_static(const tm_problem* probs_host, int count, int N, 
     return run(probs_host, count, N, M, method, scratch, TM_STATIC_SCRATCH_BYTES, status_dev, static_cast<cudaStream_t>(cuda_stream), *d);
 }
 
+struct tm_plan { Plan plan; };
+
+int tm_plan_create(const tm_problem* probs_host, int count, int N, int M, int method, void* workspace_dev, size_t workspace_bytes,
+                   tm_plan** plan_out) {
+    if (!plan_out) return TM_ERR_NULL;
+    *plan_out = nullptr;
+    DeviceState* d = nullptr;
+    int rc;
+    // validate before touching the device
+    if ((rc = validate_call(probs_host, count, N, M, method, workspace_dev, workspace_bytes)) != TM_OK) return rc;
+    if ((rc = current_device(&d)) != TM_OK) return rc;
+    tm_plan* p = new (std::nothrow) tm_plan();
+    if (!p) return TM_ERR_CUDA;
+    if ((rc = build_plan(probs_host, count, N, M, method, workspace_dev, workspace_bytes, *d, p->plan)) != TM_OK) { delete p; return rc; }
+    cudaGetDevice(&p->plan.device);
+    // the tables are uploaded once, synchronously: tm_plan_run() then issues kernels only
+    if ((rc = upload_plan(p->plan, nullptr)) != TM_OK || cudaStreamSynchronize(nullptr) != cudaSuccess) { cudaGetLastError(); delete p; return rc != TM_OK ? rc : TM_ERR_CUDA; }
+    *plan_out = p;
+    return TM_OK;
+}
+
+int tm_plan_run(const tm_plan* plan, int* status_dev, void* cuda_stream) {
+    if (!plan) return TM_ERR_NULL;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != plan->plan.device) { cudaGetLastError(); return TM_ERR_CUDA; }
+    return launch_plan(plan->plan, status_dev, static_cast<cudaStream_t>(cuda_stream));
+}
+
+void tm_plan_destroy(tm_plan* plan) { delete plan; }
+
 size_t tm_aux_workspace_bytes(void) { return kHeaderBytes + 2 * sizeof(double) * (size_t)tmask::aux_partial_slots(); }
 
 namespace {
@@ -435,6 +514,22 @@ int tm_mask_violations(const void* W, int dtype, int64_t rows, int64_t cols, int
     unsigned long long* vp = reinterpret_cast<unsigned long long*>(base + sizeof(double) * (size_t)tmask::aux_partial_slots());
     if (tmask::launch_nm1d(a, 0, 8, 0, true, op, vp, nullptr, violations_out, nullptr, d->sms,
                            static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    return TM_OK;
+}
+
+int tm_mask_hamming(const uint32_t* mask_a, const uint32_t* mask_b, int64_t words, unsigned long long* distance_out,
+                    void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
+    if (words < 0) return TM_ERR_SHAPE;
+    if (!distance_out || (words > 0 && (!mask_a || !mask_b))) return TM_ERR_NULL;
+    if ((uintptr_t)mask_a % 4 || (uintptr_t)mask_b % 4 || (uintptr_t)distance_out % 8) return TM_ERR_ALIGN;
+    int rc;
+    if ((rc = check_aux_workspace(workspace_dev, workspace_bytes)) != TM_OK) return rc;
+    DeviceState* d = nullptr;
+    if ((rc = current_device(&d)) != TM_OK) return rc;
+    unsigned long long* vp = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace_dev) + kHeaderBytes);
+    if (tmask::launch_hamming(mask_a, mask_b, words, vp, distance_out, d->sms, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        cudaGetLastError(); return TM_ERR_CUDA;
+    }
     return TM_OK;
 }
 

@@ -169,6 +169,28 @@ aux_reduce_kernel(const double* __restrict__ obj_partials, const unsigned long l
     if (threadIdx.x == 0) { if (objective_out) *objective_out = so[0]; if (violations_out) *violations_out = sv[0]; }
 }
 
+// number of differing bits of two packed masks (how much a refresh changed the mask)
+__global__ void __launch_bounds__(kAuxWarps * 32)
+hamming_kernel(const uint32_t* __restrict__ a, const uint32_t* __restrict__ b, long long words, unsigned long long* __restrict__ partials) {
+    const int lane = threadIdx.x & 31;
+    const long long gw = (long long)blockIdx.x * kAuxWarps + (threadIdx.x >> 5), nwarps = (long long)gridDim.x * kAuxWarps;
+    const long long per = ((words + nwarps - 1) / nwarps + 31) / 32 * 32, begin = gw * per, end = min(words, begin + per);
+    unsigned long long n = 0;
+    for (long long i = begin + lane; i < end; i += 32) n += __popc(__ldg(a + i) ^ __ldg(b + i));
+    for (int o = 16; o; o >>= 1) n += __shfl_xor_sync(0xFFFFFFFFu, n, o);
+    if (lane == 0) partials[gw] = n;
+}
+__global__ void __launch_bounds__(256)
+hamming_reduce_kernel(const unsigned long long* __restrict__ partials, int n, unsigned long long* out) {
+    __shared__ unsigned long long sv[256];
+    unsigned long long v = 0;
+    for (int i = threadIdx.x; i < n; i += 256) v += partials[i];
+    sv[threadIdx.x] = v;
+    __syncthreads();
+    for (int o = 128; o; o >>= 1) { if ((int)threadIdx.x < o) sv[threadIdx.x] += sv[threadIdx.x + o]; __syncthreads(); }
+    if (threadIdx.x == 0) *out = sv[0];
+}
+
 // ---- 2:4 compression ---------------------------------------------------------------------------
 // CTA tile: 32 rows x 128 columns = 8 x 32 blocks of 4x4; warp = block row, lane = block column.
 template <int DT>
@@ -280,6 +302,16 @@ cudaError_t launch_nm1d(const AuxProblem& P, int N, int M, int flags, bool viola
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     aux_reduce_kernel<<<1, 256, 0, stream>>>(obj_partials, viol_partials, grid * kAuxWarps, objective_out, violations_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_hamming(const uint32_t* a, const uint32_t* b, long long words, unsigned long long* partials, unsigned long long* out,
+                           int sms, cudaStream_t stream) {
+    const int grid = aux_grid((words + 31) / 32, sms);
+    hamming_kernel<<<grid, kAuxWarps * 32, 0, stream>>>(a, b, words, partials);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    hamming_reduce_kernel<<<1, 256, 0, stream>>>(partials, grid * kAuxWarps, out);
     return cudaGetLastError();
 }
 

@@ -50,6 +50,8 @@ int aux_partial_slots();
 cudaError_t launch_nm1d(const AuxProblem& P, int N, int M, int flags, bool violations_only, double* obj_partials,
                         unsigned long long* viol_partials, double* objective_out, unsigned long long* violations_out,
                         int* status, int sms, cudaStream_t stream);
+cudaError_t launch_hamming(const uint32_t* a, const uint32_t* b, long long words, unsigned long long* partials, unsigned long long* out,
+                           int sms, cudaStream_t stream);
 cudaError_t launch_compress24(const AuxProblem& P, void* values, uint32_t* meta, void* values_t, uint32_t* meta_t, int* status,
                               int sms, cudaStream_t stream);
 

@@ -1,0 +1,82 @@
+"""The refresh loop of sparse training from scratch: prepared plans, CUDA-graph replay, changed-bit counts (GPU),
+and the straight-through masked layer (CPU)."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2102_08124_b200 as tm
+import workloads
+from oracle import tm_oracle as orc
+from paper_2102_08124_b200.refresh import MaskRefresher, masked_linear
+from tests.gpu_util import to_device, to_host_bits
+
+
+def test_masked_linear_straight_through_on_cpu():
+    torch.manual_seed(0)
+    W = torch.randn(8, 16, dtype=torch.float64, requires_grad=True)
+    S = torch.from_numpy(orc.unpack_mask(orc.find_mask(W.detach().float().numpy(), 2, 4, orc.APPROX)["mask"], 16).astype(np.float64))
+    x = torch.randn(5, 16, dtype=torch.float64, requires_grad=True)
+    y = masked_linear(x, W, (W * S).detach())
+    gy = torch.randn_like(y)
+    y.backward(gy)
+    assert torch.allclose(y, x @ (W * S).t())
+    assert torch.allclose(x.grad, gy @ (W * S).detach())          # backward product uses the same (transposable) mask
+    assert torch.allclose(W.grad, gy.t() @ x.detach())            # dense copy receives the unmasked gradient
+    bits = S.numpy().reshape(2, 4, 4, 4)
+    assert (bits.sum(axis=1) == 2).all() and (bits.sum(axis=3) == 2).all()   # so W*S and (W*S)^T are both 2:4
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("N,M,method", [(2, 4, tm.TM_APPROX), (4, 8, tm.TM_APPROX), (2, 4, tm.TM_EXACT)])
+def test_plan_equals_batched_call(N, M, method):
+    mats = [workloads.normal_f32(32, 264, 0.05, 81), workloads.normal_bf16(64, 520, 0.02, 82), workloads.normal_bf16(16, 136, 0.02, 83)]
+    Ws = [to_device(m) for m in mats]
+    ref_masks, ref_maskeds, ref_obj, _, _ = tm.tm_find_mask_batched(Ws, N, M, method)
+    plan = tm.tm_plan_create(Ws, N, M, method)
+    for _ in range(2):
+        masks, maskeds, objs, status = tm.tm_plan_run(plan)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for k in range(len(Ws)):
+            assert np.array_equal(to_host_bits(masks[k]), to_host_bits(ref_masks[k]))
+            assert np.array_equal(to_host_bits(maskeds[k]), to_host_bits(ref_maskeds[k]))
+        assert np.array_equal(objs.cpu().numpy(), ref_obj.cpu().numpy())
+    tm.tm_plan_destroy(plan)
+
+
+@pytest.mark.gpu
+def test_mask_hamming():
+    rng = np.random.Generator(np.random.PCG64(91))
+    for n in (1, 33, 4096, 100003):
+        a = rng.integers(0, 2 ** 32, size=n, dtype=np.uint64).astype(np.uint32); b = rng.integers(0, 2 ** 32, size=n, dtype=np.uint64).astype(np.uint32)
+        want = int(np.unpackbits((a ^ b).view(np.uint8)).sum())
+        got = tm.tm_mask_hamming(torch.from_numpy(a.view(np.int32)).cuda(), torch.from_numpy(b.view(np.int32)).cuda())
+        assert int(got.item()) == want
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("use_graph", [False, True])
+def test_refresh_loop(use_graph):
+    mats = workloads.config3(layers=1)                               # four BERT-large-shaped bf16 matrices
+    Ws = [to_device(m) for m in mats]
+    r = MaskRefresher(Ws, N=4, M=8, period=40, use_graph=use_graph)
+    for k, m in enumerate(mats):
+        assert np.array_equal(to_host_bits(r.masks[k]), orc.find_mask(m, 4, 8, orc.APPROX, threads=orc.max_threads(), want_masked=False)["mask"])
+    assert r.refresh() == 0                                           # unchanged weights: no bit flips
+    # a simulated optimizer update on the dense copies, then iterations 1..80: refreshes at 40 and 80
+    mats2 = workloads.config3_perturbed(mats, 1)
+    for W, m in zip(Ws, mats2):
+        W.copy_(to_device(m))
+    did = [it for it in range(1, 81) if r.step(it)]
+    assert did == [40, 80]
+    torch.cuda.synchronize()
+    want = [orc.find_mask(m, 4, 8, orc.APPROX, threads=orc.max_threads()) for m in mats2]
+    old = [orc.find_mask(m, 4, 8, orc.APPROX, threads=orc.max_threads(), want_masked=False)["mask"] for m in mats]
+    flips = 0
+    for k in range(len(mats)):
+        assert np.array_equal(to_host_bits(r.masks[k]), want[k]["mask"])
+        assert np.array_equal(to_host_bits(r.masked_weights[k]), want[k]["masked"])
+        flips += int(np.unpackbits((want[k]["mask"] ^ old[k]).view(np.uint8)).sum())
+    assert r.changed_bits[-2:] == [flips, 0] and flips > 0
