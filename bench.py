@@ -304,6 +304,69 @@ def run_survey(args):
         torch.cuda.empty_cache()
 
 
+def run_survey_neighbours(args):
+    """Secondary measurements of the neighbouring operations (1-D N:M pruning, compression, refresh loop)."""
+    import torch
+
+    import paper_2102_08124_b200 as tm
+    from paper_2102_08124_b200.refresh import MaskRefresher
+    peak, _ = measured_peak()
+
+    def timed(fn, min_steps=5):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter(); fn(); torch.cuda.synchronize(); once = time.perf_counter() - t0
+        steps = max(min_steps, min(200, int(0.3 / max(once, 1e-5))))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record(); torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    def emit(name, op, msec, nbytes, weights):
+        gbs = nbytes / (msec * 1e-3) / 1e9
+        print(json.dumps({"workload": name, "op": op, "ms_per_call": msec, "weights_per_s": weights / (msec * 1e-3),
+                          "algorithmic_GBps": gbs, "frac_of_measured_hbm": gbs / peak}), flush=True)
+
+    for name, gen, N, M in (("config5 12288x49152 bf16 quantised", workloads.config5, 2, 4), ("config4 8192x8192 fp32 Laplace", workloads.config4, 4, 8)):
+        m = gen()[0]
+        W = torch.from_numpy(m.view(np.int16)).cuda().view(torch.bfloat16) if m.dtype == np.uint16 else torch.from_numpy(m).cuda()
+        es, n = m.itemsize, m.size
+        mask = torch.empty((W.shape[0], tm.tm_mask_words_per_row(W.shape[1])), dtype=torch.int32, device="cuda")
+        masked = torch.empty_like(W); obj = torch.zeros(1, dtype=torch.float64, device="cuda"); viol = torch.zeros(1, dtype=torch.int64, device="cuda")
+        st = torch.zeros(1, dtype=torch.int32, device="cuda"); ws = torch.empty(tm.tm_aux_workspace_bytes(), dtype=torch.uint8, device="cuda")
+        for absorb in (False, True):
+            ms_ = timed(lambda: tm.tm_nm_mask_1d(W, N, M, absorb_mean=absorb, mask_out=mask, masked_w_out=masked, objective_out=obj,
+                                                  violations_out=viol, status=st, workspace=ws))
+            emit(name, "1-D %d:%d pruning%s" % (N, M, " + mean absorption" if absorb else ""), ms_, n * (2 * es + 0.125), n)
+        ms_ = timed(lambda: tm.tm_mask_violations(W, mask, violations_out=viol, workspace=ws))
+        emit(name, "mask violations", ms_, n * (es + 0.125), n)
+        if M == 4:
+            fn = tm.tm_find_mask_bf16 if m.dtype == np.uint16 else tm.tm_find_mask
+            fn(W, 2, 4, tm.TM_APPROX, mask_out=mask, masked_w_out=masked, objective_out=obj)
+            vals = torch.empty((W.shape[0], W.shape[1] // 2), dtype=W.dtype, device="cuda"); vals_t = torch.empty((W.shape[1], W.shape[0] // 2), dtype=W.dtype, device="cuda")
+            meta = torch.empty_like(mask); meta_t = torch.empty((W.shape[1], tm.tm_mask_words_per_row(W.shape[0])), dtype=torch.int32, device="cuda")
+            ms_ = timed(lambda: tm.tm_compress_2_4(W, mask, vals, meta, vals_t, meta_t, st))
+            emit(name, "2:4 compression of W and W^T", ms_, n * (es + 0.125 + es + 0.25), n)
+        mask2 = mask.clone()
+        ms_ = timed(lambda: tm.tm_mask_hamming(mask, mask2, distance_out=viol, workspace=ws))
+        emit(name, "mask Hamming distance", ms_, n * 0.25, n)
+        del W, mask, masked, mask2
+        torch.cuda.empty_cache()
+    mats = workloads.config3()
+    Ws = [torch.from_numpy(m.view(np.int16)).cuda().view(torch.bfloat16) for m in mats]
+    n = sum(m.size for m in mats)
+    for N, M in ((2, 4), (4, 8)):
+        for graph in (False, True):
+            r = MaskRefresher(Ws, N=N, M=M, use_graph=graph)
+            ms_ = timed(lambda: r.refresh())
+            emit("config3 BERT-large-shaped, 96 matrices bf16", "refresh %d:%d (%s): masks + masked weights + changed bits, result read back"
+                 % (N, M, "CUDA graph" if graph else "eager"), ms_, n * (4.125 + 0.5), n)
+            del r
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -319,7 +382,13 @@ def main():
     ap.add_argument("--config", type=int, default=0, help="with --survey: only this workload (1..5)")
     args = ap.parse_args()
     if args.survey:
-        run_survey(args)
+        if not args.config:
+            run_survey(args)
+            run_survey_neighbours(args)
+        elif args.config == 8:
+            run_survey_neighbours(args)
+        else:
+            run_survey(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -77,77 +77,93 @@ __device__ __forceinline__ void store_unit(const AuxProblem& P, long long r, lon
 template <int DT> __device__ __forceinline__ uint32_t magnitude(uint32_t raw) { return DT == kF32 ? (raw & 0x7FFFFFFFu) : (raw & 0x7FFFu); }
 template <int DT> __device__ __forceinline__ float value_of(uint32_t raw) { return DT == kF32 ? __uint_as_float(raw) : bf16_to_float(raw); }
 
+constexpr int kSub = 4;                       // units per thread and item: keeps 64-128 bytes per thread in flight
+
 // MODE 0: 1-D N:M pruning (N kept per group of M).  MODE 1: violations of a given mask.
+// Work item = 128 consecutive units (1024 elements) of one row: lane l handles units l, l+32, l+64, l+96.
 template <int DT, int M, int MODE>
 __global__ void __launch_bounds__(kAuxWarps * 32)
 nm1d_kernel(const AuxProblem P, int N, int flags, double* __restrict__ obj_partials, unsigned long long* __restrict__ viol_partials,
             int* __restrict__ status_out) {
     const int lane = threadIdx.x & 31;
     const long long gw = (long long)blockIdx.x * kAuxWarps + (threadIdx.x >> 5), nwarps = (long long)gridDim.x * kAuxWarps;
-    const long long units = (P.cols + kUnit - 1) / kUnit, chunks = (units + 31) / 32, total = P.rows * chunks;
+    const long long units = (P.cols + kUnit - 1) / kUnit, chunks = (units + 32 * kSub - 1) / (32 * kSub), total = P.rows * chunks;
     const long long per = (total + nwarps - 1) / nwarps, begin = gw * per, end = min(total, begin + per);
     double acc = 0.0; unsigned long long viol = 0; bool bad = false;
+    long long r = begin < end ? begin / chunks : 0, chunk = begin < end ? begin - r * chunks : 0;
     for (long long item = begin; item < end; ++item) {
-        const long long r = item / chunks, chunk = item - r * chunks, unit = chunk * 32 + lane, c0 = unit * kUnit;
-        const bool active = c0 < P.cols;
-        uint32_t raw[kUnit], mag[kUnit];
-        if (active) load_unit<DT>(P, r, c0, raw);
-        else {
+        uint32_t raw[kSub][kUnit];
+        uint32_t given[kSub];
 #pragma unroll
-            for (int j = 0; j < kUnit; ++j) raw[j] = 0;
+        for (int s = 0; s < kSub; ++s) {                 // all loads of the item first
+            const long long unit = (chunk * kSub + s) * 32 + lane, c0 = unit * kUnit;
+            if (c0 < P.cols) load_unit<DT>(P, r, c0, raw[s]);
+            else {
+#pragma unroll
+                for (int j = 0; j < kUnit; ++j) raw[s][j] = 0;
+            }
+            if constexpr (MODE == 1) {
+                const long long word = unit >> 2;
+                given[s] = (c0 < P.cols && word < P.wpr) ? (__ldg(P.mask + r * P.wpr + word) >> (8 * (unit & 3))) & 0xFFu : 0xFFu;
+            }
         }
 #pragma unroll
-        for (int j = 0; j < kUnit; ++j) { mag[j] = magnitude<DT>(raw[j]); bad |= mag[j] >= (DT == kF32 ? 0x7F800000u : 0x7F80u); }
-        uint32_t keep = 0;
-        if constexpr (MODE == 0) {
+        for (int s = 0; s < kSub; ++s) {
+            const long long unit = (chunk * kSub + s) * 32 + lane, c0 = unit * kUnit;
+            const bool active = c0 < P.cols;
+            uint32_t mag[kUnit];
 #pragma unroll
-            for (int j = 0; j < kUnit; ++j) {          // kept iff fewer than N entries of the group are heavier
-                int heavier = 0;
+            for (int j = 0; j < kUnit; ++j) { mag[j] = magnitude<DT>(raw[s][j]); bad |= mag[j] >= (DT == kF32 ? 0x7F800000u : 0x7F80u); }
+            if constexpr (MODE == 0) {
+                uint32_t keep = 0;
 #pragma unroll
-                for (int k = (j / M) * M; k < (j / M) * M + M; ++k)
-                    if (k != j) heavier += (k > j) ? (mag[k] >= mag[j]) : (mag[k] > mag[j]);
-                keep |= (heavier < N ? 1u : 0u) << j;
-            }
-            const int valid = active ? (int)min((long long)kUnit, P.cols - c0) : 0;
-            keep &= (1u << valid) - 1u;
-            float s = 0.f;
-            uint32_t out[kUnit];
+                for (int j = 0; j < kUnit; ++j) {      // kept iff fewer than N entries of the group are heavier
+                    int heavier = 0;
 #pragma unroll
-            for (int j = 0; j < kUnit; ++j) {
-                const bool k = (keep >> j) & 1u;
-                out[j] = k ? raw[j] : 0u;
-                s += k ? __uint_as_float(DT == kF32 ? mag[j] : (mag[j] << 16)) : 0.f;
-                viol += (!k && j < valid && mag[j] != 0) ? 1ull : 0ull;
-            }
-            acc += (double)s;
-            if (flags & 1) {                             // mean absorption, fp64, one rounding to fp32 (then to bf16)
-#pragma unroll
-                for (int g = 0; g < kUnit / M; ++g) {
-                    double psum = 0.0; int pcnt = 0;
-#pragma unroll
-                    for (int j = g * M; j < g * M + M; ++j) if (!((keep >> j) & 1u)) { psum += (double)value_of<DT>(raw[j]); ++pcnt; }
-                    const double mu = pcnt ? psum / (double)pcnt : 0.0;
-#pragma unroll
-                    for (int j = g * M; j < g * M + M; ++j)
-                        if ((keep >> j) & 1u) {
-                            const float v = (float)((double)value_of<DT>(raw[j]) + mu);
-                            out[j] = DT == kF32 ? __float_as_uint(v) : float_to_bf16_bits(v);
-                        }
+                    for (int k = (j / M) * M; k < (j / M) * M + M; ++k)
+                        if (k != j) heavier += (k > j) ? (mag[k] >= mag[j]) : (mag[k] > mag[j]);
+                    keep |= (heavier < N ? 1u : 0u) << j;
                 }
-            }
-            if (P.masked && active) store_unit<DT>(P, r, c0, out);
-            // four lanes share a mask word
-            uint32_t bits = keep << (8 * (lane & 3));
-            bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, 1);
-            bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, 2);
-            const long long word = chunk * 8 + (lane >> 2);
-            if ((lane & 3) == 0 && word < P.wpr) P.mask[r * P.wpr + word] = bits;
-        } else {
-            const long long word = unit >> 2;
-            const uint32_t m = (active && word < P.wpr) ? (__ldg(P.mask + r * P.wpr + word) >> (8 * (unit & 3))) & 0xFFu : 0xFFu;
+                const int valid = active ? (int)min((long long)kUnit, P.cols - c0) : 0;
+                keep &= (1u << valid) - 1u;
+                float sum = 0.f;
+                uint32_t out[kUnit];
 #pragma unroll
-            for (int j = 0; j < kUnit; ++j) viol += (!((m >> j) & 1u) && mag[j] != 0) ? 1ull : 0ull;
+                for (int j = 0; j < kUnit; ++j) {
+                    const bool k = (keep >> j) & 1u;
+                    out[j] = k ? raw[s][j] : 0u;
+                    sum += k ? __uint_as_float(DT == kF32 ? mag[j] : (mag[j] << 16)) : 0.f;
+                    viol += (!k && j < valid && mag[j] != 0) ? 1ull : 0ull;
+                }
+                acc += (double)sum;
+                if (flags & 1) {                         // mean absorption, fp64, one rounding to fp32 (then to bf16)
+#pragma unroll
+                    for (int g = 0; g < kUnit / M; ++g) {
+                        double psum = 0.0; int pcnt = 0;
+#pragma unroll
+                        for (int j = g * M; j < g * M + M; ++j) if (!((keep >> j) & 1u)) { psum += (double)value_of<DT>(raw[s][j]); ++pcnt; }
+                        const double mu = pcnt ? psum / (double)pcnt : 0.0;
+#pragma unroll
+                        for (int j = g * M; j < g * M + M; ++j)
+                            if ((keep >> j) & 1u) {
+                                const float v = (float)((double)value_of<DT>(raw[s][j]) + mu);
+                                out[j] = DT == kF32 ? __float_as_uint(v) : float_to_bf16_bits(v);
+                            }
+                    }
+                }
+                if (P.masked && active) store_unit<DT>(P, r, c0, out);
+                // four lanes share a mask word
+                uint32_t bits = keep << (8 * (lane & 3));
+                bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, 1);
+                bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, 2);
+                const long long word = (chunk * kSub + s) * 8 + (lane >> 2);
+                if ((lane & 3) == 0 && word < P.wpr) P.mask[r * P.wpr + word] = bits;
+            } else {
+#pragma unroll
+                for (int j = 0; j < kUnit; ++j) viol += (!((given[s] >> j) & 1u) && mag[j] != 0) ? 1ull : 0ull;
+            }
         }
+        if (++chunk == chunks) { chunk = 0; ++r; }
     }
     for (int o = 16; o; o >>= 1) { acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o); viol += __shfl_xor_sync(0xFFFFFFFFu, viol, o); }
     if (lane == 0) { obj_partials[gw] = acc; viol_partials[gw] = viol; }
@@ -292,7 +308,7 @@ static int aux_grid(long long items, int sms) {
 cudaError_t launch_nm1d(const AuxProblem& P, int N, int M, int flags, bool violations_only, double* obj_partials,
                         unsigned long long* viol_partials, double* objective_out, unsigned long long* violations_out,
                         int* status, int sms, cudaStream_t stream) {
-    const long long units = (P.cols + kUnit - 1) / kUnit, items = P.rows * ((units + 31) / 32);
+    const long long units = (P.cols + kUnit - 1) / kUnit, items = P.rows * ((units + 32 * kSub - 1) / (32 * kSub));
     const int grid = aux_grid(items, sms);
 #define TM_NM1D(DT, MM, MODE) nm1d_kernel<DT, MM, MODE><<<grid, kAuxWarps * 32, 0, stream>>>(P, N, flags, obj_partials, viol_partials, status)
     if (violations_only) { if (P.dtype == kF32) TM_NM1D(kF32, 8, 1); else TM_NM1D(kBF16, 8, 1); }
