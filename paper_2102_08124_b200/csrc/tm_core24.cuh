@@ -14,7 +14,8 @@
 // fewer than two entries of its column are heavier.
 // Step B (greedy fill heavy -> light) is evaluated in rounds: a free entry whose row and column are
 // both short is taken in this round when, among the current candidates, fewer than d_row heavier ones
-// share its row and fewer than d_col heavier ones share its column (d = what the line still lacks).
+// share its row and fewer than d_col heavier ones share its column (d = what the line still lacks),
+// in other words when kept entries and heavier candidates together number fewer than two in each.
 // Such an entry is reached by the sequential scan before its line fills up, so the rounds reproduce
 // the scan exactly; every round takes at least one entry per unfinished block, and a block never
 // lacks more than four entries.
@@ -69,21 +70,19 @@ TM_HD uint32_t cover_2_4(const Rel24& r) {
     return ~(maj3(r.hr1, r.hr2, r.hr3) | maj3(r.hc1, r.hc2, r.hc3));
 }
 
-// Lines that already hold two kept entries / at least one, replicated over the line's bits.
+// Lines that already hold two kept entries, replicated over the line's bits.
 struct LineFill {
-    uint32_t row_full, row_has, col_full, col_has;
+    uint32_t row_full, col_full;
 };
 TM_HD LineFill line_fill(uint32_t kept) {
     LineFill f;
     {
-        const uint32_t a = kept, b = kept >> 1, c = kept >> 2, d = kept >> 3, t = a | b | c;
-        f.row_has = ((t | d) & 0x11111111u) * 15u;
-        f.row_full = ((maj3(a, b, c) | (d & t)) & 0x11111111u) * 15u;
+        const uint32_t a = kept, b = kept >> 1, c = kept >> 2, d = kept >> 3;
+        f.row_full = ((maj3(a, b, c) | (d & (a | b | c))) & 0x11111111u) * 15u;
     }
     {
-        const uint32_t a = kept, b = kept >> 4, c = kept >> 8, d = kept >> 12, t = a | b | c;
-        f.col_has = ((t | d) & 0x000F000Fu) * 0x1111u;
-        f.col_full = ((maj3(a, b, c) | (d & t)) & 0x000F000Fu) * 0x1111u;
+        const uint32_t a = kept, b = kept >> 4, c = kept >> 8, d = kept >> 12;
+        f.col_full = ((maj3(a, b, c) | (d & (a | b | c))) & 0x000F000Fu) * 0x1111u;
     }
     return f;
 }
@@ -100,12 +99,14 @@ TM_HD void heavier_in_col(const Rel24& r, uint32_t set, uint32_t& any, uint32_t&
 }
 
 // One round of step B on the candidates `cand` (= open_candidates(kept, f)): returns the entries taken.
-TM_HD uint32_t fill_accept(const Rel24& r, const LineFill& f, uint32_t cand) {
-    uint32_t ra, r2, ca, c2;
-    heavier_in_row(r, cand, ra, r2);
-    heavier_in_col(r, cand, ca, c2);
-    // a line holding one entry lacks one (no heavier candidate allowed), an empty line lacks two
-    return cand & ~(r2 | (ra & f.row_has) | c2 | (ca & f.col_has));
+// A candidate is taken when its row holds fewer than two entries that are kept or heavier candidates,
+// and its column likewise.  Seen from the other entry q = p + k of the line, "q is a heavier candidate
+// than p" reads "q is a candidate and p (k places back, i.e. 4 - k places on) is not heavier than q",
+// so one rotation per distance moves a ready-made set.
+TM_HD uint32_t fill_accept(const Rel24& r, uint32_t kept, uint32_t cand) {
+    const uint32_t row_blocked = maj3(rot_row<1>(kept | (cand & ~r.hr3)), rot_row<2>(kept | (cand & ~r.hr2)), rot_row<3>(kept | (cand & ~r.hr1)));
+    const uint32_t col_blocked = maj3(rot_col<1>(kept | (cand & ~r.hc3)), rot_col<2>(kept | (cand & ~r.hc2)), rot_col<3>(kept | (cand & ~r.hc1)));
+    return cand & ~(row_blocked | col_blocked);
 }
 
 // Steps A and B for one pair of blocks, without cross-lane votes (host tests, simple kernels).
@@ -115,7 +116,7 @@ TM_HD uint32_t cover_and_fill_2_4(const Rel24& r, LineFill& f) {
     for (int round = 0; round < 4; ++round) {
         const uint32_t cand = open_candidates(kept, f);
         if (!cand) break;
-        kept |= fill_accept(r, f, cand);
+        kept |= fill_accept(r, kept, cand);
         f = line_fill(kept);
     }
     return kept;

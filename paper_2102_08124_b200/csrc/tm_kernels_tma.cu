@@ -223,7 +223,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                     int rounds = 0;
                     while (__any_sync(0xFFFFFFFFu, cand != 0)) {
                         if (++rounds > 4) { status |= kDevInternal; break; }    // a block lacks at most four entries
-                        k |= fill_accept(rel, f, cand);
+                        k |= fill_accept(rel, k, cand);
                         f = line_fill(k);
                         cand = open_candidates(k, f);
                     }

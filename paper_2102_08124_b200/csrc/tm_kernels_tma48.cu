@@ -40,9 +40,10 @@ __device__ __forceinline__ uint32_t max_u16x2_(uint32_t a, uint32_t b) {
     return r;
 }
 
-// p[b] carries the decisions destined for bit 7-b of every byte (see gather8); only bits 0..3 wanted
+// p[b] (bytes of equal bits) carries the decisions destined for bit 7-b of every byte (see gather8);
+// only bits 0..3 are wanted, the upper four come out as copies of p4
 __device__ __forceinline__ uint32_t gather4_low(uint32_t p7, uint32_t p6, uint32_t p5, uint32_t p4) {
-    return bitsel(bitsel(p7 >> 7, p6 >> 6, 0x01010101u), bitsel(p5 >> 5, p4 >> 4, 0x04040404u), 0x03030303u);
+    return bitsel(bitsel(p7, p6, 0x01010101u), bitsel(p5, p4, 0x04040404u), 0x03030303u);
 }
 
 // ---- bf16: packed comparisons ----------------------------------------------------------------
@@ -56,7 +57,7 @@ __device__ __forceinline__ void relations48_bf16(const unsigned char* blk, Rel48
         worst = max_u16x2_(worst, max_u16x2_(max_u16x2_(R[i][0], R[i][1]), max_u16x2_(R[i][2], R[i][3])));
     }
     // column relations hc[k]: bit (i,j) <- rows (i, i+k mod 8) of column j.  One subtraction decides two
-    // adjacent columns; byte permutes line the decisions up as (byte = row, top bit), a select tree packs them.
+    // adjacent columns; byte permutes line the decisions up as (byte = row, all bits equal), a select tree packs them.
 #pragma unroll
     for (int k = 1; k <= 4; ++k) {
         uint32_t word[2] = {0, 0};
@@ -72,7 +73,7 @@ __device__ __forceinline__ void relations48_bf16(const unsigned char* blk, Rel48
                     const int i = 4 * w + r;
                     d[r] = (i + k <= 7) ? later_heavier(R[(i + k) & 7][c], R[i][c]) : earlier_heavier(R[(i + k) & 7][c], R[i][c]);
                 }
-                const uint32_t q0 = prmt(d[0], d[1], 0x7351), q1 = prmt(d[2], d[3], 0x7351);
+                const uint32_t q0 = prmt(d[0], d[1], 0xFBD9), q1 = prmt(d[2], d[3], 0xFBD9);      // decisions as whole bytes
                 cw[2 * c] = prmt(q0, q1, 0x5410);
                 cw[2 * c + 1] = prmt(q0, q1, 0x7632);
             }
@@ -101,7 +102,7 @@ __device__ __forceinline__ void relations48_bf16(const unsigned char* blk, Rel48
                 if (k == 4 && j >= 4) { pj[j] = 0; continue; }
                 const uint32_t d0 = (j + k <= 7) ? later_heavier(Y[2 * w][(j + k) & 7], Y[2 * w][j]) : earlier_heavier(Y[2 * w][(j + k) & 7], Y[2 * w][j]);
                 const uint32_t d1 = (j + k <= 7) ? later_heavier(Y[2 * w + 1][(j + k) & 7], Y[2 * w + 1][j]) : earlier_heavier(Y[2 * w + 1][(j + k) & 7], Y[2 * w + 1][j]);
-                pj[j] = prmt(d0, d1, 0x7531);      // bytes = rows 4w .. 4w+3 of column j
+                pj[j] = prmt(d0, d1, 0xFDB9);      // bytes (0x00 / 0xFF) = rows 4w .. 4w+3 of column j
             }
             if (k == 4) {
                 word[w] = gather4_low(pj[0], pj[1], pj[2], pj[3]);
@@ -290,13 +291,13 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         if constexpr (DT == kBF16) relations48_bf16(blk, rel, worst); else relations48_f32(blk, rel, worst);
         u64 kept = cover_4_8(rel);
         if constexpr (METHOD == kMethodApprox) {
-            Lack48 L = line_lack(kept);
+            Short48 L = line_short(kept);
             u64 cand = open_candidates8(kept, L);
             int rounds = 0;
             while (__any_sync(0xFFFFFFFFu, cand != 0)) {
                 if (++rounds > 16) { status |= kDevInternal; break; }      // a block lacks at most sixteen entries
-                kept |= fill_accept8(rel, L, cand);
-                L = line_lack(kept);
+                kept |= fill_accept8(rel, kept, cand);
+                L = line_short(kept);
                 cand = open_candidates8(kept, L);
             }
             int swaps = 0;
@@ -306,7 +307,7 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                     u64 fa, fb;
                     const u64 c = swap_candidates8(rel, L, kept, fa, fb);
                     if (!swap_apply8_smem<DT>(blk, kept, c, fa, fb)) { status |= kDevInternal; L.row_short = 0; }
-                    else L = line_lack(kept);
+                    else L = line_short(kept);
                 }
             }
         }

@@ -6,7 +6,8 @@
 // sharing a row or a column -- is one 32-bit subtraction deciding the same pair in both blocks:
 //   X_q - X_p + 0x80008000  has bit 15 / bit 31 set iff  q >= p  in block A / block B
 // (15-bit magnitudes: no borrow crosses the lanes).  The 48 decisions are then collected into the
-// relation masks of tm_core24.cuh with byte permutes and a select tree.
+// relation masks of tm_core24.cuh: a byte permute in sign-replicating mode turns every decision into a
+// whole byte of equal bits, so a tree of bit selects with constant masks places them without shifts.
 #pragma once
 #include "tm_core24.cuh"
 
@@ -43,13 +44,13 @@ __device__ __forceinline__ uint32_t later_heavier(uint32_t xq, uint32_t xp) { re
 // ... and for q < p (strictly larger magnitude needed)
 __device__ __forceinline__ uint32_t earlier_heavier(uint32_t xq, uint32_t xp) { return xq - xp + 0x7FFF7FFFu; }
 
-// byte 0/1 <- decisions of dx/dy for block A, byte 2/3 <- for block B (decision = top bit of the byte)
-__device__ __forceinline__ uint32_t pick(uint32_t dx, uint32_t dy) { return prmt(dx, dy, 0x7351); }
+// byte 0/1 <- decisions of dx/dy for block A, byte 2/3 <- for block B; every byte is 0x00 or 0xFF
+__device__ __forceinline__ uint32_t pick(uint32_t dx, uint32_t dy) { return prmt(dx, dy, 0xFBD9); }
 
-// p[b] carries the decisions destined for bit 7-b of every byte
+// p[b] (bytes of equal bits) carries the decisions destined for bit 7-b of every byte
 __device__ __forceinline__ uint32_t gather8(const uint32_t (&p)[8]) {
-    const uint32_t t01 = bitsel(p[0], p[1] >> 1, 0x80808080u), t23 = bitsel(p[2] >> 2, p[3] >> 3, 0x20202020u);
-    const uint32_t t45 = bitsel(p[4] >> 4, p[5] >> 5, 0x08080808u), t67 = bitsel(p[6] >> 6, p[7] >> 7, 0x02020202u);
+    const uint32_t t01 = bitsel(p[0], p[1], 0x80808080u), t23 = bitsel(p[2], p[3], 0x20202020u);
+    const uint32_t t45 = bitsel(p[4], p[5], 0x08080808u), t67 = bitsel(p[6], p[7], 0x02020202u);
     return bitsel(bitsel(t01, t23, 0xC0C0C0C0u), bitsel(t45, t67, 0x0C0C0C0Cu), 0xF0F0F0F0u);
 }
 
@@ -80,14 +81,14 @@ __device__ __forceinline__ void relations_bf16(const PairKeys& k, Rel24& r) {
         const uint32_t q6 = pick(later_heavier(x[0][3], x[0][1]), later_heavier(x[2][3], x[2][1]));
         const uint32_t q3 = pick(later_heavier(x[1][2], x[1][0]), later_heavier(x[3][2], x[3][0]));
         const uint32_t q2 = pick(later_heavier(x[1][3], x[1][1]), later_heavier(x[3][3], x[3][1]));
-        r.hr2 = bitsel(bitsel(q7 >> 7, q6 >> 6, 0x01010101u), bitsel(q3 >> 3, q2 >> 2, 0x10101010u), 0x0F0F0F0Fu);
+        r.hr2 = bitsel(bitsel(q7, q6, 0x01010101u), bitsel(q3, q2, 0x10101010u), 0x0F0F0F0Fu);      // bits 2,3 of a nibble: don't care
     }
     // hc2 (rows 0,1 only): bit 4i+j, i in {0,1}; gathered as (row 0 -> byte 0, row 1 -> byte 1), then packed
     {
         uint32_t q[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) q[j] = pick(later_heavier(x[2][j], x[0][j]), later_heavier(x[3][j], x[1][j]));
-        const uint32_t g = bitsel(bitsel(q[0] >> 7, q[1] >> 6, 0x01010101u), bitsel(q[2] >> 5, q[3] >> 4, 0x04040404u), 0x03030303u);
+        const uint32_t g = bitsel(bitsel(q[0], q[1], 0x01010101u), bitsel(q[2], q[3], 0x04040404u), 0x03030303u);
         r.hc2 = bitsel(g, g >> 4, 0x0F0F0F0Fu);
     }
     r.hr3 = 0; r.hc3 = 0;
