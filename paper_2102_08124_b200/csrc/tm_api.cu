@@ -161,7 +161,7 @@ int build_plan(const tm_problem* probs, int count, int N, int M, int method, voi
             tmask::TmaLaunch& a = pg.bandwidth;
             a.entries_host = pg.entries; a.count = n; a.total_items = total; a.partials = partials;
             a.status = nullptr; a.dtype = (g - 1) / 2; a.method = method; a.M = M; a.has_out = ((g - 1) & 1) != 0; a.stream = nullptr;
-            const int wpc = tmask::tma_warps_per_cta(a.dtype, M);
+            const int wpc = tmask::tma_warps_per_cta(a.dtype, M, method);
             const long long want = (total + wpc - 1) / wpc;
             const int cap = dev.sms < kPartialSlots / wpc ? dev.sms : kPartialSlots / wpc;
             a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));

@@ -1,18 +1,22 @@
 // Bandwidth kernels of the approximate 2:4 search (TM_APPROX / TM_APPROX_COVER, M = 4).
 //
-// Every warp runs its own software pipeline over a contiguous range of work items (4 rows x 256
-// columns of one matrix).  Items are processed two at a time:
-//   1. lane 0 keeps bulk-tensor (TMA) loads of the next batch in flight into a private ring of
-//      shared-memory stages (two stage sets, used alternately);
-//   2. each lane reads its two 4x4 blocks of a landed item with 128-bit shared loads and runs steps
+// Every warp runs its own software pipeline over a contiguous range of work items (8 rows x 256
+// columns of one matrix: two block rows, 128 blocks):
+//   1. lane 0 keeps the bulk-tensor (TMA) load of the next item in flight into the other of the warp's
+//      two private shared-memory stages;
+//   2. each lane reads its two 4x4 blocks of either block row with 128-bit shared loads and runs steps
 //      A and B of the search bit-parallel in registers (tm_core24.cuh); the rounds of step B are
-//      warp-uniform (a vote decides whether any lane still has candidates);
+//      warp-uniform (a vote decides whether any lane still has candidates); the two block rows give
+//      the scheduler two independent instruction streams;
 //   3. the blocks that need step C (about one in six) are queued in shared memory and fixed by as
 //      many lanes at once as there are queued blocks, each reading the few magnitudes it must compare
 //      straight from the stage;
-//   4. the lanes write the masked weights back into the stage, lane 0 sends it out with a TMA store,
+//   4. the lanes write the masked weights back into the stage, lane 0 sends it out with one TMA store,
 //      mask bytes meet in shared memory and leave as whole 32-bit words.
-// No CTA-wide synchronisation exists; every wait is bounded.
+// A matrix with an odd number of block rows ends in a half-empty item: the copy zero-fills the missing
+// rows on the way in and clips them on the way out, and their mask words are not written.
+// Apart from one barrier after the lane-mask table is built, no CTA-wide synchronisation exists; every
+// wait is bounded.
 #include "tm_core24.cuh"
 #include "tm_launch.h"
 #include "tm_pair_bf16.cuh"
@@ -25,18 +29,25 @@ namespace tmask {
 
 namespace {
 
-constexpr int kItemRows = 4;
+constexpr int kItemRows = 8;               // two block rows per item
+constexpr int kHalves = 2;
 constexpr int kItemCols = 256;
-constexpr int kBatch = 2;                  // items per pipeline step
-constexpr int kStages = 2 * kBatch;
 
-template <int DT> struct Geometry {
+// Warps per CTA (one CTA per SM) and stages per warp.  The search is bound by integer issue and wants many
+// warps: for bf16, 24 warps at 80 registers per thread fill the shared memory with two stages each (a
+// deeper ring with fewer warps measured no faster, also for Algorithm 1 alone).
+template <int DT, int METHOD> struct Geometry {
     static constexpr int kElem = DT == kF32 ? 4 : 2;
-    static constexpr int kWarps = DT == kF32 ? 12 : 16;       // warps per CTA, one CTA per SM
+    static constexpr int kWarps = DT == kF32 ? 12 : 24;
+    static constexpr int kStages = 2;
     static constexpr int kRowPitch = kItemCols * kElem;        // bytes between rows inside a stage
+    static constexpr int kHalfBytes = 4 * kRowPitch;           // one block row
     static constexpr int kStageBytes = kItemRows * kRowPitch;
-    // stages | mask bytes [batch][4][32] | kept [batch][32] | swap candidates [batch][32] | queue | barriers
-    static constexpr int kWarpBytes = kStages * kStageBytes + kBatch * 128 + 2 * kBatch * 128 + 128 + 64 + 64;
+    // stages | mask bytes [8][32] | kept [2][32] | swap candidates [2][32] | queue [128] | barriers
+    static constexpr int kWarpBytes = kStages * kStageBytes + 256 + 2 * 256 + 128 + 64 + 64;
+    static constexpr int kSmemBytes = kWarps * kWarpBytes + (DT == kBF16 ? kLaneLutBytes : 0);
+    static_assert(kSmemBytes <= 232448, "at most 227 KB of shared memory per CTA");
+    static_assert(kWarpBytes % 128 == 0, "stages stay 128-byte aligned");
 };
 
 // ------------------------------------------------------------------------------------------
@@ -118,15 +129,17 @@ __device__ __forceinline__ bool swap_apply_smem(const unsigned char* blk, uint32
 
 // Masked weights back into the stage, mask bytes, objective contribution of the lane's two blocks.
 template <int DT, bool HAS_OUT>
-__device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* mrow /* [4][32] */, int lane, uint32_t kept) {
+__device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* mrow /* [4][32] */, const uint4* lut, int lane, uint32_t kept) {
     float s4 = 0.f;
+    const uint32_t mb4 = mask_bytes_2_4(kept);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
+        const uint32_t mb = i == 0 ? (mb4 & 0xFFu) : prmt(mb4, 0u, 0x4440 + i);
         if constexpr (DT == kBF16) {
             const uint4 r = *reinterpret_cast<const uint4*>(stage + i * 512 + lane * 16);
-            const uint32_t raw[4] = {r.x, r.y, r.z, r.w};
-            uint32_t o[4], m[4];
-            lane_masks(kept, i, m);
+            const uint4 mm = lut[mb];
+            const uint32_t raw[4] = {r.x, r.y, r.z, r.w}, m[4] = {mm.x, mm.y, mm.z, mm.w};
+            uint32_t o[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 o[q] = raw[q] & m[q];
@@ -144,8 +157,7 @@ __device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* m
             uint32_t o[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
-                const uint32_t bit = (kept >> (4 * i + (q & 3) + (q >> 2) * 16)) & 1u;
-                o[q] = bit ? raw[q] : 0u;
+                o[q] = ((mb >> q) & 1u) ? raw[q] : 0u;
                 s4 += fabsf(__uint_as_float(o[q]));
             }
             if constexpr (HAS_OUT) {
@@ -153,24 +165,29 @@ __device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* m
                 *reinterpret_cast<uint4*>(stage + i * 1024 + lane * 32 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
             }
         }
-        mrow[i * 32 + lane] = (unsigned char)(((kept >> (4 * i)) & 0xFu) | ((kept >> (12 + 4 * i)) & 0xF0u));
+        mrow[i * 32 + lane] = (unsigned char)mb;
     }
     return s4;
 }
 
 template <int DT, int METHOD, bool HAS_OUT>
-__global__ void __launch_bounds__(Geometry<DT>::kWarps * 32, 1)
+__global__ void __launch_bounds__(Geometry<DT, METHOD>::kWarps * 32, 1)
 tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict__ table, int count, long long total_items,
              double* __restrict__ partials, int* __restrict__ status_out) {
-    using G = Geometry<DT>;
+    using G = Geometry<DT, METHOD>;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned char* stages = smem_raw + (size_t)warp * G::kWarpBytes;
-    unsigned char* mbytes = stages + kStages * G::kStageBytes;
-    uint32_t* kbuf = reinterpret_cast<uint32_t*>(mbytes + kBatch * 128);
-    uint32_t* cbuf = kbuf + kBatch * 32;
-    unsigned char* queue = reinterpret_cast<unsigned char*>(cbuf + kBatch * 32);
+    unsigned char* mbytes = stages + G::kStages * G::kStageBytes;
+    uint32_t* kbuf = reinterpret_cast<uint32_t*>(mbytes + 256);
+    uint32_t* cbuf = kbuf + kHalves * 32;
+    unsigned char* queue = reinterpret_cast<unsigned char*>(cbuf + kHalves * 32);
     uint64_t* bars = reinterpret_cast<uint64_t*>(queue + 128);
+    uint4* lut = reinterpret_cast<uint4*>(smem_raw + (size_t)G::kWarps * G::kWarpBytes);
+    if constexpr (DT == kBF16) {           // the only CTA-wide step: the lane-mask table
+        fill_lane_lut(lut, threadIdx.x, G::kWarps * 32);
+        __syncthreads();
+    }
 
     const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
     const long long per = (total_items + nwarps - 1) / nwarps;
@@ -179,12 +196,12 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     const TmaEntry* tab = table ? table : &single;
 
     if (lane == 0) {
-        for (int s = 0; s < kStages; ++s) mbar_init(&bars[s], 1);
+        for (int s = 0; s < G::kStages; ++s) mbar_init(&bars[s], 1);
         fence_mbar_init();
     }
     __syncwarp();
 
-    Cursor ld, cur;                        // next item to request / first item of the batch in process
+    Cursor ld, cur;                        // next item to request / item in process
     ld.seek(tab, count, begin);
     cur = ld;
     int loaded = 0;
@@ -196,7 +213,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         ld.advance(tab, count);
         ++loaded;
     };
-    for (int g = 0; g < kBatch && loaded < n_items; ++g) issue_next(g);
+    for (int g = 0; g < G::kStages - 1 && loaded < n_items; ++g) issue_next(g);
 
     int status = 0, acc_k = -1;
     float facc = 0.f; double acc = 0.0;
@@ -204,46 +221,44 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     const uint32_t lt = (1u << lane) - 1u;
     bool alive = true;
 
-    for (int done = 0, batch = 0; done < n_items && alive; done += kBatch, ++batch) {
-        const int nb = min(kBatch, n_items - done), set = batch & 1;
-        const uint32_t parity = (uint32_t)((batch >> 1) & 1);
+    for (int it = 0; it < n_items && alive; ++it) {
+        const int s = it % G::kStages;
+        const uint32_t parity = (uint32_t)((it / G::kStages) & 1);
+        unsigned char* stage = stages + s * G::kStageBytes;
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bars[s], parity))) { status |= kDevInternal; alive = false; }
         int qn = 0;
-        // ---- steps A and B on every item of the batch -------------------------------------------
+        // ---- steps A and B on both block rows -----------------------------------------------------
 #pragma unroll
-        for (int g = 0; g < kBatch; ++g) {
-            if (g < nb) {
-                const int s = set * kBatch + g;
-                if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bars[s], parity))) { status |= kDevInternal; alive = false; }
-                Rel24 rel;
-                front_end<DT>(stages + s * G::kStageBytes, lane, rel, worst);
-                uint32_t k = cover_2_4(rel);
-                if constexpr (METHOD == kMethodApprox) {
-                    LineFill f = line_fill(k);
-                    uint32_t cand = open_candidates(k, f);
-                    int rounds = 0;
-                    while (__any_sync(0xFFFFFFFFu, cand != 0)) {
-                        if (++rounds > 4) { status |= kDevInternal; break; }    // a block lacks at most four entries
-                        k |= fill_accept(rel, k, cand);
-                        f = line_fill(k);
-                        cand = open_candidates(k, f);
-                    }
-                    const uint32_t sb = short_blocks(f);
-                    if (__any_sync(0xFFFFFFFFu, sb != 0)) {
-                        cbuf[g * 32 + lane] = swap_candidates(rel, f, k);
+        for (int h = 0; h < kHalves; ++h) {
+            Rel24 rel;
+            front_end<DT>(stage + h * G::kHalfBytes, lane, rel, worst);
+            uint32_t k = cover_2_4(rel);
+            if constexpr (METHOD == kMethodApprox) {
+                LineFill f = line_fill(k);
+                uint32_t cand = open_candidates(k, f);
+                int rounds = 0;
+                while (__any_sync(0xFFFFFFFFu, cand != 0)) {
+                    if (++rounds > 4) { status |= kDevInternal; break; }    // a block lacks at most four entries
+                    k |= fill_accept(rel, k, cand);
+                    f = line_fill(k);
+                    cand = open_candidates(k, f);
+                }
+                const uint32_t sb = short_blocks(f);
+                if (__any_sync(0xFFFFFFFFu, sb != 0)) {
+                    cbuf[h * 32 + lane] = swap_candidates(rel, f, k);
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const bool need = (sb >> h) & 1;
-                            const uint32_t m = __ballot_sync(0xFFFFFFFFu, need);
-                            if (need) queue[qn + __popc(m & lt)] = (unsigned char)((g << 6) | (h << 5) | lane);
-                            qn += __popc(m);
-                        }
+                    for (int b = 0; b < 2; ++b) {
+                        const bool need = (sb >> b) & 1;
+                        const uint32_t m = __ballot_sync(0xFFFFFFFFu, need);
+                        if (need) queue[qn + __popc(m & lt)] = (unsigned char)((h << 6) | (b << 5) | lane);
+                        qn += __popc(m);
                     }
                 }
-                kbuf[g * 32 + lane] = k;
             }
-            if (g == 0) {      // refill the other stage set: its stores were issued one batch ago
-                if constexpr (HAS_OUT) { if (lane == 0 && batch > 0) tma_wait_read<0>(); }
-                for (int gg = 0; gg < kBatch; ++gg) if (loaded < n_items) issue_next((set ^ 1) * kBatch + gg);
+            kbuf[h * 32 + lane] = k;
+            if (h == 0 && loaded < n_items) {       // refill the stage of the previous item: its store was issued one item ago
+                if constexpr (HAS_OUT) { if (lane == 0 && it > 0) tma_wait_read<0>(); }
+                issue_next((s + G::kStages - 1) % G::kStages);
             }
         }
         __syncwarp();
@@ -252,11 +267,11 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             for (int q0 = 0; q0 < qn; q0 += 32) {
                 if (q0 + lane < qn) {
                     const uint32_t e = queue[q0 + lane];
-                    const int g = e >> 6, h = (e >> 5) & 1, ln = e & 31;
-                    unsigned short* kh = reinterpret_cast<unsigned short*>(kbuf + g * 32 + ln) + h;
+                    const int h = e >> 6, b = (e >> 5) & 1, ln = e & 31;
+                    unsigned short* kh = reinterpret_cast<unsigned short*>(kbuf + h * 32 + ln) + b;
                     uint32_t k16 = *kh;
-                    const uint32_t c16 = reinterpret_cast<const unsigned short*>(cbuf + g * 32 + ln)[h];
-                    const unsigned char* blk = stages + (set * kBatch + g) * G::kStageBytes + ln * (8 * G::kElem) + h * (4 * G::kElem);
+                    const uint32_t c16 = reinterpret_cast<const unsigned short*>(cbuf + h * 32 + ln)[b];
+                    const unsigned char* blk = stage + h * G::kHalfBytes + ln * (8 * G::kElem) + b * (4 * G::kElem);
                     if (!swap_apply_smem<DT>(blk, k16, c16)) status |= kDevInternal;
                     *kh = (unsigned short)k16;
                 }
@@ -264,52 +279,42 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             __syncwarp();
         }
         // ---- outputs ---------------------------------------------------------------------------
-        Cursor out = cur;
-#pragma unroll
-        for (int g = 0; g < kBatch; ++g) {
-            if (g < nb) {
-                if (out.k != acc_k) {                                   // a new matrix starts: flush the objective partial
-                    if (acc_k >= 0) {
-                        acc += (double)facc;
-                        for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-                        if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
-                    }
-                    acc = 0.0; facc = 0.f; acc_k = out.k;
-                }
-                uint32_t k = kbuf[g * 32 + lane];
-                // blocks past the last column (zero-filled by the copy) contribute nothing
-                const int col0 = out.cj * kItemCols + lane * 8;
-                const int cols = (int)tab[out.k].p.cols;
-                if (col0 >= cols) k = 0;
-                else if (col0 + 4 >= cols) k &= 0xFFFFu;
-                facc += back_end<DT, HAS_OUT>(stages + (set * kBatch + g) * G::kStageBytes, mbytes + g * 128, lane, k);
-                out.advance(tab, count);
+        const TmaEntry& e = tab[cur.k];
+        if (cur.k != acc_k) {                                   // a new matrix starts: flush the objective partial
+            if (acc_k >= 0) {
+                acc += (double)facc;
+                for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+                if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
             }
+            acc = 0.0; facc = 0.f; acc_k = cur.k;
         }
+        // blocks past the last column (zero-filled by the copy) contribute nothing
+        const int col0 = cur.cj * kItemCols + lane * 8;
+        const int cols = (int)e.p.cols;
+        const uint32_t colmask = col0 >= cols ? 0u : (col0 + 4 >= cols ? 0xFFFFu : 0xFFFFFFFFu);
+#pragma unroll
+        for (int h = 0; h < kHalves; ++h)
+            facc += back_end<DT, HAS_OUT>(stage + h * G::kHalfBytes, mbytes + h * 128, lut, lane, kbuf[h * 32 + lane] & colmask);
         if constexpr (HAS_OUT) fence_proxy_async_smem();
         __syncwarp();
-        out = cur;
-#pragma unroll
-        for (int g = 0; g < kBatch; ++g) {
-            if (g < nb) {
-                const TmaEntry& e = tab[out.k];
-                if constexpr (HAS_OUT) {
-                    if (lane == 0) tma_store_2d(&e.out, out.cj * kItemCols, out.bi * kItemRows, stages + (set * kBatch + g) * G::kStageBytes);
-                }
-                const int row = lane >> 3, word = out.cj * 8 + (lane & 7);
-                const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + g * 128 + row * 32 + (lane & 7) * 4);
-                if (word < e.p.wpr) e.p.mask[((long long)out.bi * kItemRows + row) * e.p.wpr + word] = w;
-                out.advance(tab, count);
-            }
+        if constexpr (HAS_OUT) {
+            if (lane == 0) { tma_store_2d(&e.out, cur.cj * kItemCols, cur.bi * kItemRows, stage); tma_commit(); }
         }
-        if constexpr (HAS_OUT) { if (lane == 0) tma_commit(); }
-        cur = out;
-        if ((batch & 31) == 31) { acc += (double)facc; facc = 0.f; }       // keep the fp32 partial short
+        const long long rows = e.p.rows;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {                               // 8 rows x 8 words of mask
+            const int idx = lane + 32 * hh, word = cur.cj * 8 + (idx & 7);
+            const long long row = (long long)cur.bi * kItemRows + (idx >> 3);
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + (idx >> 3) * 32 + (idx & 7) * 4);
+            if (word < e.p.wpr && row < rows) e.p.mask[row * e.p.wpr + word] = w;
+        }
+        cur.advance(tab, count);
+        if ((it & 31) == 31) { acc += (double)facc; facc = 0.f; }           // keep the fp32 partial short
         __syncwarp();
     }
     if (!alive && lane == 0) {
         // a copy never landed: give the copies still in flight a bounded chance to finish before the stages die
-        for (int s = 0; s < kStages; ++s) { mbar_wait_bounded(&bars[s], 0, 1u << 14); mbar_wait_bounded(&bars[s], 1, 1u << 14); }
+        for (int s = 0; s < G::kStages; ++s) { mbar_wait_bounded(&bars[s], 0, 1u << 14); mbar_wait_bounded(&bars[s], 1, 1u << 14); }
     }
     if (lane == 0) tma_wait_all<0>();
     if (acc_k >= 0) {
@@ -341,8 +346,8 @@ reduce_tma_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __res
 
 template <int DT, int METHOD, bool HAS_OUT>
 cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntry* table) {
-    using G = Geometry<DT>;
-    const size_t smem = (size_t)G::kWarps * G::kWarpBytes;
+    using G = Geometry<DT, METHOD>;
+    const size_t smem = G::kSmemBytes;
     auto kern = tma24_kernel<DT, METHOD, HAS_OUT>;
     static bool configured = false;        // per instantiation
     if (!configured) {
@@ -357,7 +362,11 @@ cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntr
 }  // namespace
 
 size_t tma_entry_bytes() { return sizeof(TmaEntry); }
-int tma_warps_per_cta(int dtype, int M) { return M == 8 ? tma48_warps_per_cta(dtype) : (dtype == kF32 ? Geometry<kF32>::kWarps : Geometry<kBF16>::kWarps); }
+int tma_warps_per_cta(int dtype, int M, int method) {
+    if (M == 8) return tma48_warps_per_cta(dtype);
+    if (dtype == kF32) return method == kMethodApprox ? Geometry<kF32, kMethodApprox>::kWarps : Geometry<kF32, kMethodCover>::kWarps;
+    return method == kMethodApprox ? Geometry<kBF16, kMethodApprox>::kWarps : Geometry<kBF16, kMethodCover>::kWarps;
+}
 
 bool tma_eligible(const DevProblem& p, int N, int M, int method) {
     if (!((N == 2 && M == 4) || (N == 4 && M == 8)) || (method != kMethodApprox && method != kMethodCover)) return false;
@@ -369,9 +378,10 @@ bool tma_eligible(const DevProblem& p, int N, int M, int method) {
     return encode_fn() != nullptr;
 }
 
-// Fills `entries_host` (count TmaEntry records) for problems that all passed tma_eligible(); an item is M rows x 256 columns.
+// Fills `entries_host` (count TmaEntry records) for problems that all passed tma_eligible(); an item is 8 rows x 256 columns.
 bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M) {
-    return build_entries(probs, count, static_cast<TmaEntry*>(entries_host), total_items, M, kItemCols);
+    (void)M;
+    return build_entries(probs, count, static_cast<TmaEntry*>(entries_host), total_items, kItemRows, kItemCols);
 }
 
 cudaError_t tma_reduce(const void* entries_host, const void* entries_dev, int count, const double* partials, long long stride, cudaStream_t stream) {
@@ -383,7 +393,7 @@ cudaError_t tma_reduce(const void* entries_host, const void* entries_dev, int co
 // All problems of one launch share dtype and the presence of masked_w_out (the caller groups them).
 cudaError_t launch_tma(const TmaLaunch& a) {
     if (a.M == 8) return launch_tma48(a);
-    const int wpc = tma_warps_per_cta(a.dtype, 4);
+    const int wpc = tma_warps_per_cta(a.dtype, 4, a.method);
     cudaError_t err = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * wpc, a.stream);
     if (err != cudaSuccess) return err;
     const TmaEntry* host = static_cast<const TmaEntry*>(a.entries_host);

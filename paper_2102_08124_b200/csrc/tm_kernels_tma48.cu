@@ -190,22 +190,22 @@ __device__ __forceinline__ bool swap_apply8_smem(const unsigned char* blk, u64& 
 
 // Masked weights back into the stage, mask bytes, objective contribution of the lane's block.
 template <int DT, bool HAS_OUT>
-__device__ __forceinline__ float back_end48(unsigned char* blk, unsigned char* mrow /* [8][32] */, int lane, u64 kept) {
+__device__ __forceinline__ float back_end48(unsigned char* blk, unsigned char* mrow /* [8][32] */, const uint4* lut, int lane, u64 kept) {
     float s8 = 0.f;
     const uint32_t kw[2] = {(uint32_t)kept, (uint32_t)(kept >> 32)};
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const uint32_t word = kw[i >> 2];
         const int base = 8 * (i & 3);
+        const uint32_t mb = (i & 3) == 0 ? (word & 0xFFu) : prmt(word, 0u, 0x4440 + (i & 3));      // the row's mask byte
         if constexpr (DT == kBF16) {
             const uint4 r = *reinterpret_cast<const uint4*>(blk + i * 512);
-            const uint32_t raw[4] = {r.x, r.y, r.z, r.w};
+            const uint4 mm = lut[mb];                  // 16-bit lane masks of the row's eight keep flags
+            const uint32_t raw[4] = {r.x, r.y, r.z, r.w}, m4[4] = {mm.x, mm.y, mm.z, mm.w};
             uint32_t o[4];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                // keep bits of columns 2c, 2c+1 -> top bit of a byte each -> 16-bit lane masks
-                const uint32_t sa = word << (31 - (base + 2 * c)), sb = word << (30 - (base + 2 * c));
-                const uint32_t m = prmt(sa, sb, 0xFFBB);
+                const uint32_t m = m4[c];
                 o[c] = raw[c] & m;
                 const uint32_t ab = raw[c] & m & 0x7FFF7FFFu;
                 unsigned short lo, hi;
@@ -228,7 +228,7 @@ __device__ __forceinline__ float back_end48(unsigned char* blk, unsigned char* m
                 *reinterpret_cast<uint4*>(blk + i * 1024 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
             }
         }
-        mrow[i * 32 + lane] = (unsigned char)(word >> base);
+        mrow[i * 32 + lane] = (unsigned char)mb;
     }
     return s8;
 }
@@ -243,6 +243,11 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     unsigned char* stages = smem_raw + (size_t)warp * G::kWarpBytes;
     unsigned char* mbytes = stages + G::kStages * G::kStageBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(mbytes + 256);
+    uint4* lut = reinterpret_cast<uint4*>(smem_raw + (size_t)G::kWarps * G::kWarpBytes);
+    if constexpr (DT == kBF16) {           // the only CTA-wide step: the lane-mask table
+        fill_lane_lut(lut, threadIdx.x, G::kWarps * 32);
+        __syncthreads();
+    }
 
     const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
     const long long per = (total_items + nwarps - 1) / nwarps;
@@ -322,7 +327,7 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             }
             acc = 0.0; facc = 0.f; acc_k = cur.k;
         }
-        facc += back_end48<DT, HAS_OUT>(blk, mbytes, lane, kept);
+        facc += back_end48<DT, HAS_OUT>(blk, mbytes, lut, lane, kept);
         if constexpr (HAS_OUT) fence_proxy_async_smem();
         __syncwarp();
         if constexpr (HAS_OUT) {
@@ -359,7 +364,7 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
 template <int DT, int METHOD, bool HAS_OUT>
 cudaError_t launch_one48(const TmaLaunch& a, const TmaEntry& single, const TmaEntry* table) {
     using G = Geo48<DT>;
-    const size_t smem = (size_t)G::kWarps * G::kWarpBytes;
+    const size_t smem = (size_t)G::kWarps * G::kWarpBytes + (DT == kBF16 ? kLaneLutBytes : 0);
     auto kern = tma48_kernel<DT, METHOD, HAS_OUT>;
     static bool configured = false;        // per instantiation
     if (!configured) {

@@ -27,7 +27,7 @@ struct TmaLaunch {
     const void* entries_dev;    // the same records in device memory, or nullptr when count == 1
     int count;
     long long total_items;
-    double* partials;           // device scratch, count * ctas * tma_warps_per_cta(dtype) doubles
+    double* partials;           // device scratch, count * ctas * tma_warps_per_cta(dtype, M, method) doubles
     int* status;
     int ctas;
     int dtype, method, M;
@@ -35,7 +35,7 @@ struct TmaLaunch {
     cudaStream_t stream;
 };
 size_t tma_entry_bytes();
-int tma_warps_per_cta(int dtype, int M);
+int tma_warps_per_cta(int dtype, int M, int method);
 bool tma_eligible(const DevProblem& p, int N, int M, int method);
 bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M);
 cudaError_t tma_reduce(const void* entries_host, const void* entries_dev, int count, const double* partials, long long stride, cudaStream_t stream);

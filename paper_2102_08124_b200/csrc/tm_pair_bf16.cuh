@@ -95,15 +95,23 @@ __device__ __forceinline__ void relations_bf16(const PairKeys& k, Rel24& r) {
     complete_relations(r);
 }
 
-// Keep flags of a pair mask as 16-bit lane masks of the natural layout: for row i returns the four
-// words that select (a_i0,a_i1), (a_i2,a_i3), (b_i0,b_i1), (b_i2,b_i3).
-__device__ __forceinline__ void lane_masks(uint32_t kept, int i, uint32_t (&m)[4]) {
-    // t_j: bit 15 <- A(i,j), bit 31 <- B(i,j)
-    const uint32_t t0 = kept << (15 - 4 * i), t1 = kept << (14 - 4 * i), t2 = kept << (13 - 4 * i), t3 = kept << (12 - 4 * i);
-    m[0] = prmt(t0, t1, 0xDD99);   // bytes 0,1 <- sign of t0.byte1; bytes 2,3 <- sign of t1.byte1
-    m[1] = prmt(t2, t3, 0xDD99);
-    m[2] = prmt(t0, t1, 0xFFBB);   // same with byte 3 (block B)
-    m[3] = prmt(t2, t3, 0xFFBB);
+// Keep flags as 16-bit lane masks, by table: entry e of the 256-entry table holds four words whose
+// 16-bit lane j is all ones iff bit j of e is set.  The kernels build it in shared memory once per CTA.
+constexpr int kLaneLutBytes = 256 * 16;
+__device__ __forceinline__ void fill_lane_lut(uint4* lut, int tid, int nthreads) {
+    for (int e = tid; e < 256; e += nthreads) {
+        uint32_t w[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) w[c] = (((e >> (2 * c)) & 1) ? 0x0000FFFFu : 0u) | (((e >> (2 * c + 1)) & 1) ? 0xFFFF0000u : 0u);
+        lut[e] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+// The four mask bytes of a pair mask, byte i = (row i of block B) << 4 | (row i of block A): the layout
+// of the packed mask for the thread's eight columns.
+__device__ __forceinline__ uint32_t mask_bytes_2_4(uint32_t kept) {
+    const uint32_t t = kept & 0x0F0F0F0Fu, u = (kept >> 4) & 0x0F0F0F0Fu;      // rows 0,2 / rows 1,3 (A in bytes 0,1; B in bytes 2,3)
+    return prmt(t | (t >> 12), u | (u >> 12), 0x5140);
 }
 
 }  // namespace tmask

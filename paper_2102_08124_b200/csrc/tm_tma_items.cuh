@@ -1,6 +1,7 @@
 // Work-item bookkeeping shared by the bandwidth kernels: one descriptor record per matrix (tensor maps
 // for loads and stores plus the problem), a cursor that walks the items of a table of matrices in
-// order, and the host-side construction of the records.  An item is M rows x 256 columns.
+// order, and the host-side construction of the records.  An item is 8 rows x 256 columns (the last
+// item row of a matrix may be half empty when M = 4).
 #pragma once
 #include <cstring>
 
@@ -13,7 +14,7 @@ struct alignas(128) TmaEntry {
     CUtensorMap in, out;
     DevProblem p;
     int cchunks;       // items per block row (256 columns each)
-    int brows;         // block rows
+    int brows;         // item rows (8 matrix rows each)
 };
 static_assert(sizeof(TmaEntry) == 384 || sizeof(TmaEntry) == 512, "descriptor records stay 128-byte aligned in tables");
 
@@ -73,7 +74,7 @@ inline bool build_entries(const DevProblem* probs, int count, TmaEntry* e, long 
         memset(&e[k], 0, sizeof(TmaEntry));
         e[k].p = probs[k];
         e[k].cchunks = (int)((probs[k].cols + item_cols - 1) / item_cols);
-        e[k].brows = (int)(probs[k].rows / item_rows);
+        e[k].brows = (int)((probs[k].rows + item_rows - 1) / item_rows);
         e[k].p.item_begin = total;
         total += (long long)e[k].brows * e[k].cchunks;
         if (probs[k].rows == 0 || probs[k].cols == 0) continue;

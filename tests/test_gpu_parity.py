@@ -21,7 +21,7 @@ METHODS = [tm.TM_EXACT, tm.TM_APPROX, tm.TM_APPROX_COVER]
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_small_ragged_shapes(N, M, method, dtype):
     # several work items per block row, a ragged last item, a partial last mask word
-    for rows, cols, seed in [(5 * M, 70 * M, 1), (M, M, 2), (3 * M, 33 * M, 3), (2 * M, 32 * M, 4)]:
+    for rows, cols, seed in [(5 * M, 70 * M, 1), (M, M, 2), (3 * M, 33 * M, 3), (2 * M, 32 * M, 4), (7 * M, 301 * M, 5)]:
         W = workloads.normal_f32(rows, cols, 0.02, seed)
         if dtype == "bf16":
             W = workloads.f32_to_bf16_bits(W)
