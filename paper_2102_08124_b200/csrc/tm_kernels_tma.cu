@@ -43,8 +43,12 @@ template <int DT, int METHOD> struct Geometry {
     static constexpr int kRowPitch = kItemCols * kElem;        // bytes between rows inside a stage
     static constexpr int kHalfBytes = 4 * kRowPitch;           // one block row
     static constexpr int kStageBytes = kItemRows * kRowPitch;
-    // stages | mask bytes [8][32] | kept [2][32] | swap candidates [2][32] | queue [128] | barriers
-    static constexpr int kWarpBytes = kStages * kStageBytes + 256 + 2 * 256 + 128 + 64 + 64;
+    // Mask bytes of this many consecutive items are collected before they leave, so that a row's words go
+    // out as one longer run instead of 32-byte pieces.  Measured: it helps where the kernel waits for memory
+    // (Algorithm 1 alone) and costs more than it gives where it waits for the integer pipe (full search).
+    static constexpr int kMaskItems = DT == kF32 ? 4 : (METHOD == kMethodApprox ? 1 : 2);
+    // stages | mask bytes [items][8][32] | kept [2][32] | swap candidates [2][32] | queue [128] | barriers
+    static constexpr int kWarpBytes = kStages * kStageBytes + kMaskItems * 256 + 2 * 256 + 128 + 128;
     static constexpr int kSmemBytes = kWarps * kWarpBytes + (DT == kBF16 ? kLaneLutBytes : 0);
     static_assert(kSmemBytes <= 232448, "at most 227 KB of shared memory per CTA");
     static_assert(kWarpBytes % 128 == 0, "stages stay 128-byte aligned");
@@ -71,7 +75,8 @@ __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, 
 #pragma unroll
         for (int i = 0; i < 4; ++i) m[i] = max_u16x2(max_u16x2(pk.x[i][0], pk.x[i][1]), max_u16x2(pk.x[i][2], pk.x[i][3]));
         worst = max_u16x2(worst, max_u16x2(max_u16x2(m[0], m[1]), max_u16x2(m[2], m[3])));
-        relations_bf16(pk, rel);
+        if (__any_sync(0xFFFFFFFFu, nonfinite_bf16x2(worst))) relations_bf16<false>(pk, rel);      // bit-pattern order for Inf and NaN
+        else relations_bf16<true>(pk, rel);
     } else {
         uint32_t ka[16], kb[16];
 #pragma unroll
@@ -179,7 +184,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned char* stages = smem_raw + (size_t)warp * G::kWarpBytes;
     unsigned char* mbytes = stages + G::kStages * G::kStageBytes;
-    uint32_t* kbuf = reinterpret_cast<uint32_t*>(mbytes + 256);
+    uint32_t* kbuf = reinterpret_cast<uint32_t*>(mbytes + G::kMaskItems * 256);
     uint32_t* cbuf = kbuf + kHalves * 32;
     unsigned char* queue = reinterpret_cast<unsigned char*>(cbuf + kHalves * 32);
     uint64_t* bars = reinterpret_cast<uint64_t*>(queue + 128);
@@ -220,6 +225,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     uint32_t worst = 0;                                                  // largest magnitude pattern seen (per 16-bit lane for bf16)
     const uint32_t lt = (1u << lane) - 1u;
     bool alive = true;
+    int mfirst = -1;                                                     // first slot of the mask-byte buffer in use
 
     for (int it = 0; it < n_items && alive; ++it) {
         const int s = it % G::kStages;
@@ -292,21 +298,29 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         const int col0 = cur.cj * kItemCols + lane * 8;
         const int cols = (int)e.p.cols;
         const uint32_t colmask = col0 >= cols ? 0u : (col0 + 4 >= cols ? 0xFFFFu : 0xFFFFFFFFu);
+        const int slot = cur.cj & (G::kMaskItems - 1);
+        if (mfirst < 0) mfirst = slot;
 #pragma unroll
         for (int h = 0; h < kHalves; ++h)
-            facc += back_end<DT, HAS_OUT>(stage + h * G::kHalfBytes, mbytes + h * 128, lut, lane, kbuf[h * 32 + lane] & colmask);
+            facc += back_end<DT, HAS_OUT>(stage + h * G::kHalfBytes, mbytes + slot * 256 + h * 128, lut, lane, kbuf[h * 32 + lane] & colmask);
         if constexpr (HAS_OUT) fence_proxy_async_smem();
         __syncwarp();
         if constexpr (HAS_OUT) {
             if (lane == 0) { tma_store_2d(&e.out, cur.cj * kItemCols, cur.bi * kItemRows, stage); tma_commit(); }
         }
-        const long long rows = e.p.rows;
+        // mask words leave once the buffer holds the last item of an aligned group, of the block row or of this warp
+        if (slot == G::kMaskItems - 1 || cur.cj == cur.cchunks - 1 || it == n_items - 1) {
+            const long long rows = e.p.rows;
+            constexpr int kRowWords = 8 * G::kMaskItems;
+            const int word0 = (cur.cj - slot) * 8;
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {                               // 8 rows x 8 words of mask
-            const int idx = lane + 32 * hh, word = cur.cj * 8 + (idx & 7);
-            const long long row = (long long)cur.bi * kItemRows + (idx >> 3);
-            const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + (idx >> 3) * 32 + (idx & 7) * 4);
-            if (word < e.p.wpr && row < rows) e.p.mask[row * e.p.wpr + word] = w;
+            for (int t = 0; t < 2 * G::kMaskItems; ++t) {               // 8 rows x (8 words per item)
+                const int idx = lane + 32 * t, r = idx / kRowWords, wq = idx % kRowWords, q = wq >> 3;
+                const long long row = (long long)cur.bi * kItemRows + r;
+                const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + q * 256 + r * 32 + (wq & 7) * 4);
+                if (q >= mfirst && q <= slot && word0 + wq < e.p.wpr && row < rows) e.p.mask[row * e.p.wpr + word0 + wq] = w;
+            }
+            mfirst = -1;
         }
         cur.advance(tab, count);
         if ((it & 31) == 31) { acc += (double)facc; facc = 0.f; }           // keep the fp32 partial short
@@ -323,7 +337,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
     }
     if constexpr (DT == kF32) { if (worst >= 0x7F800000u) status |= kDevNonFinite; }
-    else { if ((worst & 0xFFFFu) >= 0x7F80u || (worst >> 16) >= 0x7F80u) status |= kDevNonFinite; }
+    else { if (nonfinite_bf16x2(worst)) status |= kDevNonFinite; }
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(0xFFFFFFFFu, status, o);
     if (lane == 0 && status && status_out) atomicOr(status_out, status);
 }

@@ -42,20 +42,40 @@ __device__ __forceinline__ uint32_t max_u16x2_(uint32_t a, uint32_t b) {
 
 // p[b] (bytes of equal bits) carries the decisions destined for bit 7-b of every byte (see gather8);
 // only bits 0..3 are wanted, the upper four come out as copies of p4
+template <bool NEG>                              // NEG: the four arrive negated
 __device__ __forceinline__ uint32_t gather4_low(uint32_t p7, uint32_t p6, uint32_t p5, uint32_t p4) {
-    return bitsel(bitsel(p7, p6, 0x01010101u), bitsel(p5, p4, 0x04040404u), 0x03030303u);
+    return bitsel(bitsel_n<NEG, NEG>(p7, p6, 0x01010101u), bitsel_n<NEG, NEG>(p5, p4, 0x04040404u), 0x03030303u);
 }
 
 // ---- bf16: packed comparisons ----------------------------------------------------------------
-// blk: row 0 of the lane's block inside the stage (row pitch 512 bytes)
-__device__ __forceinline__ void relations48_bf16(const unsigned char* blk, Rel48& rel, uint32_t& worst) {
-    uint32_t R[8][4];                              // R[i][c] = (|x_i,2c|, |x_i,2c+1|)
+// hr[K] from the row-paired magnitudes Y[i'][j] = (|x_2i',j|, |x_2i'+1,j|); for K = 4 only columns 0..3
+template <bool ARITH, int K>
+__device__ __forceinline__ u64 row_relation(const uint32_t (&Y)[4][8]) {
+    uint32_t word[2];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const uint4 v = *reinterpret_cast<const uint4*>(blk + i * 512);
-        R[i][0] = v.x & 0x7FFF7FFFu; R[i][1] = v.y & 0x7FFF7FFFu; R[i][2] = v.z & 0x7FFF7FFFu; R[i][3] = v.w & 0x7FFF7FFFu;
-        worst = max_u16x2_(worst, max_u16x2_(max_u16x2_(R[i][0], R[i][1]), max_u16x2_(R[i][2], R[i][3])));
+    for (int w = 0; w < 2; ++w) {
+        uint32_t pj[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (K == 4 && j >= 4) { pj[j] = 0; continue; }
+            const uint32_t d0 = (j + K <= 7) ? later_heavier<ARITH>(Y[2 * w][(j + K) & 7], Y[2 * w][j]) : earlier_heavier<ARITH>(Y[2 * w][(j + K) & 7], Y[2 * w][j]);
+            const uint32_t d1 = (j + K <= 7) ? later_heavier<ARITH>(Y[2 * w + 1][(j + K) & 7], Y[2 * w + 1][j]) : earlier_heavier<ARITH>(Y[2 * w + 1][(j + K) & 7], Y[2 * w + 1][j]);
+            pj[j] = prmt(d0, d1, 0xFDB9);      // bytes (0x00 / 0xFF) = rows 4w .. 4w+3 of column j
+        }
+        if constexpr (K == 4) {
+            word[w] = gather4_low<ARITH>(pj[0], pj[1], pj[2], pj[3]);
+        } else {
+            const uint32_t p[8] = {pj[7], pj[6], pj[5], pj[4], pj[3], pj[2], pj[1], pj[0]};
+            word[w] = gather8<ARITH ? (0xFFu & ~((1u << K) - 1u)) : 0u>(p);            // p[b] = column 7-b: a later partner iff b >= K
+        }
     }
+    return (u64)word[0] | ((u64)word[1] << 32);
+}
+
+// R[i][c] = (|x_i,2c|, |x_i,2c+1|) of the lane's block.  ARITH selects the form of the comparison (see
+// tm_pair_bf16.cuh): packed bf16 subtraction for finite data, integer subtraction for any bit pattern.
+template <bool ARITH>
+__device__ __forceinline__ void relations48_bf16(const uint32_t (&R)[8][4], Rel48& rel) {
     // column relations hc[k]: bit (i,j) <- rows (i, i+k mod 8) of column j.  One subtraction decides two
     // adjacent columns; byte permutes line the decisions up as (byte = row, all bits equal), a select tree packs them.
 #pragma unroll
@@ -71,14 +91,16 @@ __device__ __forceinline__ void relations48_bf16(const unsigned char* blk, Rel48
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
                     const int i = 4 * w + r;
-                    d[r] = (i + k <= 7) ? later_heavier(R[(i + k) & 7][c], R[i][c]) : earlier_heavier(R[(i + k) & 7][c], R[i][c]);
+                    d[r] = (i + k <= 7) ? later_heavier<ARITH>(R[(i + k) & 7][c], R[i][c]) : earlier_heavier<ARITH>(R[(i + k) & 7][c], R[i][c]);
                 }
                 const uint32_t q0 = prmt(d[0], d[1], 0xFBD9), q1 = prmt(d[2], d[3], 0xFBD9);      // decisions as whole bytes
                 cw[2 * c] = prmt(q0, q1, 0x5410);
                 cw[2 * c + 1] = prmt(q0, q1, 0x7632);
             }
             const uint32_t p[8] = {cw[7], cw[6], cw[5], cw[4], cw[3], cw[2], cw[1], cw[0]};
-            word[w] = gather8(p);
+            word[w] = gather8<ARITH ? 0xFFu : 0u>(p);
+            // rows that wrap around (i + k > 7) compare with an earlier entry: their decisions were not negated
+            if constexpr (ARITH) { if (w == 1) word[w] ^= 0xFFFFFFFFu << (8 * (4 - k)); }
         }
         rel.hc[k] = (u64)word[0] | ((u64)word[1] << 32);
     }
@@ -91,28 +113,8 @@ __device__ __forceinline__ void relations48_bf16(const unsigned char* blk, Rel48
             Y[ip][2 * c] = prmt(R[2 * ip][c], R[2 * ip + 1][c], 0x5410);
             Y[ip][2 * c + 1] = prmt(R[2 * ip][c], R[2 * ip + 1][c], 0x7632);
         }
-#pragma unroll
-    for (int k = 1; k <= 4; ++k) {
-        uint32_t word[2];
-#pragma unroll
-        for (int w = 0; w < 2; ++w) {
-            uint32_t pj[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (k == 4 && j >= 4) { pj[j] = 0; continue; }
-                const uint32_t d0 = (j + k <= 7) ? later_heavier(Y[2 * w][(j + k) & 7], Y[2 * w][j]) : earlier_heavier(Y[2 * w][(j + k) & 7], Y[2 * w][j]);
-                const uint32_t d1 = (j + k <= 7) ? later_heavier(Y[2 * w + 1][(j + k) & 7], Y[2 * w + 1][j]) : earlier_heavier(Y[2 * w + 1][(j + k) & 7], Y[2 * w + 1][j]);
-                pj[j] = prmt(d0, d1, 0xFDB9);      // bytes (0x00 / 0xFF) = rows 4w .. 4w+3 of column j
-            }
-            if (k == 4) {
-                word[w] = gather4_low(pj[0], pj[1], pj[2], pj[3]);
-            } else {
-                const uint32_t p[8] = {pj[7], pj[6], pj[5], pj[4], pj[3], pj[2], pj[1], pj[0]};
-                word[w] = gather8(p);
-            }
-        }
-        rel.hr[k] = (u64)word[0] | ((u64)word[1] << 32);
-    }
+    rel.hr[1] = row_relation<ARITH, 1>(Y); rel.hr[2] = row_relation<ARITH, 2>(Y);
+    rel.hr[3] = row_relation<ARITH, 3>(Y); rel.hr[4] = row_relation<ARITH, 4>(Y);
     complete_relations8(rel);
 }
 
@@ -293,7 +295,19 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         unsigned char* blk = stage + lane * (8 * G::kElem);
 
         Rel48 rel;
-        if constexpr (DT == kBF16) relations48_bf16(blk, rel, worst); else relations48_f32(blk, rel, worst);
+        if constexpr (DT == kBF16) {
+            uint32_t R[8][4];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint4 v = *reinterpret_cast<const uint4*>(blk + i * 512);
+                R[i][0] = v.x & 0x7FFF7FFFu; R[i][1] = v.y & 0x7FFF7FFFu; R[i][2] = v.z & 0x7FFF7FFFu; R[i][3] = v.w & 0x7FFF7FFFu;
+                worst = max_u16x2_(worst, max_u16x2_(max_u16x2_(R[i][0], R[i][1]), max_u16x2_(R[i][2], R[i][3])));
+            }
+            if (__any_sync(0xFFFFFFFFu, nonfinite_bf16x2(worst))) relations48_bf16<false>(R, rel);      // bit-pattern order for Inf and NaN
+            else relations48_bf16<true>(R, rel);
+        } else {
+            relations48_f32(blk, rel, worst);
+        }
         u64 kept = cover_4_8(rel);
         if constexpr (METHOD == kMethodApprox) {
             Short48 L = line_short(kept);
@@ -356,7 +370,7 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
     }
     if constexpr (DT == kF32) { if (worst >= 0x7F800000u) status |= kDevNonFinite; }
-    else { if ((worst & 0xFFFFu) >= 0x7F80u || (worst >> 16) >= 0x7F80u) status |= kDevNonFinite; }
+    else { if (nonfinite_bf16x2(worst)) status |= kDevNonFinite; }
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(0xFFFFFFFFu, status, o);
     if (lane == 0 && status && status_out) atomicOr(status_out, status);
 }

@@ -3,11 +3,19 @@
 // Input: the thread's 4 rows x 8 bf16 (block A = columns 0..3, block B = columns 4..7) as four
 // 128-bit words.  The sixteen magnitudes of both blocks are interleaved into sixteen registers
 // X[i][j] = (|a_ij|, |b_ij|) (16-bit lanes), so that every comparison the search needs -- entries
-// sharing a row or a column -- is one 32-bit subtraction deciding the same pair in both blocks:
-//   X_q - X_p + 0x80008000  has bit 15 / bit 31 set iff  q >= p  in block A / block B
-// (15-bit magnitudes: no borrow crosses the lanes).  The 48 decisions are then collected into the
-// relation masks of tm_core24.cuh: a byte permute in sign-replicating mode turns every decision into a
-// whole byte of equal bits, so a tree of bit selects with constant masks places them without shifts.
+// sharing a row or a column -- is one 32-bit instruction deciding the same pair in both blocks.
+// Two forms of that instruction exist:
+//   arithmetic  X_q - X_p as a packed bf16 subtraction: the sign of either lane says "q lighter than
+//               p" (a difference of two finite bf16 numbers never rounds to zero or across zero).  It
+//               runs on the floating-point pipe, which the search leaves idle; it is used while every
+//               magnitude seen is finite;
+//   integer     X_q - X_p + 0x80008000 has bit 15 / bit 31 set iff q >= p (15-bit magnitudes: no
+//               borrow crosses the lanes).  It orders any bit patterns, Inf and NaN included, and takes
+//               over as soon as a warp has met one.
+// The 48 decisions are then collected into the relation masks of tm_core24.cuh: a byte permute in
+// sign-replicating mode turns every decision into a whole byte of equal bits, so a tree of bit
+// selects with constant masks places them without shifts; decisions that arrive negated (the
+// arithmetic form of ">=") are turned in the first level of the tree at no cost.
 #pragma once
 #include "tm_core24.cuh"
 
@@ -22,6 +30,14 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 __device__ __forceinline__ uint32_t bitsel(uint32_t a, uint32_t b, uint32_t m) {
     uint32_t r;
     asm("lop3.b32 %0, %1, %2, %3, 0xCA;" : "=r"(r) : "r"(m), "r"(a), "r"(b));   // m ? a : b
+    return r;
+}
+// the same with a and / or b complemented first
+template <bool NA, bool NB>
+__device__ __forceinline__ uint32_t bitsel_n(uint32_t a, uint32_t b, uint32_t m) {
+    constexpr int lut = (0xF0 & (NA ? 0x33 : 0xCC)) | (0x0F & (NB ? 0x55 : 0xAA));
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, %4;" : "=r"(r) : "r"(m), "r"(a), "r"(b), "n"(lut));
     return r;
 }
 
@@ -39,21 +55,37 @@ __device__ __forceinline__ void interleave_keys(const uint4 (&v)[4], PairKeys& k
     }
 }
 
-// decision words: "q heavier than p" for positions q > p (ties go to the later position) ...
-__device__ __forceinline__ uint32_t later_heavier(uint32_t xq, uint32_t xp) { return xq - xp + 0x80008000u; }
-// ... and for q < p (strictly larger magnitude needed)
-__device__ __forceinline__ uint32_t earlier_heavier(uint32_t xq, uint32_t xp) { return xq - xp + 0x7FFF7FFFu; }
+// Decision words.  ARITH = false: the top bit of either 16-bit lane says "q heavier than p".
+// ARITH = true: later_heavier() returns the negated decision (sign of X_q - X_p = "q lighter"),
+// earlier_heavier() the plain one (sign of X_p - X_q = "p lighter").
+__device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+// q > p in position: ties go to q
+template <bool ARITH> __device__ __forceinline__ uint32_t later_heavier(uint32_t xq, uint32_t xp) {
+    if constexpr (ARITH) return sub_bf16x2(xq, xp); else return xq - xp + 0x80008000u;
+}
+// q < p in position: a strictly larger magnitude is needed
+template <bool ARITH> __device__ __forceinline__ uint32_t earlier_heavier(uint32_t xq, uint32_t xp) {
+    if constexpr (ARITH) return sub_bf16x2(xp, xq); else return xq - xp + 0x7FFF7FFFu;
+}
 
 // byte 0/1 <- decisions of dx/dy for block A, byte 2/3 <- for block B; every byte is 0x00 or 0xFF
 __device__ __forceinline__ uint32_t pick(uint32_t dx, uint32_t dy) { return prmt(dx, dy, 0xFBD9); }
 
-// p[b] (bytes of equal bits) carries the decisions destined for bit 7-b of every byte
+// p[b] (bytes of equal bits) carries the decision destined for bit 7-b of every byte, negated where bit b of NEG is set
+template <unsigned NEG>
 __device__ __forceinline__ uint32_t gather8(const uint32_t (&p)[8]) {
-    const uint32_t t01 = bitsel(p[0], p[1], 0x80808080u), t23 = bitsel(p[2], p[3], 0x20202020u);
-    const uint32_t t45 = bitsel(p[4], p[5], 0x08080808u), t67 = bitsel(p[6], p[7], 0x02020202u);
+    const uint32_t t01 = bitsel_n<(NEG & 1) != 0, (NEG & 2) != 0>(p[0], p[1], 0x80808080u);
+    const uint32_t t23 = bitsel_n<(NEG & 4) != 0, (NEG & 8) != 0>(p[2], p[3], 0x20202020u);
+    const uint32_t t45 = bitsel_n<(NEG & 16) != 0, (NEG & 32) != 0>(p[4], p[5], 0x08080808u);
+    const uint32_t t67 = bitsel_n<(NEG & 64) != 0, (NEG & 128) != 0>(p[6], p[7], 0x02020202u);
     return bitsel(bitsel(t01, t23, 0xC0C0C0C0u), bitsel(t45, t67, 0x0C0C0C0Cu), 0xF0F0F0F0u);
 }
 
+template <bool ARITH>
 __device__ __forceinline__ void relations_bf16(const PairKeys& k, Rel24& r) {
     const uint32_t (&x)[4][4] = k.x;
     uint32_t p[8];
@@ -61,39 +93,44 @@ __device__ __forceinline__ void relations_bf16(const PairKeys& k, Rel24& r) {
 #pragma unroll
     for (int b = 0; b < 8; ++b) {
         const int i = (7 - b) >> 2, j = (7 - b) & 3;
-        const uint32_t dx = j < 3 ? later_heavier(x[i][j + 1], x[i][j]) : earlier_heavier(x[i][0], x[i][3]);
-        const uint32_t dy = j < 3 ? later_heavier(x[i + 2][j + 1], x[i + 2][j]) : earlier_heavier(x[i + 2][0], x[i + 2][3]);
+        const uint32_t dx = j < 3 ? later_heavier<ARITH>(x[i][j + 1], x[i][j]) : earlier_heavier<ARITH>(x[i][0], x[i][3]);
+        const uint32_t dy = j < 3 ? later_heavier<ARITH>(x[i + 2][j + 1], x[i + 2][j]) : earlier_heavier<ARITH>(x[i + 2][0], x[i + 2][3]);
         p[b] = pick(dx, dy);
     }
-    r.hr1 = gather8(p);
+    r.hr1 = gather8<ARITH ? 0xEEu : 0u>(p);                           // j = 3 (b = 0 and 4) compares with an earlier entry
     // hc1: bit 4i+j <- pair (i, i+1 mod 4) of column j
 #pragma unroll
     for (int b = 0; b < 8; ++b) {
         const int i = (7 - b) >> 2, j = (7 - b) & 3;                  // i in {0,1}; the partner byte holds i+2
-        const uint32_t dx = later_heavier(x[i + 1][j], x[i][j]);
-        const uint32_t dy = (i + 2 < 3) ? later_heavier(x[(i + 3) & 3][j], x[i + 2][j]) : earlier_heavier(x[0][j], x[3][j]);
+        const uint32_t dx = later_heavier<ARITH>(x[i + 1][j], x[i][j]);
+        uint32_t dy;
+        if (i + 2 < 3) dy = later_heavier<ARITH>(x[(i + 3) & 3][j], x[i + 2][j]);
+        else { dy = earlier_heavier<ARITH>(x[0][j], x[3][j]); if constexpr (ARITH) dy ^= 0x80008000u; }    // same sense as dx
         p[b] = pick(dx, dy);
     }
-    r.hc1 = gather8(p);
+    r.hc1 = gather8<ARITH ? 0xFFu : 0u>(p);
     // hr2 (columns 0,1 only): bits 4i+j, j in {0,1}
     {
-        const uint32_t q7 = pick(later_heavier(x[0][2], x[0][0]), later_heavier(x[2][2], x[2][0]));
-        const uint32_t q6 = pick(later_heavier(x[0][3], x[0][1]), later_heavier(x[2][3], x[2][1]));
-        const uint32_t q3 = pick(later_heavier(x[1][2], x[1][0]), later_heavier(x[3][2], x[3][0]));
-        const uint32_t q2 = pick(later_heavier(x[1][3], x[1][1]), later_heavier(x[3][3], x[3][1]));
-        r.hr2 = bitsel(bitsel(q7, q6, 0x01010101u), bitsel(q3, q2, 0x10101010u), 0x0F0F0F0Fu);      // bits 2,3 of a nibble: don't care
+        const uint32_t q7 = pick(later_heavier<ARITH>(x[0][2], x[0][0]), later_heavier<ARITH>(x[2][2], x[2][0]));
+        const uint32_t q6 = pick(later_heavier<ARITH>(x[0][3], x[0][1]), later_heavier<ARITH>(x[2][3], x[2][1]));
+        const uint32_t q3 = pick(later_heavier<ARITH>(x[1][2], x[1][0]), later_heavier<ARITH>(x[3][2], x[3][0]));
+        const uint32_t q2 = pick(later_heavier<ARITH>(x[1][3], x[1][1]), later_heavier<ARITH>(x[3][3], x[3][1]));
+        r.hr2 = bitsel(bitsel_n<ARITH, ARITH>(q7, q6, 0x01010101u), bitsel_n<ARITH, ARITH>(q3, q2, 0x10101010u), 0x0F0F0F0Fu);   // bits 2,3 of a nibble: don't care
     }
     // hc2 (rows 0,1 only): bit 4i+j, i in {0,1}; gathered as (row 0 -> byte 0, row 1 -> byte 1), then packed
     {
         uint32_t q[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) q[j] = pick(later_heavier(x[2][j], x[0][j]), later_heavier(x[3][j], x[1][j]));
-        const uint32_t g = bitsel(bitsel(q[0], q[1], 0x01010101u), bitsel(q[2], q[3], 0x04040404u), 0x03030303u);
+        for (int j = 0; j < 4; ++j) q[j] = pick(later_heavier<ARITH>(x[2][j], x[0][j]), later_heavier<ARITH>(x[3][j], x[1][j]));
+        const uint32_t g = bitsel(bitsel_n<ARITH, ARITH>(q[0], q[1], 0x01010101u), bitsel_n<ARITH, ARITH>(q[2], q[3], 0x04040404u), 0x03030303u);
         r.hc2 = bitsel(g, g >> 4, 0x0F0F0F0Fu);
     }
     r.hr3 = 0; r.hc3 = 0;
     complete_relations(r);
 }
+
+// Some 16-bit lane of `worst` (a running maximum of magnitudes) is Inf or NaN.
+__device__ __forceinline__ bool nonfinite_bf16x2(uint32_t worst) { return ((worst + 0x00800080u) & 0x80008000u) != 0; }
 
 // Keep flags as 16-bit lane masks, by table: entry e of the 256-entry table holds four words whose
 // 16-bit lane j is all ones iff bit j of e is set.  The kernels build it in shared memory once per CTA.

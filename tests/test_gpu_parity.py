@@ -88,6 +88,33 @@ def test_nonfinite_inputs_raise_the_status_bit(N, M):
 
 
 @pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
+def test_bf16_nonfinite_inputs_follow_the_bit_pattern_order(N, M):
+    """Inf and several NaN patterns inside bf16 data: the packed-subtraction comparisons must give way to the
+    integer ones for the whole warp, before and after the first such value is met."""
+    W = workloads.normal_bf16(6 * M, 300 * M, 0.02, 31)
+    W[1, 3] = 0x7F80; W[2, 5] = 0xFF80; W[M + 1, 7 * M] = 0x7FC0; W[M + 1, 7 * M + 1] = 0x7F81; W[M + 2, 7 * M + 1] = 0xFFFF
+    W[5 * M + 3, 299 * M + 2] = 0x7FFF; W[5 * M + 2, 299 * M + 2] = 0x7FA0
+    for method in (tm.TM_APPROX, tm.TM_APPROX_COVER):
+        assert_parity(W, N, M, method, rel=None)
+
+
+@pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
+def test_bf16_subnormals_and_extremes_compare_exactly(N, M):
+    """Subnormal, smallest-normal and largest finite bf16 magnitudes, many of them equal or one step apart."""
+    rng = np.random.Generator(np.random.PCG64(32))
+    rows, cols = 4 * M, 160 * M
+    W = rng.integers(0, 0x0100, size=(rows, cols)).astype(np.uint16)            # subnormals and the first normals
+    W[:, ::3] = rng.integers(0x7000, 0x7080, size=W[:, ::3].shape).astype(np.uint16)     # large values, close together
+    W[::2, ::5] = rng.integers(0, 4, size=W[::2, ::5].shape).astype(np.uint16)
+    W |= (rng.integers(0, 2, size=W.shape).astype(np.uint16) << 15)
+    V = W.copy()
+    V[1::3, 1::7] = rng.integers(0x7F70, 0x7F80, size=V[1::3, 1::7].shape).astype(np.uint16)   # up to the largest finite value
+    for method in (tm.TM_APPROX, tm.TM_APPROX_COVER):
+        assert_parity(W, N, M, method, rel=1e-6)
+        assert_parity(V, N, M, method, rel=None)                        # fp32 partial sums may overflow here
+
+
+@pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
 def test_optional_outputs_and_in_place(N, M):
     W = workloads.normal_f32(4 * M, 45 * M, 0.02, 13)
     want = orc.find_mask(W, N, M, orc.APPROX)
