@@ -33,7 +33,7 @@ ROWS = FULL_ROWS
 N_KEEP, M_BLOCK = 2, 4
 BYTES_PER_WEIGHT = 2 + 2 + 1.0 / 8          # read W, write masked W, write one mask bit (bf16)
 # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture on the 2048-row case (see profiles/), per weight
-TRAFFIC_PER_WEIGHT = (201.39e6 + 165.37e6) / (2048 * 49152)
+TRAFFIC_PER_WEIGHT = (201.37e6 + 163.01e6) / (2048 * 49152)
 TRAFFIC_SOURCE = "ncu --set full on the 2048 x 49152 case, scaled by rows (profiles/tma24_kernel_approx_2_4_bf16_2048x49152_full.md)"
 METRIC = "transposable-mask weights/s (2:4 approx, bf16, 1 GPU: achieved HBM GB/s vs peak in `roofline`)"
 WORKLOAD = "%dx49152 bf16, N(0,0.02) quantised to 256 levels (frequent ties), 2:4 approximate, per-step recompute"
@@ -76,7 +76,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         try:
             for line in open(self.path):
                 f = [x.strip() for x in line.split(",")]
@@ -86,6 +86,10 @@ class ClockSampler:
                     sm.append(float(f[1])); mx.append(float(f[2]))
                 except ValueError:
                     continue
+                try:
+                    pw.append(float(f[3]))
+                except ValueError:
+                    pass
                 for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                     if val.lower().startswith("active"):
                         reasons.add(name)
@@ -93,7 +97,8 @@ class ClockSampler:
         except Exception:
             pass
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm),
+                       power_w=statistics.median(pw) if pw else None)
         return out
 
 
@@ -169,6 +174,18 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    # a first look before the part heats up: W warm-up steps, K timed steps (reported beside the main number)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sync()
+    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    b0.record()
+    for _ in range(args.steps):
+        step()
+    b1.record()
+    sync()
+    ms_cold = b0.elapsed_time(b1) / args.steps
+
     # warm-up: at least W steps and long enough for the clock sampler (started first) to see the GPU under load
     sampler = ClockSampler(local_rank)
     if rank == 0 and not args.skip_clocks:
@@ -242,6 +259,9 @@ def run_gpu(args):
                      "traffic": TRAFFIC_PER_WEIGHT * weights if ROWS == FULL_ROWS else None, "traffic_source": TRAFFIC_SOURCE,
                      "peak_source": peak_src, "algorithmic_bytes_per_launch": weights * BYTES_PER_WEIGHT,
                      "frac_of_8000": achieved / 8000.0,
+                     "cold": {"ms_per_step": ms_cold, "achieved": weights * BYTES_PER_WEIGHT / (ms_cold * 1e-3) / 1e9,
+                              "frac": weights * BYTES_PER_WEIGHT / (ms_cold * 1e-3) / 1e9 / peak,
+                              "note": "the same K steps timed right after W warm-up steps, before the sustained warm-up under the clock sampler"},
                      "note": "duration = CUDA-event time of one step (search kernel + its tiny partial-zeroing and reduction launches)"},
         "cpu_baseline": {"value": cpu_value, "unit": "weights/s", "cores": 1, "kind": "oracle",
                          "sample": "first %d rows of the matrix (%d weights), %.1f s" % (cpu_rows, cpu_rows * COLS, cpu_dt)},
