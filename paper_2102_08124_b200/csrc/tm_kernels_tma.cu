@@ -70,12 +70,15 @@ __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, 
 #pragma unroll
         for (int i = 0; i < 4; ++i) v[i] = *reinterpret_cast<const uint4*>(stage + i * 512 + lane * 16);
         PairKeys pk;
-        interleave_keys(v, pk);
+        interleave_keys<true>(v, pk);
         uint32_t m[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) m[i] = max_u16x2(max_u16x2(pk.x[i][0], pk.x[i][1]), max_u16x2(pk.x[i][2], pk.x[i][3]));
         worst = max_u16x2(worst, max_u16x2(max_u16x2(m[0], m[1]), max_u16x2(m[2], m[3])));
-        if (__any_sync(0xFFFFFFFFu, nonfinite_bf16x2(worst))) relations_bf16<false>(pk, rel);      // bit-pattern order for Inf and NaN
+        if (__any_sync(0xFFFFFFFFu, nonfinite_bf16x2(worst))) {        // Inf or NaN met: integer keys, bit-pattern order
+            interleave_keys<false>(v, pk);
+            relations_bf16<false>(pk, rel);
+        }
         else relations_bf16<true>(pk, rel);
     } else {
         uint32_t ka[16], kb[16];
@@ -148,7 +151,7 @@ __device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* m
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 o[q] = raw[q] & m[q];
-                const uint32_t ab = raw[q] & m[q] & 0x7FFF7FFFu;
+                const uint32_t ab = abs_bf16x2(o[q]);
                 unsigned short lo, hi;
                 asm("mov.b32 {%0,%1}, %2;" : "=h"(lo), "=h"(hi) : "r"(ab));
                 asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(s4) : "h"(lo));        // fp32 accumulator + bf16 addend

@@ -209,7 +209,7 @@ __device__ __forceinline__ float back_end48(unsigned char* blk, unsigned char* m
             for (int c = 0; c < 4; ++c) {
                 const uint32_t m = m4[c];
                 o[c] = raw[c] & m;
-                const uint32_t ab = raw[c] & m & 0x7FFF7FFFu;
+                const uint32_t ab = abs_bf16x2(o[c]);
                 unsigned short lo, hi;
                 asm("mov.b32 {%0,%1}, %2;" : "=h"(lo), "=h"(hi) : "r"(ab));
                 asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(s8) : "h"(lo));
@@ -300,11 +300,19 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const uint4 v = *reinterpret_cast<const uint4*>(blk + i * 512);
-                R[i][0] = v.x & 0x7FFF7FFFu; R[i][1] = v.y & 0x7FFF7FFFu; R[i][2] = v.z & 0x7FFF7FFFu; R[i][3] = v.w & 0x7FFF7FFFu;
+                R[i][0] = abs_bf16x2(v.x); R[i][1] = abs_bf16x2(v.y); R[i][2] = abs_bf16x2(v.z); R[i][3] = abs_bf16x2(v.w);
                 worst = max_u16x2_(worst, max_u16x2_(max_u16x2_(R[i][0], R[i][1]), max_u16x2_(R[i][2], R[i][3])));
             }
-            if (__any_sync(0xFFFFFFFFu, nonfinite_bf16x2(worst))) relations48_bf16<false>(R, rel);      // bit-pattern order for Inf and NaN
-            else relations48_bf16<true>(R, rel);
+            if (__any_sync(0xFFFFFFFFu, nonfinite_bf16x2(worst))) {        // Inf or NaN met: integer keys, bit-pattern order
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(blk + i * 512);
+                    R[i][0] = v.x & 0x7FFF7FFFu; R[i][1] = v.y & 0x7FFF7FFFu; R[i][2] = v.z & 0x7FFF7FFFu; R[i][3] = v.w & 0x7FFF7FFFu;
+                }
+                relations48_bf16<false>(R, rel);
+            } else {
+                relations48_bf16<true>(R, rel);
+            }
         } else {
             relations48_f32(blk, rel, worst);
         }

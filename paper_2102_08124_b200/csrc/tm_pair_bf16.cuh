@@ -45,13 +45,23 @@ struct PairKeys {
     uint32_t x[4][4];   // (|a_ij|, |b_ij|)
 };
 
+// |x| of both lanes on the floating-point pipe; bit-exact for every finite value and Inf (a NaN may
+// come back with another payload, which the integer path below never sees)
+__device__ __forceinline__ uint32_t abs_bf16x2(uint32_t a) {
+    uint32_t r;
+    asm("abs.bf16x2 %0, %1;" : "=r"(r) : "r"(a));
+    return r;
+}
+
+// ARITH = false clears the sign bits with integer logic instead (exact for every bit pattern)
+template <bool ARITH>
 __device__ __forceinline__ void interleave_keys(const uint4 (&v)[4], PairKeys& k) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        k.x[i][0] = prmt(v[i].x, v[i].z, 0x5410) & 0x7FFF7FFFu;
-        k.x[i][1] = prmt(v[i].x, v[i].z, 0x7632) & 0x7FFF7FFFu;
-        k.x[i][2] = prmt(v[i].y, v[i].w, 0x5410) & 0x7FFF7FFFu;
-        k.x[i][3] = prmt(v[i].y, v[i].w, 0x7632) & 0x7FFF7FFFu;
+        const uint32_t a = prmt(v[i].x, v[i].z, 0x5410), b = prmt(v[i].x, v[i].z, 0x7632);
+        const uint32_t c = prmt(v[i].y, v[i].w, 0x5410), d = prmt(v[i].y, v[i].w, 0x7632);
+        if constexpr (ARITH) { k.x[i][0] = abs_bf16x2(a); k.x[i][1] = abs_bf16x2(b); k.x[i][2] = abs_bf16x2(c); k.x[i][3] = abs_bf16x2(d); }
+        else { k.x[i][0] = a & 0x7FFF7FFFu; k.x[i][1] = b & 0x7FFF7FFFu; k.x[i][2] = c & 0x7FFF7FFFu; k.x[i][3] = d & 0x7FFF7FFFu; }
     }
 }
 
@@ -129,8 +139,9 @@ __device__ __forceinline__ void relations_bf16(const PairKeys& k, Rel24& r) {
     complete_relations(r);
 }
 
-// Some 16-bit lane of `worst` (a running maximum of magnitudes) is Inf or NaN.
-__device__ __forceinline__ bool nonfinite_bf16x2(uint32_t worst) { return ((worst + 0x00800080u) & 0x80008000u) != 0; }
+// Some 16-bit lane of `worst` (a running maximum of magnitudes) is Inf or NaN.  The sign bits are
+// ignored: the arithmetic |x| may hand a NaN back with its sign still set.
+__device__ __forceinline__ bool nonfinite_bf16x2(uint32_t worst) { return (((worst & 0x7FFF7FFFu) + 0x00800080u) & 0x80008000u) != 0; }
 
 // Keep flags as 16-bit lane masks, by table: entry e of the 256-entry table holds four words whose
 // 16-bit lane j is all ones iff bit j of e is set.  The kernels build it in shared memory once per CTA.
