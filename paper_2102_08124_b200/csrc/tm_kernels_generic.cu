@@ -97,6 +97,12 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
     const long long end = min(total_items, begin + per);
     const DevProblem* tab = table ? table : &single;
 
+    // per-thread columns of the flow solver's state (only the exact instantiations that use it get dynamic shared memory)
+    extern __shared__ __align__(16) unsigned char flow_smem[];
+    uint4* spot = reinterpret_cast<uint4*>(flow_smem) + threadIdx.x;
+    uint4* sdist = spot + 2 * M * (kWarpsPerCta * 32);
+    uint32_t* su = reinterpret_cast<uint32_t*>(flow_smem + 2 * (2 * M) * 16 * (kWarpsPerCta * 32)) + threadIdx.x;
+
     int k = 0, status = 0;
     double acc = 0.0;
     int acc_k = -1;
@@ -129,7 +135,7 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
         uint64_t kept;
         if constexpr (METHOD == kMethodExact) {
             if constexpr (M == 4 && N == 2) kept = exact_2_4(u, P.dtype == kBF16 ? 16 : 0);
-            else kept = exact_ssp<N, M>(u, status);
+            else kept = exact_ssp<N, M>(u, status, su, spot, sdist, kWarpsPerCta * 32);
         } else {
             kept = cover_mask<N, M>(u);
             if constexpr (METHOD == kMethodApprox) {
@@ -197,7 +203,18 @@ template <int N, int M>
 cudaError_t launch_nm(const LaunchArgs& a) {
     const dim3 grid((unsigned)a.ctas), block(kWarpsPerCta * 32);
     switch (a.method) {
-    case kMethodExact: generic_kernel<N, M, kMethodExact><<<grid, block, 0, a.stream>>>(a.single, a.table, a.count, a.total_items, a.partials, a.status); break;
+    case kMethodExact: {
+        // the flow solver (everything but 2:4) keeps its state in shared memory
+        constexpr size_t smem = (N == 2 && M == 4) ? 0 : (size_t)flow_shared_bytes_per_thread(M) * kWarpsPerCta * 32;
+        static bool configured = false;    // per instantiation
+        if (smem > 48 * 1024 && !configured) {
+            cudaError_t e = cudaFuncSetAttribute(generic_kernel<N, M, kMethodExact>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            configured = true;
+        }
+        generic_kernel<N, M, kMethodExact><<<grid, block, smem, a.stream>>>(a.single, a.table, a.count, a.total_items, a.partials, a.status);
+        break;
+    }
     case kMethodApprox: generic_kernel<N, M, kMethodApprox><<<grid, block, 0, a.stream>>>(a.single, a.table, a.count, a.total_items, a.partials, a.status); break;
     default: generic_kernel<N, M, kMethodCover><<<grid, block, 0, a.stream>>>(a.single, a.table, a.count, a.total_items, a.partials, a.status); break;
     }

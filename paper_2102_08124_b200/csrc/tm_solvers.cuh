@@ -436,14 +436,143 @@ __device__ __noinline__ uint64_t exact_flow_run(const uint32_t (&u)[M * M], int 
     return ~pruned & all;
 }
 
+// The same repair written for a whole warp at once: one block per lane, state in shared memory, and one
+// instruction stream for all lanes.  The scalar version above branches on the node it has just settled, so
+// the 32 lanes of a warp drift apart and execute one after the other; here every data-dependent choice is a
+// select or a predicated store, every loop is uniform (a vote ends it when no lane needs another turn), and
+// a settled node's row and column cases share one body.  A thread's magnitudes, potentials and distances
+// are three strided columns (stride T entries); predecessors and column loads are packed four bits each
+// into registers.  Must be called by all 32 lanes; lanes with `enabled` false take part in the votes only.
+constexpr int flow_shared_bytes_per_thread(int M) { return M * M * 4 + 2 * (2 * M) * 16; }
+
+__device__ __forceinline__ __int128 ld128(const uint4* p) {
+    const uint4 v = *p;
+    return (__int128)(((unsigned __int128)(((unsigned long long)v.w << 32) | v.z) << 64) | (((unsigned long long)v.y << 32) | v.x));
+}
+__device__ __forceinline__ void st128(uint4* p, __int128 x) {
+    const unsigned long long lo = (unsigned long long)x, hi = (unsigned long long)((unsigned __int128)x >> 64);
+    *p = make_uint4((uint32_t)lo, (uint32_t)(lo >> 32), (uint32_t)hi, (uint32_t)(hi >> 32));
+}
+__device__ __forceinline__ __int128 edge_cost128(uint32_t u, int Emin, int p) {
+    uint32_t sig; int E; split_float(u, sig, E);
+    return ((__int128)((long long)sig << (sig ? E - Emin : 0)) << 64) + ((__int128)1 << p);
+}
+
 template <int N, int M>
-__device__ __forceinline__ uint64_t exact_ssp(const uint32_t (&u)[M * M], int& status) {
+__device__ __noinline__ uint64_t exact_flow_warp(const uint32_t (&u)[M * M], int Emin, bool enabled, int& status,
+                                                 uint32_t* su, uint4* spot, uint4* sdist, int T) {
+    constexpr int P = M - N;
+    constexpr unsigned kFull = 0xFFFFFFFFu;
+    uint64_t pruned = 0;
+    uint32_t load = 0;                                                  // nibble j: pruned entries of column j
+#pragma unroll
+    for (int j = 0; j < M; ++j) st128(spot + (M + j) * T, 0);
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+#pragma unroll
+        for (int j = 0; j < M; ++j) {
+            su[(i * M + j) * T] = u[i * M + j];
+            int heavier = 0;
+#pragma unroll
+            for (int k = 0; k < M; ++k)
+                heavier += (k != j) && (u[i * M + k] > u[i * M + j] || (u[i * M + k] == u[i * M + j] && k > j));
+            if (heavier >= N) { pruned |= 1ull << (i * M + j); load += 1u << (4 * j); }
+            if (heavier == N) st128(spot + i * T, -edge_cost128(u[i * M + j], Emin, i * M + j));   // reduced cost c + pot[row] - pot[col]: <= 0 pruned, >= 0 kept
+        }
+    }
+    bool failed = false;
+    for (int unit = 0; unit <= M * P; ++unit) {
+        unsigned reach = 0, done = 0;
+        uint64_t pre = 0;                                               // nibble n: predecessor of node n
+#pragma unroll
+        for (int j = 0; j < M; ++j) {
+            const bool over = enabled && !failed && (int)((load >> (4 * j)) & 15u) > P;
+            if (over) st128(sdist + (M + j) * T, 0);
+            reach |= (over ? 1u : 0u) << (M + j);
+        }
+        const unsigned sources = reach;
+        const bool active = reach != 0;                                 // this lane's columns are not all at M-N yet
+        if (!__any_sync(kFull, active)) break;
+        if (unit == M * P) { failed |= active; break; }
+        int target = -1;
+        for (int step = 0; step < 2 * M; ++step) {
+            const bool searching = active && target < 0;
+            if (!__any_sync(kFull, searching)) break;
+            // settle the open node at the smallest distance
+            const unsigned open = searching ? (reach & ~done) : 0u;
+            int v = -1; __int128 dv = 0;
+#pragma unroll
+            for (int n = 0; n < 2 * M; ++n) {
+                const __int128 d = ld128(sdist + n * T);
+                const bool better = ((open >> n) & 1) && (v < 0 || d < dv);
+                v = better ? n : v; dv = better ? d : dv;
+            }
+            const bool has = v >= 0;
+            const int vv = has ? v : 0;
+            done |= has ? (1u << vv) : 0u;
+            const bool iscol = vv >= M;
+            const bool hit = has && iscol && (int)((load >> (4 * (vv & (M - 1)))) & 15u) < P;
+            target = hit ? vv : target;
+            const bool relax = has && !hit;
+            // relax its M arcs: a column un-prunes one of its pruned entries, a row prunes one more of its kept ones
+            const __int128 base = dv + ld128(spot + vv * T);
+#pragma unroll
+            for (int k = 0; k < M; ++k) {
+                const int nb = iscol ? k : M + k;
+                const int p = iscol ? k * M + (vv - M) : vv * M + k;
+                const bool is_pruned = (pruned >> p) & 1;
+                const bool elig = relax && (is_pruned == iscol) && !((done >> nb) & 1);
+                const __int128 c = edge_cost128(su[p * T], Emin, p);
+                const __int128 nd = base - ld128(spot + nb * T) + (iscol ? -c : c);
+                const bool better = elig && (!((reach >> nb) & 1) || nd < ld128(sdist + nb * T));
+                if (better) st128(sdist + nb * T, nd);
+                pre = better ? ((pre & ~(15ull << (4 * nb))) | ((uint64_t)vv << (4 * nb))) : pre;
+                reach |= (better ? 1u : 0u) << nb;
+            }
+        }
+        const bool ok = active && target >= 0;
+        failed |= active && target < 0;
+        // potentials: settled nodes closer than the target move by their distance, all others by the target's
+        const int tt = ok ? target : M;
+        const __int128 D = ld128(sdist + tt * T);
+#pragma unroll
+        for (int n = 0; n < 2 * M; ++n) {
+            const __int128 d = ld128(sdist + n * T);
+            const __int128 add = (((done >> n) & 1) && d < D) ? d : D;
+            if (ok) st128(spot + n * T, ld128(spot + n * T) + add);
+        }
+        // flip the arcs of the path back to its source column
+        int v = tt;
+        load += ok ? (1u << (4 * (tt - M))) : 0u;
+#pragma unroll 1
+        for (int s = 0; s < 2 * M + 2; ++s) {
+            const bool go = ok && !((sources >> v) & 1);
+            if (!__any_sync(kFull, go)) break;
+            const int w = (int)((pre >> (4 * v)) & 15u);
+            const uint64_t bit = v >= M ? (1ull << ((w & (M - 1)) * M + (v - M))) : (1ull << (v * M + (w & (M - 1))));
+            pruned = go ? (v >= M ? (pruned | bit) : (pruned & ~bit)) : pruned;     // row w -> column v-M prunes; column w-M -> row v un-prunes
+            v = go ? w : v;
+        }
+        const bool home = ok && ((sources >> v) & 1);
+        load -= home ? (1u << (4 * (v - M))) : 0u;
+        failed |= ok && !home;
+    }
+    if (failed) status |= kDevInternal;
+    const uint64_t all = (M == 8) ? ~0ull : ((1ull << (M * M)) - 1);
+    return ~pruned & all;
+}
+
+// Called by all 32 lanes of a warp.
+template <int N, int M>
+__device__ __forceinline__ uint64_t exact_ssp(const uint32_t (&u)[M * M], int& status, uint32_t* su, uint4* spot, uint4* sdist, int T) {
     int Emin, Emax;
     if (!exponent_range<M * M>(u, Emin, Emax)) { Emin = 1; Emax = 1; }
     // 128-bit costs: 64 tie bits + 24 significand bits + spread; paths (<= 2M arcs) and potentials (<= M(M-N)
-    // updates) add 4 + 5 bits, the sign one more
-    if (Emax - Emin <= 26) return exact_flow_run<Cost128, N, M>(u, Emin, status);
-    return exact_flow_run<CostWide, N, M>(u, Emin, status);
+    // updates) add 4 + 5 bits, the sign one more; beyond that the block takes the wide integers, on its own
+    const bool wide = Emax - Emin > 26;
+    uint64_t kept = exact_flow_warp<N, M>(u, Emin, !wide, status, su, spot, sdist, T);
+    if (wide) kept = exact_flow_run<CostWide, N, M>(u, Emin, status);
+    return kept;
 }
 
 }  // namespace tmask
