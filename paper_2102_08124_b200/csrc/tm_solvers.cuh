@@ -320,11 +320,58 @@ __device__ __forceinline__ uint64_t exact_2_4_classes(const uint32_t (&u)[16], i
     return best & 0xFFFFull;
 }
 
-// drop_bits: low significand bits known to be zero in every entry (16 for widened bf16 inputs)
+// The same 19 classes in 32-bit arithmetic, for blocks whose sums leave room: value(row i, pair) =
+// (q_a + q_b) * 2^12 + (pair index << 3i).  The pair index (0..5) grows with the row's nibble, so the twelve
+// low bits order the patterns exactly as the 16-bit mask code does.  Needs 8-bit significands (bf16) and an
+// exponent spread of at most 9: 8 + 9 + 3 bits of sum above 12 bits of code.
+template <int C, int D>
+__device__ __forceinline__ uint32_t shared_column_case32(const uint32_t (&v)[4][6]) {
+    constexpr int a = other_column(C, D, 0), b = other_column(C, D, 1);
+    constexpr int ca = pair_index(C, a), cb = pair_index(C, b), da = pair_index(D, a), db = pair_index(D, b);
+    return max(v[0][ca] + v[1][cb], v[0][cb] + v[1][ca]) + max(v[2][da] + v[3][db], v[2][db] + v[3][da]);
+}
+__device__ __forceinline__ uint64_t exact_2_4_classes32(const uint32_t (&u)[16], int Emin) {
+    uint32_t v[4][6];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint32_t q[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t sig; int E; split_float(u[i * 4 + j], sig, E);
+            q[j] = sig ? ((sig >> 16) << (E - Emin + 12)) : 0u;
+        }
+#pragma unroll
+        for (int b = 1; b < 4; ++b)
+#pragma unroll
+            for (int a = 0; a < b; ++a)
+                v[i][pair_index(a, b)] = q[a] + q[b] + ((uint32_t)pair_index(a, b) << (3 * i));
+    }
+    uint32_t best = 0, up_c = 0, lo_c = 0;
+#pragma unroll
+    for (int k = 0; k < 6; ++k) {
+        best = max(best, v[0][k] + v[1][k] + v[2][5 - k] + v[3][5 - k]);
+        up_c = max(up_c, v[0][k] + v[1][5 - k]);
+        lo_c = max(lo_c, v[2][k] + v[3][5 - k]);
+    }
+    best = max(best, up_c + lo_c);
+    best = max(best, max(max(shared_column_case32<0, 1>(v), shared_column_case32<0, 2>(v)), shared_column_case32<0, 3>(v)));
+    best = max(best, max(max(shared_column_case32<1, 0>(v), shared_column_case32<1, 2>(v)), shared_column_case32<1, 3>(v)));
+    best = max(best, max(max(shared_column_case32<2, 0>(v), shared_column_case32<2, 1>(v)), shared_column_case32<2, 3>(v)));
+    best = max(best, max(max(shared_column_case32<3, 0>(v), shared_column_case32<3, 1>(v)), shared_column_case32<3, 2>(v)));
+    // pair indices back to nibbles: 0x3, 0x5, 0x6, 0x9, 0xA, 0xC
+    uint32_t code = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) code |= ((0xCA9653u >> (4 * ((best >> (3 * i)) & 7u))) & 0xFu) << (4 * i);
+    return code;
+}
+
+// drop_bits: low significand bits known to be zero in every entry (16 for widened bf16 inputs).
+// Called by all 32 lanes of a warp (the 32-bit scorer is taken when every lane's block fits it).
 __device__ __forceinline__ uint64_t exact_2_4(const uint32_t (&u)[16], int drop_bits) {
     int Emin, Emax;
     if (!exponent_range<16>(u, Emin, Emax)) { Emin = 1; Emax = 1; }     // all zero: every sum is 0, the largest code wins
     const int spread = Emax - Emin;
+    if (__all_sync(0xFFFFFFFFu, drop_bits == 16 && spread <= 9)) return exact_2_4_classes32(u, Emin);
     // (24 - drop) significand bits + spread + 3 bits for eight terms + 16 code bits must stay below 2^63
     if (spread <= 19 + drop_bits) return exact_2_4_classes(u, Emin, drop_bits);
     if (spread <= 34) return exact_2_4_int64(u, Emin);

@@ -114,6 +114,19 @@ def test_bf16_subnormals_and_extremes_compare_exactly(N, M):
         assert_parity(V, N, M, method, rel=None)                        # fp32 partial sums may overflow here
 
 
+def test_exact_2_4_bf16_narrow_blocks_take_the_32_bit_scorer():
+    """Quantised bf16 (every block spans few binades, ties everywhere): the 32-bit scorer must give the optimum and
+    break ties by the mask code exactly as the 64-bit one; a second matrix mixes in blocks it cannot take."""
+    W = workloads.quantised_bf16(64, 1024, 0.02, 41)
+    assert_parity(W, 2, 4, tm.TM_EXACT)
+    Z = W.copy()
+    Z[:, :] = Z[:, :] & np.uint16(0x8003) | np.uint16(0x3C00)          # four magnitudes only: ties in every block
+    assert_parity(Z, 2, 4, tm.TM_EXACT)
+    V = W.copy()
+    V[5, 100] = 0x0001; V[40, 777] = 0x7F00; V[41, 20] = 0x0080         # blocks with a wide exponent spread
+    assert_parity(V, 2, 4, tm.TM_EXACT)
+
+
 @pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
 def test_optional_outputs_and_in_place(N, M):
     W = workloads.normal_f32(4 * M, 45 * M, 0.02, 13)
