@@ -22,9 +22,9 @@
 // Step C (one 2-for-1 swap) is needed by roughly one block in six.  After step B such a block has
 // exactly one short row r and one short column c, each holding the single entry (r,c); the swap
 // removes the lightest kept entry x = (r',c') outside row r (none of them lies in column c) and adds
-// (r,c') and (r',c).  x is lighter than the other kept entry of its row and of its column, so it is
-// one of the at most three "local minima" that swap_candidates() marks from the relation masks;
-// only those few need their magnitudes compared.
+// (r,c') and (r',c).  Only the flagged blocks do this, each on a lane of its own, comparing the six
+// magnitudes directly (marking the local minima from the relation masks first would spare three of the
+// comparisons but cost every lane of every item a dozen instructions).
 #pragma once
 #include <cstdint>
 
@@ -127,41 +127,40 @@ TM_HD uint32_t short_blocks(const LineFill& f) {
     return ((f.row_full & 0xFFFFu) != 0xFFFFu ? 1u : 0u) | ((f.row_full >> 16) != 0xFFFFu ? 2u : 0u);
 }
 
-// Step C, first half (bit-parallel, meaningful for blocks flagged by short_blocks): the kept entries
-// outside the short row that are lighter than the other kept entry of their row and of their column.
-TM_HD uint32_t swap_candidates(const Rel24& r, const LineFill& f, uint32_t kept) {
-    const uint32_t e = kept & f.row_full;           // rows other than the short one
-    uint32_t ra, r2, ca, c2;
-    heavier_in_row(r, e, ra, r2);
-    heavier_in_col(r, e, ca, c2);
-    return e & ra & ca;
+// index of the lowest set bit (x != 0)
+TM_HD int lowest_bit(uint32_t x) {
+#if defined(__CUDA_ARCH__)
+    return __ffs((int)x) - 1;
+#else
+    int p = 0;
+    while (!((x >> p) & 1)) ++p;
+    return p;
+#endif
 }
 
-// Step C, second half, for one block: `cands16` = swap_candidates of the block (1..3 entries), key(p)
-// returns the magnitude pattern of entry p.  Returns false (mask unchanged) on an unexpected shape.
+// Step C for one block flagged by short_blocks(): key(p) returns the magnitude pattern of entry p.  The
+// entry to give way is the lightest of the six kept entries outside the short row (the earliest of equal
+// magnitudes).  Returns false (mask unchanged) on an unexpected shape.
 template <class KeyFn>
-TM_HD bool swap_apply_2_4(uint32_t& kept16, uint32_t cands16, KeyFn key) {
+TM_HD bool swap_apply_2_4(uint32_t& kept16, KeyFn key) {
     // the short row / column: the only ones not holding two entries
     const uint32_t a = kept16, t = a | (a >> 1) | (a >> 2);
-    const uint32_t rfull = (maj3(a, a >> 1, a >> 2) | ((a >> 3) & t)) & 0x1111u;
+    const uint32_t rshort = ((maj3(a, a >> 1, a >> 2) | ((a >> 3) & t)) & 0x1111u) ^ 0x1111u;
     const uint32_t u = a | (a >> 4) | (a >> 8);
-    const uint32_t cfull = (maj3(a, a >> 4, a >> 8) | ((a >> 12) & u)) & 0x000Fu;
-    const uint32_t rshort = rfull ^ 0x1111u, cshort = cfull ^ 0xFu;
-    if (!rshort || (rshort & (rshort - 1)) || !cshort || (cshort & (cshort - 1)) || !cands16) return false;
+    const uint32_t cshort = ((maj3(a, a >> 4, a >> 8) | ((a >> 12) & u)) & 0xFu) ^ 0xFu;
+    if (!rshort || (rshort & (rshort - 1)) || !cshort || (cshort & (cshort - 1))) return false;
+    const int r4 = lowest_bit(rshort), c = lowest_bit(cshort);     // r4 = 4 * short row
+    if (!((kept16 >> (r4 + c)) & 1)) return false;
+    uint32_t cands = kept16 & ~(0xFu << r4);
     int x = -1; uint32_t best = 0;
-    for (int n = 0; n < 3 && cands16; ++n) {                    // ascending positions: the earliest of equals wins
-        int p = 0;
-        { uint32_t low = cands16 & (0u - cands16); while (!((low >> p) & 1)) ++p; }
-        cands16 &= cands16 - 1;
+    for (int n = 0; n < 6 && cands; ++n) {                          // ascending positions: the earliest of equals wins
+        const int p = lowest_bit(cands);
+        cands &= cands - 1;
         const uint32_t kp = key(p);
         if (x < 0 || kp < best) { x = p; best = kp; }
     }
-    if (cands16) return false;
-    int r = 0, c = 0;
-    while (!((rshort >> (4 * r)) & 1)) ++r;
-    while (!((cshort >> c) & 1)) ++c;
-    if (!((kept16 >> (4 * r + c)) & 1)) return false;
-    kept16 = (kept16 & ~(1u << x)) | (1u << (4 * r + (x & 3))) | (1u << ((x & ~3) + c));
+    if (cands || x < 0) return false;
+    kept16 = (kept16 & ~(1u << x)) | (1u << (r4 + (x & 3))) | (1u << ((x & ~3) + c));
     return true;
 }
 

@@ -9,7 +9,7 @@
 //      warp-uniform (a vote decides whether any lane still has candidates); the two block rows give
 //      the scheduler two independent instruction streams;
 //   3. the blocks that need step C (about one in six) are queued in shared memory and fixed by as
-//      many lanes at once as there are queued blocks, each reading the few magnitudes it must compare
+//      many lanes at once as there are queued blocks, each reading the six magnitudes it must compare
 //      straight from the stage;
 //   4. the lanes write the masked weights back into the stage, lane 0 sends it out with one TMA store,
 //      mask bytes meet in shared memory and leave as whole 32-bit words.
@@ -47,8 +47,8 @@ template <int DT, int METHOD> struct Geometry {
     // out as one longer run instead of 32-byte pieces.  Measured: it helps where the kernel waits for memory
     // (Algorithm 1 alone) and costs more than it gives where it waits for the integer pipe (full search).
     static constexpr int kMaskItems = DT == kF32 ? 4 : (METHOD == kMethodApprox ? 1 : 2);
-    // stages | mask bytes [items][8][32] | kept [2][32] | swap candidates [2][32] | queue [128] | barriers
-    static constexpr int kWarpBytes = kStages * kStageBytes + kMaskItems * 256 + 2 * 256 + 128 + 128;
+    // stages | mask bytes [items][8][32] | kept [2][32] | queue [128] | barriers
+    static constexpr int kWarpBytes = kStages * kStageBytes + kMaskItems * 256 + 256 + 128 + 128;
     static constexpr int kSmemBytes = kWarps * kWarpBytes + (DT == kBF16 ? kLaneLutBytes : 0);
     static_assert(kSmemBytes <= 232448, "at most 227 KB of shared memory per CTA");
     static_assert(kWarpBytes % 128 == 0, "stages stay 128-byte aligned");
@@ -109,30 +109,13 @@ __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, 
     }
 }
 
-// Step C, second half, on a block whose magnitudes sit in shared memory (natural layout).
+// Step C on a block whose magnitudes sit in shared memory (natural layout).
 template <int DT>
-__device__ __forceinline__ bool swap_apply_smem(const unsigned char* blk, uint32_t& kept16, uint32_t cands16) {
-    const uint32_t a = kept16, t = a | (a >> 1) | (a >> 2);
-    const uint32_t rshort = ((maj3(a, a >> 1, a >> 2) | ((a >> 3) & t)) & 0x1111u) ^ 0x1111u;
-    const uint32_t u = a | (a >> 4) | (a >> 8);
-    const uint32_t cshort = ((maj3(a, a >> 4, a >> 8) | ((a >> 12) & u)) & 0xFu) ^ 0xFu;
-    if (__popc(rshort) != 1 || __popc(cshort) != 1 || cands16 == 0 || __popc(cands16) > 3) return false;
-    int x = -1; uint32_t best = 0;
-#pragma unroll
-    for (int n = 0; n < 3; ++n) {                                   // ascending positions: the earliest of equals wins
-        if (cands16) {
-            const int p = __ffs(cands16) - 1;
-            cands16 &= cands16 - 1;
-            uint32_t kp;
-            if constexpr (DT == kBF16) kp = *reinterpret_cast<const unsigned short*>(blk + (p >> 2) * 512 + (p & 3) * 2) & 0x7FFFu;
-            else kp = *reinterpret_cast<const uint32_t*>(blk + (p >> 2) * 1024 + (p & 3) * 4) & 0x7FFFFFFFu;
-            if (x < 0 || kp < best) { x = p; best = kp; }
-        }
-    }
-    const int r4 = __ffs(rshort) - 1, c = __ffs(cshort) - 1;        // r4 = 4 * short row
-    if (!((kept16 >> (r4 + c)) & 1)) return false;
-    kept16 = (kept16 & ~(1u << x)) | (1u << (r4 + (x & 3))) | (1u << ((x & ~3) + c));
-    return true;
+__device__ __forceinline__ bool swap_apply_smem(const unsigned char* blk, uint32_t& kept16) {
+    return swap_apply_2_4(kept16, [blk](int p) -> uint32_t {
+        if constexpr (DT == kBF16) return *reinterpret_cast<const unsigned short*>(blk + (p >> 2) * 512 + (p & 3) * 2) & 0x7FFFu;
+        else return *reinterpret_cast<const uint32_t*>(blk + (p >> 2) * 1024 + (p & 3) * 4) & 0x7FFFFFFFu;
+    });
 }
 
 // Masked weights back into the stage, mask bytes, objective contribution of the lane's two blocks.
@@ -188,8 +171,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     unsigned char* stages = smem_raw + (size_t)warp * G::kWarpBytes;
     unsigned char* mbytes = stages + G::kStages * G::kStageBytes;
     uint32_t* kbuf = reinterpret_cast<uint32_t*>(mbytes + G::kMaskItems * 256);
-    uint32_t* cbuf = kbuf + kHalves * 32;
-    unsigned char* queue = reinterpret_cast<unsigned char*>(cbuf + kHalves * 32);
+    unsigned char* queue = reinterpret_cast<unsigned char*>(kbuf + kHalves * 32);
     uint64_t* bars = reinterpret_cast<uint64_t*>(queue + 128);
     uint4* lut = reinterpret_cast<uint4*>(smem_raw + (size_t)G::kWarps * G::kWarpBytes);
     if constexpr (DT == kBF16) {           // the only CTA-wide step: the lane-mask table
@@ -254,7 +236,6 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                 }
                 const uint32_t sb = short_blocks(f);
                 if (__any_sync(0xFFFFFFFFu, sb != 0)) {
-                    cbuf[h * 32 + lane] = swap_candidates(rel, f, k);
 #pragma unroll
                     for (int b = 0; b < 2; ++b) {
                         const bool need = (sb >> b) & 1;
@@ -279,9 +260,8 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                     const int h = e >> 6, b = (e >> 5) & 1, ln = e & 31;
                     unsigned short* kh = reinterpret_cast<unsigned short*>(kbuf + h * 32 + ln) + b;
                     uint32_t k16 = *kh;
-                    const uint32_t c16 = reinterpret_cast<const unsigned short*>(cbuf + h * 32 + ln)[b];
                     const unsigned char* blk = stage + h * G::kHalfBytes + ln * (8 * G::kElem) + b * (4 * G::kElem);
-                    if (!swap_apply_smem<DT>(blk, k16, c16)) status |= kDevInternal;
+                    if (!swap_apply_smem<DT>(blk, k16)) status |= kDevInternal;
                     *kh = (unsigned short)k16;
                 }
             }
