@@ -299,6 +299,12 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
 
 int aux_partial_slots() { return 8192; }
 
+cudaError_t launch_aux_reduce(const double* obj_partials, const unsigned long long* viol_partials, int n, double* objective_out,
+                              unsigned long long* violations_out, cudaStream_t stream) {
+    aux_reduce_kernel<<<1, 256, 0, stream>>>(obj_partials, viol_partials, n, objective_out, violations_out);
+    return cudaGetLastError();
+}
+
 static int aux_grid(long long items, int sms) {
     const long long want = (items + kAuxWarps - 1) / kAuxWarps;
     const long long cap = (long long)sms * 8 < 1024 ? (long long)sms * 8 : 1024;

@@ -63,8 +63,9 @@ __device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
     return r;
 }
 
-template <int DT>
-__device__ __forceinline__ void front_end(const unsigned char* stage, int lane, Rel24& rel, uint32_t& worst) {
+// NZ: also return the pair mask of the non-zero entries (for the pattern-violation count)
+template <int DT, bool NZ>
+__device__ __forceinline__ void front_end(const unsigned char* stage, int lane, Rel24& rel, uint32_t& worst, uint32_t& nonzero) {
     if constexpr (DT == kBF16) {
         uint4 v[4];
 #pragma unroll
@@ -80,6 +81,15 @@ __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, 
             relations_bf16<false>(pk, rel);
         }
         else relations_bf16<true>(pk, rel);
+        if constexpr (NZ) {                    // x + 0x7FFF sets the top bit of a 15-bit magnitude iff x != 0 (a NaN kept its sign: still set)
+            uint32_t p[8];
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+                const int i = (7 - b) >> 2, j = (7 - b) & 3;
+                p[b] = pick((pk.x[i][j] & 0x7FFF7FFFu) + 0x7FFF7FFFu, (pk.x[i + 2][j] & 0x7FFF7FFFu) + 0x7FFF7FFFu);
+            }
+            nonzero = gather8<0u>(p);
+        }
     } else {
         uint32_t ka[16], kb[16];
 #pragma unroll
@@ -106,6 +116,11 @@ __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, 
             }
         }
         complete_relations(rel);
+        if constexpr (NZ) {
+            nonzero = 0;
+#pragma unroll
+            for (int p = 0; p < 16; ++p) nonzero |= (ka[p] ? 1u : 0u) << p | (kb[p] ? 1u : 0u) << (16 + p);
+        }
     }
 }
 
@@ -164,7 +179,7 @@ __device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* m
 template <int DT, int METHOD, bool HAS_OUT>
 __global__ void __launch_bounds__(Geometry<DT, METHOD>::kWarps * 32, 1)
 tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict__ table, int count, long long total_items,
-             double* __restrict__ partials, int* __restrict__ status_out) {
+             double* __restrict__ partials, int* __restrict__ status_out, int n_keep, unsigned long long* __restrict__ vpartials) {
     using G = Geometry<DT, METHOD>;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -211,6 +226,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     const uint32_t lt = (1u << lane) - 1u;
     bool alive = true;
     int mfirst = -1;                                                     // first slot of the mask-byte buffer in use
+    unsigned long long viol = 0;                                         // kMethodRows: non-zero entries pruned by this lane
 
     for (int it = 0; it < n_items && alive; ++it) {
         const int s = it % G::kStages;
@@ -222,8 +238,18 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
 #pragma unroll
         for (int h = 0; h < kHalves; ++h) {
             Rel24 rel;
-            front_end<DT>(stage + h * G::kHalfBytes, lane, rel, worst);
-            uint32_t k = cover_2_4(rel);
+            uint32_t nonzero = 0;
+            front_end<DT, METHOD == kMethodRows>(stage + h * G::kHalfBytes, lane, rel, worst, nonzero);
+            uint32_t k;
+            if constexpr (METHOD == kMethodRows) {
+                // N of 4 along rows: kept iff fewer than N entries of the row are heavier
+                k = n_keep == 2 ? ~maj3(rel.hr1, rel.hr2, rel.hr3) : (n_keep == 1 ? ~(rel.hr1 | rel.hr2 | rel.hr3) : ~(rel.hr1 & rel.hr2 & rel.hr3));
+                const int c0 = cur.cj * kItemCols + lane * 8, nc = (int)tab[cur.k].p.cols;
+                const uint32_t inside = c0 >= nc ? 0u : (c0 + 4 >= nc ? 0xFFFFu : 0xFFFFFFFFu);
+                viol += (unsigned)__popc(~k & nonzero & inside);
+            } else {
+                k = cover_2_4(rel);
+            }
             if constexpr (METHOD == kMethodApprox) {
                 LineFill f = line_fill(k);
                 uint32_t cand = open_candidates(k, f);
@@ -323,6 +349,10 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     else { if (nonfinite_bf16x2(worst)) status |= kDevNonFinite; }
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(0xFFFFFFFFu, status, o);
     if (lane == 0 && status && status_out) atomicOr(status_out, status);
+    if constexpr (METHOD == kMethodRows) {
+        for (int o = 16; o; o >>= 1) viol += __shfl_xor_sync(0xFFFFFFFFu, viol, o);
+        if (lane == 0 && vpartials) vpartials[gw] = viol;
+    }
 }
 
 // objective[k] = sum of the problem's partials in a fixed order (one CTA per problem)
@@ -352,7 +382,7 @@ cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntr
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status);
+    kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status, a.n_keep, a.vpartials);
     return cudaGetLastError();
 }
 
@@ -361,12 +391,13 @@ cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntr
 size_t tma_entry_bytes() { return sizeof(TmaEntry); }
 int tma_warps_per_cta(int dtype, int M, int method) {
     if (M == 8) return tma48_warps_per_cta(dtype);
-    if (dtype == kF32) return method == kMethodApprox ? Geometry<kF32, kMethodApprox>::kWarps : Geometry<kF32, kMethodCover>::kWarps;
-    return method == kMethodApprox ? Geometry<kBF16, kMethodApprox>::kWarps : Geometry<kBF16, kMethodCover>::kWarps;
+    if (dtype == kF32) return method == kMethodApprox ? Geometry<kF32, kMethodApprox>::kWarps : (method == kMethodRows ? Geometry<kF32, kMethodRows>::kWarps : Geometry<kF32, kMethodCover>::kWarps);
+    return method == kMethodApprox ? Geometry<kBF16, kMethodApprox>::kWarps : (method == kMethodRows ? Geometry<kBF16, kMethodRows>::kWarps : Geometry<kBF16, kMethodCover>::kWarps);
 }
 
 bool tma_eligible(const DevProblem& p, int N, int M, int method) {
-    if (!((N == 2 && M == 4) || (N == 4 && M == 8)) || (method != kMethodApprox && method != kMethodCover)) return false;
+    if (method == kMethodRows) { if (M != 4 || N < 1 || N > 3) return false; }
+    else if (!((N == 2 && M == 4) || (N == 4 && M == 8)) || (method != kMethodApprox && method != kMethodCover)) return false;
     const size_t elem = p.dtype == kF32 ? 4 : 2;
     if ((uintptr_t)p.W % 16 || ((size_t)p.ld * elem) % 16) return false;
     if (p.masked && (uintptr_t)p.masked % 16) return false;
@@ -398,11 +429,12 @@ cudaError_t launch_tma(const TmaLaunch& a) {
     if (a.total_items > 0) {
 #define TM_DISPATCH(DT, METHOD)                                                                                   \
     err = a.has_out ? launch_one<DT, METHOD, true>(a, host[0], table) : launch_one<DT, METHOD, false>(a, host[0], table)
-        if (a.dtype == kF32) { if (a.method == kMethodApprox) TM_DISPATCH(kF32, kMethodApprox); else TM_DISPATCH(kF32, kMethodCover); }
-        else { if (a.method == kMethodApprox) TM_DISPATCH(kBF16, kMethodApprox); else TM_DISPATCH(kBF16, kMethodCover); }
+        if (a.dtype == kF32) { if (a.method == kMethodApprox) TM_DISPATCH(kF32, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kF32, kMethodRows); else TM_DISPATCH(kF32, kMethodCover); }
+        else { if (a.method == kMethodApprox) TM_DISPATCH(kBF16, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kBF16, kMethodRows); else TM_DISPATCH(kBF16, kMethodCover); }
 #undef TM_DISPATCH
         if (err != cudaSuccess) return err;
     }
+    if (a.method == kMethodRows) return cudaSuccess;       // the caller sums objective and violation partials together
     reduce_tma_kernel<<<a.count, 256, 0, a.stream>>>(host[0], table, a.partials, (long long)a.ctas * wpc);
     return cudaGetLastError();
 }

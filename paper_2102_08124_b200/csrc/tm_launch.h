@@ -32,6 +32,8 @@ struct TmaLaunch {
     int ctas;
     int dtype, method, M;
     bool has_out;               // masked_w_out present (all problems of one launch agree)
+    int n_keep = 2;             // kMethodRows only: entries kept per group of four (1..3)
+    unsigned long long* vpartials = nullptr;   // kMethodRows only (count == 1): ctas * warps pattern-violation partials; the caller reduces
     cudaStream_t stream;
 };
 size_t tma_entry_bytes();
@@ -47,6 +49,8 @@ cudaError_t launch_tma(const TmaLaunch& a);
 
 // Neighbouring operations (tm_kernels_aux.cu)
 int aux_partial_slots();
+cudaError_t launch_aux_reduce(const double* obj_partials, const unsigned long long* viol_partials, int n, double* objective_out,
+                              unsigned long long* violations_out, cudaStream_t stream);
 cudaError_t launch_nm1d(const AuxProblem& P, int N, int M, int flags, bool violations_only, double* obj_partials,
                         unsigned long long* viol_partials, double* objective_out, unsigned long long* violations_out,
                         int* status, int sms, cudaStream_t stream);
