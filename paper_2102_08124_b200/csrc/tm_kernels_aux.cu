@@ -185,6 +185,58 @@ aux_reduce_kernel(const double* __restrict__ obj_partials, const unsigned long l
     if (threadIdx.x == 0) { if (objective_out) *objective_out = so[0]; if (violations_out) *violations_out = sv[0]; }
 }
 
+// Pattern violations of a given mask, streaming form for aligned matrices (16-byte aligned rows, cols % 8 == 0):
+// a lane takes eight consecutive weights (one mask byte) at a time, four such units in flight; the non-zero
+// test is two weights per operation for bf16.  Work item = 1024 consecutive weights of one row.
+template <int DT>
+__global__ void __launch_bounds__(kAuxWarps * 32)
+violations_stream_kernel(const AuxProblem P, unsigned long long* __restrict__ viol_partials) {
+    const int lane = threadIdx.x & 31;
+    const long long gw = (long long)blockIdx.x * kAuxWarps + (threadIdx.x >> 5), nwarps = (long long)gridDim.x * kAuxWarps;
+    const long long units = P.cols / kUnit, chunks = (units + 127) / 128, total = P.rows * chunks;
+    const long long per = (total + nwarps - 1) / nwarps, begin = gw * per, end = min(total, begin + per);
+    const unsigned char* mbytes = reinterpret_cast<const unsigned char*>(P.mask);
+    unsigned long long viol = 0;
+    long long r = begin < end ? begin / chunks : 0, chunk = begin < end ? begin - r * chunks : 0;
+    for (long long item = begin; item < end; ++item) {
+        constexpr int kWords = DT == kF32 ? 8 : 4;
+        uint32_t w[4][kWords], given[4];
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {                         // all loads of the item first
+            const long long unit = (chunk * 4 + s) * 32 + lane;
+            const bool in = unit < units;
+            given[s] = in ? (uint32_t)__ldg(mbytes + r * P.wpr * 4 + unit) : 0xFFu;
+            if constexpr (DT == kF32) {
+                const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(P.W) + r * P.ld + unit * kUnit);
+                const uint4 a = in ? __ldg(p) : make_uint4(0, 0, 0, 0), b = in ? __ldg(p + 1) : make_uint4(0, 0, 0, 0);
+                w[s][0] = a.x; w[s][1] = a.y; w[s][2] = a.z; w[s][3] = a.w; w[s][4] = b.x; w[s][5] = b.y; w[s][6] = b.z; w[s][7] = b.w;
+            } else {
+                const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(P.W) + r * P.ld + unit * kUnit);
+                const uint4 a = in ? __ldg(p) : make_uint4(0, 0, 0, 0);
+                w[s][0] = a.x; w[s][1] = a.y; w[s][2] = a.z; w[s][3] = a.w;
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+            uint32_t nz = 0;
+            if constexpr (DT == kF32) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) nz |= ((w[s][j] & 0x7FFFFFFFu) ? 1u : 0u) << j;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {                 // 15-bit magnitude + 0x7FFF has its top bit set iff the magnitude is not zero
+                    const uint32_t t = ((w[s][j] & 0x7FFF7FFFu) + 0x7FFF7FFFu) >> 15;
+                    nz |= ((t & 1u) | ((t >> 15) & 2u)) << (2 * j);
+                }
+            }
+            viol += (unsigned)__popc(nz & ~given[s]);
+        }
+        if (++chunk == chunks) { chunk = 0; ++r; }
+    }
+    for (int o = 16; o; o >>= 1) viol += __shfl_xor_sync(0xFFFFFFFFu, viol, o);
+    if (lane == 0) viol_partials[gw] = viol;
+}
+
 // number of differing bits of two packed masks (how much a refresh changed the mask)
 __global__ void __launch_bounds__(kAuxWarps * 32)
 hamming_kernel(const uint32_t* __restrict__ a, const uint32_t* __restrict__ b, long long words, unsigned long long* __restrict__ partials) {
@@ -317,6 +369,16 @@ cudaError_t launch_nm1d(const AuxProblem& P, int N, int M, int flags, bool viola
     const long long units = (P.cols + kUnit - 1) / kUnit, items = P.rows * ((units + 32 * kSub - 1) / (32 * kSub));
     const int grid = aux_grid(items, sms);
 #define TM_NM1D(DT, MM, MODE) nm1d_kernel<DT, MM, MODE><<<grid, kAuxWarps * 32, 0, stream>>>(P, N, flags, obj_partials, viol_partials, status)
+    const size_t elem = P.dtype == kF32 ? 4 : 2;
+    const bool streamable = violations_only && P.cols % kUnit == 0 && (uintptr_t)P.W % 16 == 0 && ((size_t)P.ld * elem) % 16 == 0;
+    if (streamable) {
+        if (P.dtype == kF32) violations_stream_kernel<kF32><<<grid, kAuxWarps * 32, 0, stream>>>(P, viol_partials);
+        else violations_stream_kernel<kBF16><<<grid, kAuxWarps * 32, 0, stream>>>(P, viol_partials);
+        cudaError_t es = cudaGetLastError();
+        if (es != cudaSuccess) return es;
+        hamming_reduce_kernel<<<1, 256, 0, stream>>>(viol_partials, grid * kAuxWarps, violations_out);
+        return cudaGetLastError();
+    }
     if (violations_only) { if (P.dtype == kF32) TM_NM1D(kF32, 8, 1); else TM_NM1D(kBF16, 8, 1); }
     else if (P.dtype == kF32) { if (M == 2) TM_NM1D(kF32, 2, 0); else if (M == 4) TM_NM1D(kF32, 4, 0); else TM_NM1D(kF32, 8, 0); }
     else { if (M == 2) TM_NM1D(kBF16, 2, 0); else if (M == 4) TM_NM1D(kBF16, 4, 0); else TM_NM1D(kBF16, 8, 0); }
