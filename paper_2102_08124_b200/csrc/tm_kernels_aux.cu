@@ -260,86 +260,109 @@ hamming_reduce_kernel(const unsigned long long* __restrict__ partials, int n, un
 }
 
 // ---- 2:4 compression ---------------------------------------------------------------------------
-// CTA tile: 32 rows x 128 columns = 8 x 32 blocks of 4x4; warp = block row, lane = block column.
+// CTA tile: 128 rows x 128 columns = 32 x 32 blocks of 4x4; a warp takes block rows w, w+8, w+16, w+24 of the
+// tile, lane = block column.  The row form (values, meta) is written straight from registers, 128 bytes per
+// row and warp.  The column form is collected in shared memory so that every column of the tile leaves as one
+// run of 64 values (128 bytes of bf16) written with 16-byte stores, and its four metadata words in one go.
+// Shared tile: the kept pair of (column c, block row br) at word ((c & 3) * 32 + (c >> 2)) * pitch + br * kVW:
+// lanes of a warp (columns four apart) fall into different banks.
 template <int DT>
 __global__ void __launch_bounds__(256)
 compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __restrict__ meta, void* __restrict__ values_t,
                   uint32_t* __restrict__ meta_t, int* __restrict__ status_out) {
-    using elem_t = typename std::conditional<DT == kF32, uint32_t, uint16_t>::type;
-    __shared__ elem_t tile_t[128][16 + 2];              // [column of the tile][value index along rows]
-    __shared__ uint32_t tile_mt[128];                   // transposed metadata word of every column
+    constexpr int kVW = DT == kF32 ? 2 : 1;             // words per kept pair
+    constexpr int kPitch = 32 * kVW + 1;
+    __shared__ uint32_t tile_t[128 * kPitch];
+    __shared__ uint32_t tile_mt[128][4];                // transposed metadata words of every column (32 rows each)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long long tiles_c = (P.cols + 127) / 128, tiles_r = (P.rows + 31) / 32;
+    const long long tiles_c = (P.cols + 127) / 128, tiles_r = (P.rows + 127) / 128;
     const long long wpr_t = (P.rows + 31) / 32, half_c = P.cols / 2, half_r = P.rows / 2;
+    const size_t ebytes = DT == kF32 ? 4 : 2;
+    const bool vec_t = (uintptr_t)values_t % 16 == 0 && ((size_t)half_r * ebytes) % 16 == 0;
     bool bad = false;
     for (long long t = blockIdx.x; t < tiles_r * tiles_c; t += gridDim.x) {
         const long long tr = t / tiles_c, tc = t - tr * tiles_c;
-        const long long r0 = tr * 32 + warp * 4, c0 = tc * 128 + lane * 4;
-        const bool active = r0 < P.rows && c0 < P.cols;
-        if (threadIdx.x < 128) tile_mt[threadIdx.x] = 0;
+        const long long c0 = tc * 128 + lane * 4;
+        for (int k = threadIdx.x; k < 128 * 4; k += 256) (&tile_mt[0][0])[k] = 0;
         __syncthreads();
-        uint32_t v[4][4] = {}, mbits = 0;                // mbits bit 4i+j = mask of (row i, column j)
-        if (active) {
+#pragma unroll 1
+        for (int it = 0; it < 4; ++it) {
+            const int br = it * 8 + warp;                // block row inside the tile
+            const long long r0 = tr * 128 + br * 4;
+            const bool active = r0 < P.rows && c0 < P.cols;
+            uint32_t v[4][4] = {}, mbits = 0;            // mbits bit 4i+j = mask of (row i, column j)
+            if (active) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if constexpr (DT == kF32) {
+                        const uint4 a = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(P.W) + (r0 + i) * P.ld + c0));
+                        v[i][0] = a.x; v[i][1] = a.y; v[i][2] = a.z; v[i][3] = a.w;
+                    } else {
+                        const uint2 a = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(P.W) + (r0 + i) * P.ld + c0));
+                        v[i][0] = a.x & 0xFFFFu; v[i][1] = a.x >> 16; v[i][2] = a.y & 0xFFFFu; v[i][3] = a.y >> 16;
+                    }
+                    mbits |= ((__ldg(P.mask + (r0 + i) * P.wpr + (c0 >> 5)) >> (c0 & 31)) & 0xFu) << (4 * i);
+                }
+            }
+            // row form: two kept values per row, in column order, and their indices
+            uint32_t row_nibbles = 0;                    // nibble i = metadata of row i
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                if constexpr (DT == kF32) {
-                    const uint4 a = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(P.W) + (r0 + i) * P.ld + c0));
-                    v[i][0] = a.x; v[i][1] = a.y; v[i][2] = a.z; v[i][3] = a.w;
-                } else {
-                    const uint2 a = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(P.W) + (r0 + i) * P.ld + c0));
-                    v[i][0] = a.x & 0xFFFFu; v[i][1] = a.x >> 16; v[i][2] = a.y & 0xFFFFu; v[i][3] = a.y >> 16;
+                const uint32_t m = (mbits >> (4 * i)) & 0xFu;
+                uint32_t a = 0, b = 0, nib = 0;
+                if (__popc(m) == 2) {
+                    const int i0 = __ffs(m) - 1, i1 = 31 - __clz(m);
+                    a = i0 == 0 ? v[i][0] : (i0 == 1 ? v[i][1] : v[i][2]);
+                    b = i1 == 1 ? v[i][1] : (i1 == 2 ? v[i][2] : v[i][3]);
+                    nib = (uint32_t)(i0 | (i1 << 2));
+                } else if (active) bad = true;
+                row_nibbles |= nib << (4 * i);
+                if (active) {
+                    if constexpr (DT == kF32) *reinterpret_cast<uint2*>(reinterpret_cast<uint32_t*>(values) + (r0 + i) * half_c + (c0 >> 1)) = make_uint2(a, b);
+                    else *reinterpret_cast<uint32_t*>(reinterpret_cast<uint16_t*>(values) + (r0 + i) * half_c + (c0 >> 1)) = a | (b << 16);
                 }
-                mbits |= ((__ldg(P.mask + (r0 + i) * P.wpr + (c0 >> 5)) >> (c0 & 31)) & 0xFu) << (4 * i);
             }
-        }
-        // row form: two kept values per row, in column order, and their indices
-        uint32_t row_nibbles = 0;                        // nibble i = metadata of row i
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t m = (mbits >> (4 * i)) & 0xFu;
-            uint32_t a = 0, b = 0, nib = 0;
-            if (__popc(m) == 2) {
-                const int i0 = __ffs(m) - 1, i1 = 31 - __clz(m);
-                a = i0 == 0 ? v[i][0] : (i0 == 1 ? v[i][1] : v[i][2]);
-                b = i1 == 1 ? v[i][1] : (i1 == 2 ? v[i][2] : v[i][3]);
-                nib = (uint32_t)(i0 | (i1 << 2));
-            } else if (active) bad = true;
-            row_nibbles |= nib << (4 * i);
-            if (active) {
-                if constexpr (DT == kF32) *reinterpret_cast<uint2*>(reinterpret_cast<uint32_t*>(values) + (r0 + i) * half_c + (c0 >> 1)) = make_uint2(a, b);
-                else *reinterpret_cast<uint32_t*>(reinterpret_cast<uint16_t*>(values) + (r0 + i) * half_c + (c0 >> 1)) = a | (b << 16);
+            for (int i = 0; i < 4; ++i) {                // eight lanes share a metadata word of a row
+                uint32_t w = ((row_nibbles >> (4 * i)) & 0xFu) << (4 * (lane & 7));
+                w |= __shfl_xor_sync(0xFFFFFFFFu, w, 1); w |= __shfl_xor_sync(0xFFFFFFFFu, w, 2); w |= __shfl_xor_sync(0xFFFFFFFFu, w, 4);
+                if ((lane & 7) == 0 && active) meta[(r0 + i) * P.wpr + (c0 >> 5)] = w;
             }
-        }
+            // column form into the shared tile
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {                    // eight lanes share a metadata word of a row
-            uint32_t w = ((row_nibbles >> (4 * i)) & 0xFu) << (4 * (lane & 7));
-            w |= __shfl_xor_sync(0xFFFFFFFFu, w, 1); w |= __shfl_xor_sync(0xFFFFFFFFu, w, 2); w |= __shfl_xor_sync(0xFFFFFFFFu, w, 4);
-            if ((lane & 7) == 0 && active) meta[(r0 + i) * P.wpr + (c0 >> 5)] = w;
-        }
-        // column form through the shared tile: column c of the tile gets its two kept values of this block row
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint32_t m = ((mbits >> j) & 1u) | (((mbits >> (4 + j)) & 1u) << 1) | (((mbits >> (8 + j)) & 1u) << 2) | (((mbits >> (12 + j)) & 1u) << 3);
-            uint32_t a = 0, b = 0, nib = 0;
-            if (__popc(m) == 2) {
-                const int i0 = __ffs(m) - 1, i1 = 31 - __clz(m);
-                a = i0 == 0 ? v[0][j] : (i0 == 1 ? v[1][j] : v[2][j]);
-                b = i1 == 1 ? v[1][j] : (i1 == 2 ? v[2][j] : v[3][j]);
-                nib = (uint32_t)(i0 | (i1 << 2));
-            } else if (active) bad = true;
-            tile_t[lane * 4 + j][warp * 2] = (elem_t)a;
-            tile_t[lane * 4 + j][warp * 2 + 1] = (elem_t)b;
-            if (nib) atomicOr(&tile_mt[lane * 4 + j], nib << (4 * warp));
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t m = ((mbits >> j) & 1u) | (((mbits >> (4 + j)) & 1u) << 1) | (((mbits >> (8 + j)) & 1u) << 2) | (((mbits >> (12 + j)) & 1u) << 3);
+                uint32_t a = 0, b = 0, nib = 0;
+                if (__popc(m) == 2) {
+                    const int i0 = __ffs(m) - 1, i1 = 31 - __clz(m);
+                    a = i0 == 0 ? v[0][j] : (i0 == 1 ? v[1][j] : v[2][j]);
+                    b = i1 == 1 ? v[1][j] : (i1 == 2 ? v[2][j] : v[3][j]);
+                    nib = (uint32_t)(i0 | (i1 << 2));
+                } else if (active) bad = true;
+                uint32_t* slot = tile_t + (j * 32 + lane) * kPitch + br * kVW;
+                if constexpr (DT == kF32) { slot[0] = a; slot[1] = b; } else slot[0] = a | (b << 16);
+                if (nib) atomicOr(&tile_mt[lane * 4 + j][it], nib << (4 * warp));
+            }
         }
         __syncthreads();
-        {   // 128 columns x 16 values: two threads per column, eight values each
+        {   // 128 columns: two threads per column, each half of its 64 values and two of its four metadata words
             const int c = threadIdx.x >> 1, h = threadIdx.x & 1;
-            const long long col = tc * 128 + c, vr0 = tr * 16 + h * 8;      // first value index along the transposed row
+            const long long col = tc * 128 + c;
             if (col < P.cols) {
+                const uint32_t* src = tile_t + ((c & 3) * 32 + (c >> 2)) * kPitch + h * 16 * kVW;
+                const long long v0 = tr * 64 + h * 32;                      // first value index along the transposed row
+                unsigned char* dst = reinterpret_cast<unsigned char*>(values_t) + ((size_t)col * half_r + v0) * ebytes;
+                if (vec_t && v0 + 32 <= half_r) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    if (vr0 + k < half_r) reinterpret_cast<elem_t*>(values_t)[col * half_r + vr0 + k] = tile_t[c][h * 8 + k];
-                if (h == 0) meta_t[col * wpr_t + tr] = tile_mt[c];
+                    for (int q = 0; q < 4 * kVW; ++q)
+                        reinterpret_cast<uint4*>(dst)[q] = make_uint4(src[4 * q], src[4 * q + 1], src[4 * q + 2], src[4 * q + 3]);
+                } else {
+                    for (int k = 0; k < 16 * kVW; ++k)                      // pairs of values (bf16) or single values (fp32), 4 bytes each
+                        if (v0 + (DT == kF32 ? k : 2 * k) < half_r) reinterpret_cast<uint32_t*>(dst)[k] = src[k];
+                }
+#pragma unroll
+                for (int k = 0; k < 2; ++k)
+                    if (tr * 4 + h * 2 + k < wpr_t) meta_t[col * wpr_t + tr * 4 + h * 2 + k] = tile_mt[c][h * 2 + k];
             }
         }
         __syncthreads();
@@ -401,7 +424,7 @@ cudaError_t launch_hamming(const uint32_t* a, const uint32_t* b, long long words
 
 cudaError_t launch_compress24(const AuxProblem& P, void* values, uint32_t* meta, void* values_t, uint32_t* meta_t, int* status,
                               int sms, cudaStream_t stream) {
-    const long long tiles = ((P.rows + 31) / 32) * ((P.cols + 127) / 128);
+    const long long tiles = ((P.rows + 127) / 128) * ((P.cols + 127) / 128);
     if (tiles == 0) return cudaSuccess;
     const int grid = (int)(tiles < (long long)sms * 8 ? tiles : (long long)sms * 8);
     if (P.dtype == kF32) compress24_kernel<kF32><<<grid, 256, 0, stream>>>(P, values, meta, values_t, meta_t, status);

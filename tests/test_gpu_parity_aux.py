@@ -65,7 +65,7 @@ def test_mask_violations(dtype):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_compress_2_4(dtype):
-    for rows, cols, seed in [(4, 4, 21), (36, 132, 22), (64, 512, 23), (100, 260, 24)]:
+    for rows, cols, seed in [(4, 4, 21), (36, 132, 22), (64, 512, 23), (100, 260, 24), (272, 384, 25)]:
         W = _case(dtype, rows, cols, seed) if dtype == "f32" or cols % 8 == 0 or True else None
         Wd = to_device(W)
         fn = tm.tm_find_mask_bf16 if dtype == "bf16" else tm.tm_find_mask
