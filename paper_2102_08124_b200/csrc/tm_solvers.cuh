@@ -1,4 +1,5 @@
-// Per-block solvers of the transposable N:M mask search, one thread per M x M block.
+// Per-block solvers of the transposable N:M mask search, one thread per M x M block (the flow solver: one
+// block per lane, a whole warp in step).
 //
 // Every routine takes the block as M*M magnitudes u[p] (fp32 bit pattern of |w|, p = i*M + j) and
 // returns the kept set as a bit mask (bit p = S_ij of Eq. 1).  The order of entries is (u, p):
@@ -12,7 +13,9 @@
 //   exact_2_4       the optimum of Eq. 1 for M = 4 by scoring all 90 valid patterns.
 //   exact_ssp       the optimum for any M <= 8 by shortest augmenting paths on the flow network of
 //                   Fig. 3 (rows supply M-N units, columns demand M-N, unit-capacity coefficient
-//                   edges; a unit on (i,j) prunes W_ij), started from a row-feasible pseudo-flow.
+//                   edges; a unit on (i,j) prunes W_ij), started from a row-feasible pseudo-flow:
+//                   exact_flow_warp (128-bit costs, warp-uniform) and exact_flow_run (384-bit costs,
+//                   scalar, for blocks spanning more than 26 binades).
 //
 // Exact arithmetic.  |w_p| = sig_p * 2^(E_p - 150); with Emin the smallest exponent among the
 // block's non-zero entries, q_p = sig_p << (E_p - Emin) is an integer proportional to |w_p|.  When
@@ -383,16 +386,6 @@ __device__ __forceinline__ uint64_t exact_2_4(const uint32_t (&u)[16], int drop_
 // ------------------------------------------------------------------------------------------
 // Cost of the coefficient edge of entry p: q_p * 2^64 + 2^p (the tie rule folded into the cost:
 // minimising the pruned cost maximises (sum of kept |w|, code)).
-struct Cost128 { __int128 v; };
-template <> struct CostOps<Cost128> {
-    static __device__ __forceinline__ Cost128 zero() { return Cost128{0}; }
-    static __device__ __forceinline__ Cost128 add(Cost128 a, Cost128 b) { return Cost128{a.v + b.v}; }
-    static __device__ __forceinline__ Cost128 neg(Cost128 a) { return Cost128{-a.v}; }
-    static __device__ __forceinline__ bool less(Cost128 a, Cost128 b) { return a.v < b.v; }
-    static __device__ __forceinline__ Cost128 edge(uint32_t sig, int shift, int p) {
-        return Cost128{((__int128)((long long)sig << shift) << 64) + ((__int128)1 << p)};
-    }
-};
 struct CostWide { Wide v; };
 template <> struct CostOps<CostWide> {
     static __device__ __forceinline__ CostWide zero() { return CostWide{wide_zero()}; }

@@ -39,6 +39,37 @@ def test_nm_1d(dtype, N, M, absorb):
         assert abs(float(obj.item()) - want["objective"]) <= 1e-6 * abs(want["objective"]) + 1e-300
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N", [1, 2, 3])
+def test_nm_1d_groups_of_four_edge_values(dtype, N):
+    """Shapes the bandwidth kernel takes (16-byte aligned rows): zeros of both signs, subnormals, equal magnitudes,
+    an odd number of rows, several column chunks; then Inf and NaN, which must be ordered by bit pattern and flagged."""
+    rows, cols = 13, 776
+    rng = np.random.Generator(np.random.PCG64(50 + N))
+    W = workloads.normal_f32(rows, cols, 0.02, 51)
+    W[rng.random(W.shape) < 0.25] = 0.0
+    W[rng.random(W.shape) < 0.05] = -0.0
+    W[rng.random(W.shape) < 0.05] = np.float32(1e-40)
+    W[:, 100:140] = np.float32(0.5) * np.sign(W[:, 100:140] + 1e-9)
+    if dtype == "bf16":
+        W = workloads.f32_to_bf16_bits(W)
+    for nonfinite in (False, True):
+        if nonfinite:
+            if dtype == "bf16":
+                W[2, 5] = 0x7F80; W[3, 300] = 0xFFC1; W[3, 301] = 0x7FC0; W[12, 775] = 0xFF80
+            else:
+                W[2, 5] = np.inf; W[3, 300] = np.nan; W[3, 301] = -np.nan; W[12, 775] = -np.inf
+        want = orc.nm_mask_1d(W, N, 4)
+        mask, masked, obj, viol, status = tm.tm_nm_mask_1d(to_device(W), N, 4)
+        torch.cuda.synchronize()
+        assert int(status.item()) == (tm.TM_DEV_NONFINITE if nonfinite else 0)
+        assert np.array_equal(to_host_bits(mask), want["mask"])
+        assert np.array_equal(to_host_bits(masked), want["masked"].view(np.uint16 if dtype == "bf16" else np.uint32))
+        assert int(viol.item()) == want["violations"]
+        if not nonfinite:
+            assert abs(float(obj.item()) - want["objective"]) <= 1e-6 * abs(want["objective"]) + 1e-300
+
+
 def test_nm_1d_strided_rows_and_unaligned_pitch():
     base = to_device(_case("bf16", 12, 100, 7))                  # 200-byte pitch: rows are only 8-byte aligned
     W = base[:, :92]                                             # a strided view
