@@ -492,8 +492,8 @@ int tm_nm_mask_1d(const tm_problem* prob_host, int N, int M, int flags, unsigned
     char* base = static_cast<char*>(workspace_dev) + kHeaderBytes;
     double* op = reinterpret_cast<double*>(base);
     unsigned long long* vp = reinterpret_cast<unsigned long long*>(base + sizeof(double) * (size_t)tmask::aux_partial_slots());
-    // groups of four without mean absorption ride the bandwidth kernel of the 2:4 search (row rule instead of steps A-C)
-    if (M == 4 && N >= 1 && N <= 3 && !(flags & TM_NM1D_ABSORB_MEAN) && p.rows > 0 && p.cols > 0) {
+    // groups of four ride the bandwidth kernel of the 2:4 search (row rule instead of steps A-C)
+    if (M == 4 && N >= 1 && N <= 3 && p.rows > 0 && p.cols > 0) {
         const DevProblem dp = to_dev(p, 4, 0);
         if (tmask::tma_eligible(dp, N, 4, tmask::kMethodRows)) {
             alignas(128) unsigned char entry[512];
@@ -502,7 +502,7 @@ int tm_nm_mask_1d(const tm_problem* prob_host, int N, int M, int flags, unsigned
                 tmask::TmaLaunch t;
                 t.entries_host = entry; t.entries_dev = nullptr; t.count = 1; t.total_items = total; t.partials = op; t.status = status_dev;
                 t.dtype = p.dtype; t.method = tmask::kMethodRows; t.M = 4; t.has_out = p.masked_w_out != nullptr;
-                t.stream = static_cast<cudaStream_t>(cuda_stream); t.n_keep = N; t.vpartials = vp;
+                t.stream = static_cast<cudaStream_t>(cuda_stream); t.n_keep = N | ((flags & TM_NM1D_ABSORB_MEAN) ? 0x100 : 0); t.vpartials = vp;
                 const int wpc = tmask::tma_warps_per_cta(t.dtype, 4, t.method);
                 const long long want = (total + wpc - 1) / wpc;
                 const int cap = d->sms < tmask::aux_partial_slots() / wpc ? d->sms : tmask::aux_partial_slots() / wpc;

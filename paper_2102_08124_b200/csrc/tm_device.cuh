@@ -43,4 +43,12 @@ struct AuxProblem {
 // unsigned order of the patterns is the order of |w|, and -0 == +0.
 __device__ __forceinline__ float pattern_as_float(uint32_t u) { return __uint_as_float(u); }
 
+__device__ __forceinline__ float bf16_to_float(uint32_t h) { return __uint_as_float(h << 16); }
+// fp32 -> bf16, round to nearest even; NaN stays NaN
+__device__ __forceinline__ uint32_t float_to_bf16_bits(float f) {
+    const uint32_t u = __float_as_uint(f);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (u >> 16) | 0x40u;
+    return (u + 0x7FFFu + ((u >> 16) & 1u)) >> 16;
+}
+
 }  // namespace tmask

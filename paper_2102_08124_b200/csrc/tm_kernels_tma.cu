@@ -176,6 +176,56 @@ __device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* m
     return s4;
 }
 
+// Back end of the 1-D pruning with mean absorption (Section 5): every kept weight of a group of four receives
+// the mean of the group's pruned weights -- their sum in position order in fp64, divided by their number, added
+// in fp64, rounded once to fp32 and from there (bf16 tensors) to bf16, nearest even.  The row rule keeps exactly
+// n_keep entries of every group, so the divisor is the same for the whole call.  The objective stays the sum of
+// the kept magnitudes before absorption.
+template <int DT>
+__device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned char* mrow /* [4][32] */, int lane, uint32_t kept, int n_keep) {
+    float s4 = 0.f;
+    const uint32_t mb4 = mask_bytes_2_4(kept);
+    const double pruned = (double)(4 - n_keep);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t mb = (mb4 >> (8 * i)) & 0xFFu;
+        uint32_t raw[8];
+        if constexpr (DT == kBF16) {
+            const uint4 r = *reinterpret_cast<const uint4*>(stage + i * 512 + lane * 16);
+            raw[0] = r.x << 16; raw[1] = r.x & 0xFFFF0000u; raw[2] = r.y << 16; raw[3] = r.y & 0xFFFF0000u;
+            raw[4] = r.z << 16; raw[5] = r.z & 0xFFFF0000u; raw[6] = r.w << 16; raw[7] = r.w & 0xFFFF0000u;
+        } else {
+            const uint4 ra = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32);
+            const uint4 rb = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32 + 16);
+            raw[0] = ra.x; raw[1] = ra.y; raw[2] = ra.z; raw[3] = ra.w; raw[4] = rb.x; raw[5] = rb.y; raw[6] = rb.z; raw[7] = rb.w;
+        }
+        uint32_t o[8];
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {                    // block A, block B: one group of four each
+            double psum = 0.0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) psum += ((mb >> (4 * g + j)) & 1u) ? 0.0 : (double)__uint_as_float(raw[4 * g + j]);
+            // a block past the last column (kept = 0 everywhere) is all zeros: its mean is 0 whatever the divisor
+            const double mu = n_keep == 2 ? psum * 0.5 : (n_keep == 3 ? psum : __ddiv_rn(psum, pruned));
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool k = (mb >> (4 * g + j)) & 1u;
+                const float v = (float)((double)__uint_as_float(raw[4 * g + j]) + mu);
+                o[4 * g + j] = k ? (DT == kF32 ? __float_as_uint(v) : float_to_bf16_bits(v)) : 0u;
+                s4 += k ? fabsf(__uint_as_float(raw[4 * g + j])) : 0.f;
+            }
+        }
+        if constexpr (DT == kBF16) {
+            *reinterpret_cast<uint4*>(stage + i * 512 + lane * 16) = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), o[4] | (o[5] << 16), o[6] | (o[7] << 16));
+        } else {
+            *reinterpret_cast<uint4*>(stage + i * 1024 + lane * 32) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(stage + i * 1024 + lane * 32 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
+        }
+        mrow[i * 32 + lane] = (unsigned char)mb;
+    }
+    return s4;
+}
+
 template <int DT, int METHOD, bool HAS_OUT>
 __global__ void __launch_bounds__(Geometry<DT, METHOD>::kWarps * 32, 1)
 tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict__ table, int count, long long total_items,
@@ -243,7 +293,8 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             uint32_t k;
             if constexpr (METHOD == kMethodRows) {
                 // N of 4 along rows: kept iff fewer than N entries of the row are heavier
-                k = n_keep == 2 ? ~maj3(rel.hr1, rel.hr2, rel.hr3) : (n_keep == 1 ? ~(rel.hr1 | rel.hr2 | rel.hr3) : ~(rel.hr1 & rel.hr2 & rel.hr3));
+                const int nk = n_keep & 0xFF;
+                k = nk == 2 ? ~maj3(rel.hr1, rel.hr2, rel.hr3) : (nk == 1 ? ~(rel.hr1 | rel.hr2 | rel.hr3) : ~(rel.hr1 & rel.hr2 & rel.hr3));
                 const int c0 = cur.cj * kItemCols + lane * 8, nc = (int)tab[cur.k].p.cols;
                 const uint32_t inside = c0 >= nc ? 0u : (c0 + 4 >= nc ? 0xFFFFu : 0xFFFFFFFFu);
                 viol += (unsigned)__popc(~k & nonzero & inside);
@@ -309,9 +360,15 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         const uint32_t colmask = col0 >= cols ? 0u : (col0 + 4 >= cols ? 0xFFFFu : 0xFFFFFFFFu);
         const int slot = cur.cj & (G::kMaskItems - 1);
         if (mfirst < 0) mfirst = slot;
+        if (METHOD == kMethodRows && HAS_OUT && (n_keep & 0x100)) {       // mean absorption requested
 #pragma unroll
-        for (int h = 0; h < kHalves; ++h)
-            facc += back_end<DT, HAS_OUT>(stage + h * G::kHalfBytes, mbytes + slot * 256 + h * 128, lut, lane, kbuf[h * 32 + lane] & colmask);
+            for (int h = 0; h < kHalves; ++h)
+                facc += back_end_absorb<DT>(stage + h * G::kHalfBytes, mbytes + slot * 256 + h * 128, lane, kbuf[h * 32 + lane] & colmask, n_keep & 0xFF);
+        } else {
+#pragma unroll
+            for (int h = 0; h < kHalves; ++h)
+                facc += back_end<DT, HAS_OUT>(stage + h * G::kHalfBytes, mbytes + slot * 256 + h * 128, lut, lane, kbuf[h * 32 + lane] & colmask);
+        }
         if constexpr (HAS_OUT) fence_proxy_async_smem();
         __syncwarp();
         if constexpr (HAS_OUT) {
