@@ -1,20 +1,21 @@
 // Bandwidth kernels of the approximate 2:4 search (TM_APPROX / TM_APPROX_COVER, M = 4).
 //
-// Every warp runs its own software pipeline over a contiguous range of work items (8 rows x 256
-// columns of one matrix: two block rows, 128 blocks):
+// Every warp runs its own software pipeline over a contiguous range of work items (4 rows x 512
+// columns of one matrix: one block row, 128 blocks, in two halves of 256 columns):
 //   1. lane 0 keeps the bulk-tensor (TMA) load of the next item in flight into the other of the warp's
 //      two private shared-memory stages;
 //   2. each lane reads its two 4x4 blocks of either block row with 128-bit shared loads and runs steps
 //      A and B of the search bit-parallel in registers (tm_core24.cuh); the rounds of step B are
-//      warp-uniform (a vote decides whether any lane still has candidates); the two block rows give
+//      warp-uniform (a vote decides whether any lane still has candidates); the two halves give
 //      the scheduler two independent instruction streams;
 //   3. the blocks that need step C (about one in six) are queued in shared memory and fixed by as
 //      many lanes at once as there are queued blocks, each reading the six magnitudes it must compare
 //      straight from the stage;
 //   4. the lanes write the masked weights back into the stage, lane 0 sends it out with one TMA store,
 //      mask bytes meet in shared memory and leave as whole 32-bit words.
-// A matrix with an odd number of block rows ends in a half-empty item: the copy zero-fills the missing
-// rows on the way in and clips them on the way out, and their mask words are not written.
+// An item that reaches past the last column (or, for the 1-D pruning, past the last row) is zero-filled by
+// the copy on the way in and clipped on the way out, and its surplus mask words are not written.  Row segments of 1 KB (bf16) or 2 KB (fp32) keep
+// the DRAM pages busier than narrower, taller items of the same size.
 // Apart from one barrier after the lane-mask table is built, no CTA-wide synchronisation exists; every
 // wait is bounded.
 #include "tm_core24.cuh"
@@ -29,9 +30,10 @@ namespace tmask {
 
 namespace {
 
-constexpr int kItemRows = 8;               // two block rows per item
-constexpr int kHalves = 2;
-constexpr int kItemCols = 256;
+constexpr int kItemRows = 4;               // one block row per item
+constexpr int kHalves = 2;                 // processed as two halves of 256 columns: a lane owns two adjacent blocks of either
+constexpr int kItemCols = 512;
+constexpr int kHalfCols = kItemCols / kHalves;
 
 // Warps per CTA (one CTA per SM) and stages per warp.  The search is bound by integer issue and wants many
 // warps: for bf16, 24 warps at 80 registers per thread fill the shared memory with two stages each (a
@@ -41,13 +43,13 @@ template <int DT, int METHOD> struct Geometry {
     static constexpr int kWarps = DT == kF32 ? 12 : 24;
     static constexpr int kStages = 2;
     static constexpr int kRowPitch = kItemCols * kElem;        // bytes between rows inside a stage
-    static constexpr int kHalfBytes = 4 * kRowPitch;           // one block row
+    static constexpr int kHalfBytes = kHalfCols * kElem;       // from the first half of a row to the second
     static constexpr int kStageBytes = kItemRows * kRowPitch;
     // Mask bytes of this many consecutive items are collected before they leave, so that a row's words go
     // out as one longer run instead of 32-byte pieces.  Measured: it helps where the kernel waits for memory
     // (Algorithm 1 alone) and costs more than it gives where it waits for the integer pipe (full search).
     static constexpr int kMaskItems = DT == kF32 ? 4 : (METHOD == kMethodApprox ? 1 : 2);
-    // stages | mask bytes [items][8][32] | kept [2][32] | queue [128] | barriers
+    // stages | mask bytes [items][half][4][32] | kept [2][32] | queue [128] | barriers
     static constexpr int kWarpBytes = kStages * kStageBytes + kMaskItems * 256 + 256 + 128 + 128;
     static constexpr int kSmemBytes = kWarps * kWarpBytes + (DT == kBF16 ? kLaneLutBytes : 0);
     static_assert(kSmemBytes <= 232448, "at most 227 KB of shared memory per CTA");
@@ -66,10 +68,11 @@ __device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
 // NZ: also return the pair mask of the non-zero entries (for the pattern-violation count)
 template <int DT, bool NZ>
 __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, Rel24& rel, uint32_t& worst, uint32_t& nonzero) {
+    constexpr int kPitch = kItemCols * (DT == kF32 ? 4 : 2);
     if constexpr (DT == kBF16) {
         uint4 v[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) v[i] = *reinterpret_cast<const uint4*>(stage + i * 512 + lane * 16);
+        for (int i = 0; i < 4; ++i) v[i] = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 16);
         PairKeys pk;
         interleave_keys<true>(v, pk);
         uint32_t m[4];
@@ -94,8 +97,8 @@ __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, 
         uint32_t ka[16], kb[16];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const uint4 a = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32);
-            const uint4 b = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32 + 16);
+            const uint4 a = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 32);
+            const uint4 b = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 32 + 16);
             ka[4 * i] = a.x & 0x7FFFFFFFu; ka[4 * i + 1] = a.y & 0x7FFFFFFFu; ka[4 * i + 2] = a.z & 0x7FFFFFFFu; ka[4 * i + 3] = a.w & 0x7FFFFFFFu;
             kb[4 * i] = b.x & 0x7FFFFFFFu; kb[4 * i + 1] = b.y & 0x7FFFFFFFu; kb[4 * i + 2] = b.z & 0x7FFFFFFFu; kb[4 * i + 3] = b.w & 0x7FFFFFFFu;
         }
@@ -128,21 +131,22 @@ __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, 
 template <int DT>
 __device__ __forceinline__ bool swap_apply_smem(const unsigned char* blk, uint32_t& kept16) {
     return swap_apply_2_4(kept16, [blk](int p) -> uint32_t {
-        if constexpr (DT == kBF16) return *reinterpret_cast<const unsigned short*>(blk + (p >> 2) * 512 + (p & 3) * 2) & 0x7FFFu;
-        else return *reinterpret_cast<const uint32_t*>(blk + (p >> 2) * 1024 + (p & 3) * 4) & 0x7FFFFFFFu;
+        if constexpr (DT == kBF16) return *reinterpret_cast<const unsigned short*>(blk + (p >> 2) * (kItemCols * 2) + (p & 3) * 2) & 0x7FFFu;
+        else return *reinterpret_cast<const uint32_t*>(blk + (p >> 2) * (kItemCols * 4) + (p & 3) * 4) & 0x7FFFFFFFu;
     });
 }
 
 // Masked weights back into the stage, mask bytes, objective contribution of the lane's two blocks.
 template <int DT, bool HAS_OUT>
 __device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* mrow /* [4][32] */, const uint4* lut, int lane, uint32_t kept) {
+    constexpr int kPitch = kItemCols * (DT == kF32 ? 4 : 2);
     float s4 = 0.f;
     const uint32_t mb4 = mask_bytes_2_4(kept);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const uint32_t mb = i == 0 ? (mb4 & 0xFFu) : prmt(mb4, 0u, 0x4440 + i);
         if constexpr (DT == kBF16) {
-            const uint4 r = *reinterpret_cast<const uint4*>(stage + i * 512 + lane * 16);
+            const uint4 r = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 16);
             const uint4 mm = lut[mb];
             const uint32_t raw[4] = {r.x, r.y, r.z, r.w}, m[4] = {mm.x, mm.y, mm.z, mm.w};
             uint32_t o[4];
@@ -155,10 +159,10 @@ __device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* m
                 asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(s4) : "h"(lo));        // fp32 accumulator + bf16 addend
                 asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(s4) : "h"(hi));
             }
-            if constexpr (HAS_OUT) *reinterpret_cast<uint4*>(stage + i * 512 + lane * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+            if constexpr (HAS_OUT) *reinterpret_cast<uint4*>(stage + i * kPitch + lane * 16) = make_uint4(o[0], o[1], o[2], o[3]);
         } else {
-            const uint4 ra = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32);
-            const uint4 rb = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32 + 16);
+            const uint4 ra = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 32);
+            const uint4 rb = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 32 + 16);
             const uint32_t raw[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
             uint32_t o[8];
 #pragma unroll
@@ -167,8 +171,8 @@ __device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* m
                 s4 += fabsf(__uint_as_float(o[q]));
             }
             if constexpr (HAS_OUT) {
-                *reinterpret_cast<uint4*>(stage + i * 1024 + lane * 32) = make_uint4(o[0], o[1], o[2], o[3]);
-                *reinterpret_cast<uint4*>(stage + i * 1024 + lane * 32 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
+                *reinterpret_cast<uint4*>(stage + i * kPitch + lane * 32) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4*>(stage + i * kPitch + lane * 32 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
             }
         }
         mrow[i * 32 + lane] = (unsigned char)mb;
@@ -183,6 +187,7 @@ __device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* m
 // the kept magnitudes before absorption.
 template <int DT>
 __device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned char* mrow /* [4][32] */, int lane, uint32_t kept, int n_keep) {
+    constexpr int kPitch = kItemCols * (DT == kF32 ? 4 : 2);
     float s4 = 0.f;
     const uint32_t mb4 = mask_bytes_2_4(kept);
     const double pruned = (double)(4 - n_keep);
@@ -191,12 +196,12 @@ __device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned 
         const uint32_t mb = (mb4 >> (8 * i)) & 0xFFu;
         uint32_t raw[8];
         if constexpr (DT == kBF16) {
-            const uint4 r = *reinterpret_cast<const uint4*>(stage + i * 512 + lane * 16);
+            const uint4 r = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 16);
             raw[0] = r.x << 16; raw[1] = r.x & 0xFFFF0000u; raw[2] = r.y << 16; raw[3] = r.y & 0xFFFF0000u;
             raw[4] = r.z << 16; raw[5] = r.z & 0xFFFF0000u; raw[6] = r.w << 16; raw[7] = r.w & 0xFFFF0000u;
         } else {
-            const uint4 ra = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32);
-            const uint4 rb = *reinterpret_cast<const uint4*>(stage + i * 1024 + lane * 32 + 16);
+            const uint4 ra = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 32);
+            const uint4 rb = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 32 + 16);
             raw[0] = ra.x; raw[1] = ra.y; raw[2] = ra.z; raw[3] = ra.w; raw[4] = rb.x; raw[5] = rb.y; raw[6] = rb.z; raw[7] = rb.w;
         }
         uint32_t o[8];
@@ -216,10 +221,10 @@ __device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned 
             }
         }
         if constexpr (DT == kBF16) {
-            *reinterpret_cast<uint4*>(stage + i * 512 + lane * 16) = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), o[4] | (o[5] << 16), o[6] | (o[7] << 16));
+            *reinterpret_cast<uint4*>(stage + i * kPitch + lane * 16) = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), o[4] | (o[5] << 16), o[6] | (o[7] << 16));
         } else {
-            *reinterpret_cast<uint4*>(stage + i * 1024 + lane * 32) = make_uint4(o[0], o[1], o[2], o[3]);
-            *reinterpret_cast<uint4*>(stage + i * 1024 + lane * 32 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
+            *reinterpret_cast<uint4*>(stage + i * kPitch + lane * 32) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(stage + i * kPitch + lane * 32 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
         }
         mrow[i * 32 + lane] = (unsigned char)mb;
     }
@@ -263,7 +268,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     auto issue_next = [&](int s) {         // all lanes track the cursor, lane 0 issues the copy
         if (lane == 0) {
             mbar_expect_tx(&bars[s], G::kStageBytes);
-            tma_load_2d(stages + s * G::kStageBytes, &tab[ld.k].in, ld.cj * kItemCols, ld.bi * kItemRows, &bars[s]);
+            tma_load_2d(stages + s * G::kStageBytes, &tab[ld.k].in, ld.cj * kTmaBoxUnits, ld.bi * kItemRows, &bars[s]);
         }
         ld.advance(tab, count);
         ++loaded;
@@ -295,7 +300,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                 // N of 4 along rows: kept iff fewer than N entries of the row are heavier
                 const int nk = n_keep & 0xFF;
                 k = nk == 2 ? ~maj3(rel.hr1, rel.hr2, rel.hr3) : (nk == 1 ? ~(rel.hr1 | rel.hr2 | rel.hr3) : ~(rel.hr1 & rel.hr2 & rel.hr3));
-                const int c0 = cur.cj * kItemCols + lane * 8, nc = (int)tab[cur.k].p.cols;
+                const int c0 = cur.cj * kItemCols + h * kHalfCols + lane * 8, nc = (int)tab[cur.k].p.cols;
                 const uint32_t inside = c0 >= nc ? 0u : (c0 + 4 >= nc ? 0xFFFFu : 0xFFFFFFFFu);
                 viol += (unsigned)__popc(~k & nonzero & inside);
             } else {
@@ -355,35 +360,39 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             acc = 0.0; facc = 0.f; acc_k = cur.k;
         }
         // blocks past the last column (zero-filled by the copy) contribute nothing
-        const int col0 = cur.cj * kItemCols + lane * 8;
         const int cols = (int)e.p.cols;
-        const uint32_t colmask = col0 >= cols ? 0u : (col0 + 4 >= cols ? 0xFFFFu : 0xFFFFFFFFu);
+        uint32_t colmask[kHalves];
+#pragma unroll
+        for (int h = 0; h < kHalves; ++h) {
+            const int col0 = cur.cj * kItemCols + h * kHalfCols + lane * 8;
+            colmask[h] = col0 >= cols ? 0u : (col0 + 4 >= cols ? 0xFFFFu : 0xFFFFFFFFu);
+        }
         const int slot = cur.cj & (G::kMaskItems - 1);
         if (mfirst < 0) mfirst = slot;
         if (METHOD == kMethodRows && HAS_OUT && (n_keep & 0x100)) {       // mean absorption requested
 #pragma unroll
             for (int h = 0; h < kHalves; ++h)
-                facc += back_end_absorb<DT>(stage + h * G::kHalfBytes, mbytes + slot * 256 + h * 128, lane, kbuf[h * 32 + lane] & colmask, n_keep & 0xFF);
+                facc += back_end_absorb<DT>(stage + h * G::kHalfBytes, mbytes + slot * 256 + h * 128, lane, kbuf[h * 32 + lane] & colmask[h], n_keep & 0xFF);
         } else {
 #pragma unroll
             for (int h = 0; h < kHalves; ++h)
-                facc += back_end<DT, HAS_OUT>(stage + h * G::kHalfBytes, mbytes + slot * 256 + h * 128, lut, lane, kbuf[h * 32 + lane] & colmask);
+                facc += back_end<DT, HAS_OUT>(stage + h * G::kHalfBytes, mbytes + slot * 256 + h * 128, lut, lane, kbuf[h * 32 + lane] & colmask[h]);
         }
         if constexpr (HAS_OUT) fence_proxy_async_smem();
         __syncwarp();
         if constexpr (HAS_OUT) {
-            if (lane == 0) { tma_store_2d(&e.out, cur.cj * kItemCols, cur.bi * kItemRows, stage); tma_commit(); }
+            if (lane == 0) { tma_store_2d(&e.out, cur.cj * kTmaBoxUnits, cur.bi * kItemRows, stage); tma_commit(); }
         }
         // mask words leave once the buffer holds the last item of an aligned group, of the block row or of this warp
         if (slot == G::kMaskItems - 1 || cur.cj == cur.cchunks - 1 || it == n_items - 1) {
-            const long long rows = e.p.rows;
-            constexpr int kRowWords = 8 * G::kMaskItems;
-            const int word0 = (cur.cj - slot) * 8;
+            const long long rows = e.p.rows;                            // the 1-D pruning takes any number of rows
+            constexpr int kItemWords = kItemCols / 32, kRowWords = kItemWords * G::kMaskItems;
+            const int word0 = (cur.cj - slot) * kItemWords;
 #pragma unroll
-            for (int t = 0; t < 2 * G::kMaskItems; ++t) {               // 8 rows x (8 words per item)
-                const int idx = lane + 32 * t, r = idx / kRowWords, wq = idx % kRowWords, q = wq >> 3;
+            for (int t = 0; t < 2 * G::kMaskItems; ++t) {               // 4 rows x (16 words per item: 8 of either half)
+                const int idx = lane + 32 * t, r = idx / kRowWords, wq = idx % kRowWords, q = wq / kItemWords, hw = wq % kItemWords;
                 const long long row = (long long)cur.bi * kItemRows + r;
-                const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + q * 256 + r * 32 + (wq & 7) * 4);
+                const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + q * 256 + (hw >> 3) * 128 + r * 32 + (hw & 7) * 4);
                 if (q >= mfirst && q <= slot && word0 + wq < e.p.wpr && row < rows) e.p.mask[row * e.p.wpr + word0 + wq] = w;
             }
             mfirst = -1;
@@ -463,9 +472,10 @@ bool tma_eligible(const DevProblem& p, int N, int M, int method) {
     return encode_fn() != nullptr;
 }
 
-// Fills `entries_host` (count TmaEntry records) for problems that all passed tma_eligible(); an item is 8 rows x 256 columns.
+// Fills `entries_host` (count TmaEntry records) for problems that all passed tma_eligible(); an item is one block row
+// of 4 x 512 (M = 4) or 8 x 256 (M = 8) elements.
 bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M) {
-    (void)M;
+    if (M == 8) return build_entries(probs, count, static_cast<TmaEntry*>(entries_host), total_items, 8, 256);
     return build_entries(probs, count, static_cast<TmaEntry*>(entries_host), total_items, kItemRows, kItemCols);
 }
 

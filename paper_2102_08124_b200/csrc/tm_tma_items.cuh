@@ -1,7 +1,7 @@
 // Work-item bookkeeping shared by the bandwidth kernels: one descriptor record per matrix (tensor maps
 // for loads and stores plus the problem), a cursor that walks the items of a table of matrices in
-// order, and the host-side construction of the records.  An item is 8 rows x 256 columns (the last
-// item row of a matrix may be half empty when M = 4).
+// order, and the host-side construction of the records.  An item is one block row of the matrix wide enough
+// to fill a stage: 4 rows x 512 columns for M = 4, 8 rows x 256 columns for M = 8.
 #pragma once
 #include <cstring>
 
@@ -13,8 +13,8 @@ namespace tmask {
 struct alignas(128) TmaEntry {
     CUtensorMap in, out;
     DevProblem p;
-    int cchunks;       // items per block row (256 columns each)
-    int brows;         // item rows (8 matrix rows each)
+    int cchunks;       // items per item row
+    int brows;         // item rows (one block row of the matrix each)
 };
 static_assert(sizeof(TmaEntry) == 384 || sizeof(TmaEntry) == 512, "descriptor records stay 128-byte aligned in tables");
 
@@ -55,14 +55,24 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// A box is at most 256 elements wide, so a wider item is described in units of 2 or 4 matrix elements (the
+// copy moves bytes; rows are 16-byte multiples and the column count a multiple of M, so the units divide
+// evenly and the zero fill past the last column falls on whole units).  The x coordinate of item cj is
+// cj * kTmaBoxUnits for every item shape.
+constexpr int kTmaBoxUnits = 256;
 inline bool encode_map(CUtensorMap* m, const void* base, int dtype, long long rows, long long cols, long long ld, int box_rows, int box_cols) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)ld * (dtype == kF32 ? 4 : 2)};
-    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const int esz = dtype == kF32 ? 4 : 2;
+    const int unit = box_cols * esz / kTmaBoxUnits;                      // bytes per tensor-map element: 2, 4 or 8
+    if (unit != 2 && unit != 4 && unit != 8) return false;
+    if ((cols * esz) % unit) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)(cols * esz / unit), (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * esz};
+    const cuuint32_t box[2] = {(cuuint32_t)kTmaBoxUnits, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    return fn(m, dtype == kF32 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), dims, strides,
+    const CUtensorMapDataType type = unit == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : (unit == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_UINT64);
+    return fn(m, type, 2, const_cast<void*>(base), dims, strides,
               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
