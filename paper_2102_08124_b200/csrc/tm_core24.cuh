@@ -127,40 +127,56 @@ TM_HD uint32_t short_blocks(const LineFill& f) {
     return ((f.row_full & 0xFFFFu) != 0xFFFFu ? 1u : 0u) | ((f.row_full >> 16) != 0xFFFFu ? 2u : 0u);
 }
 
-// index of the lowest set bit (x != 0)
-TM_HD int lowest_bit(uint32_t x) {
+// index of the highest set bit (x != 0)
+TM_HD int highest_bit(uint32_t x) {
 #if defined(__CUDA_ARCH__)
-    return __ffs((int)x) - 1;
+    return 31 - __clz((int)x);
 #else
-    int p = 0;
-    while (!((x >> p) & 1)) ++p;
+    int p = 31;
+    while (!((x >> p) & 1)) --p;
     return p;
 #endif
 }
 
 // Step C for one block flagged by short_blocks(): key(p) returns the magnitude pattern of entry p.  The
 // entry to give way is the lightest of the six kept entries outside the short row (the earliest of equal
-// magnitudes).  Returns false (mask unchanged) on an unexpected shape.
-template <class KeyFn>
+// magnitudes).  SMALL: magnitudes fit in 28 bits, so magnitude and position are compared as one word.
+// Returns false (mask unchanged) on an unexpected shape.
+template <bool SMALL, class KeyFn>
 TM_HD bool swap_apply_2_4(uint32_t& kept16, KeyFn key) {
-    // the short row / column: the only ones not holding two entries
-    const uint32_t a = kept16, t = a | (a >> 1) | (a >> 2);
-    const uint32_t rshort = ((maj3(a, a >> 1, a >> 2) | ((a >> 3) & t)) & 0x1111u) ^ 0x1111u;
-    const uint32_t u = a | (a >> 4) | (a >> 8);
-    const uint32_t cshort = ((maj3(a, a >> 4, a >> 8) | ((a >> 12) & u)) & 0xFu) ^ 0xFu;
-    if (!rshort || (rshort & (rshort - 1)) || !cshort || (cshort & (cshort - 1))) return false;
-    const int r4 = lowest_bit(rshort), c = lowest_bit(cshort);     // r4 = 4 * short row
-    if (!((kept16 >> (r4 + c)) & 1)) return false;
-    uint32_t cands = kept16 & ~(0xFu << r4);
-    int x = -1; uint32_t best = 0;
-    for (int n = 0; n < 6 && cands; ++n) {                          // ascending positions: the earliest of equals wins
-        const int p = lowest_bit(cands);
-        cands &= cands - 1;
-        const uint32_t kp = key(p);
-        if (x < 0 || kp < best) { x = p; best = kp; }
+    const uint32_t a = kept16;
+    const uint32_t s = a - ((a >> 1) & 0x5555u);
+    const uint32_t t = (s & 0x3333u) + ((s >> 2) & 0x3333u);       // kept entries per row, one nibble each
+    const uint32_t rs = t ^ 0x2222u;                               // 3 in the nibble of the row that holds one, 0 where a row holds two
+    if (!rs) return false;
+    const int r4 = highest_bit(rs) - 1;                            // 4 * short row
+    if (r4 < 0 || rs != (3u << r4)) return false;
+    const uint32_t only = (a >> r4) & 0xFu;                        // the short row's single entry: it marks the short column
+    const int c = highest_bit(only);
+    uint32_t cands = a & ~(0xFu << r4);                            // two entries in each of the three other rows
+    int x;
+    if constexpr (SMALL) {
+        uint32_t best = 0xFFFFFFFFu;
+#pragma unroll
+        for (int n = 0; n < 6; ++n) {
+            const int p = highest_bit(cands);
+            cands ^= 1u << p;
+            const uint32_t kp = key(p) * 16u + (uint32_t)p;
+            best = kp < best ? kp : best;
+        }
+        x = (int)(best & 15u);
+    } else {
+        uint32_t best = 0xFFFFFFFFu;
+        x = 0;
+#pragma unroll
+        for (int n = 0; n < 6; ++n) {                              // descending positions: of equals the earliest stays
+            const int p = highest_bit(cands);
+            cands ^= 1u << p;
+            const uint32_t kp = key(p);
+            if (kp <= best) { best = kp; x = p; }
+        }
     }
-    if (cands || x < 0) return false;
-    kept16 = (kept16 & ~(1u << x)) | (1u << (r4 + (x & 3))) | (1u << ((x & ~3) + c));
+    kept16 = (a ^ (1u << x)) | (1u << (r4 + (x & 3))) | (1u << ((x & 12) + c));
     return true;
 }
 

@@ -127,12 +127,15 @@ __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, 
     }
 }
 
-// Step C on a block whose magnitudes sit in shared memory (natural layout).
+// Step C on a block whose magnitudes sit in shared memory (natural layout): entry p = 4i + j lies i rows and j elements on.
 template <int DT>
 __device__ __forceinline__ bool swap_apply_smem(const unsigned char* blk, uint32_t& kept16) {
-    return swap_apply_2_4(kept16, [blk](int p) -> uint32_t {
-        if constexpr (DT == kBF16) return *reinterpret_cast<const unsigned short*>(blk + (p >> 2) * (kItemCols * 2) + (p & 3) * 2) & 0x7FFFu;
-        else return *reinterpret_cast<const uint32_t*>(blk + (p >> 2) * (kItemCols * 4) + (p & 3) * 4) & 0x7FFFFFFFu;
+    constexpr int kElemBytes = DT == kF32 ? 4 : 2;
+    constexpr int kRowStep = kItemCols * kElemBytes / 4 - kElemBytes;      // offset(p) = p * elem + (p & 12) * kRowStep
+    return swap_apply_2_4<DT == kBF16>(kept16, [blk](int p) -> uint32_t {
+        const unsigned char* at = blk + p * kElemBytes + (p & 12) * kRowStep;
+        if constexpr (DT == kBF16) return *reinterpret_cast<const unsigned short*>(at) & 0x7FFFu;
+        else return *reinterpret_cast<const uint32_t*>(at) & 0x7FFFFFFFu;
     });
 }
 
