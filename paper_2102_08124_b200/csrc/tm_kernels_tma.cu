@@ -45,12 +45,8 @@ template <int DT, int METHOD> struct Geometry {
     static constexpr int kRowPitch = kItemCols * kElem;        // bytes between rows inside a stage
     static constexpr int kHalfBytes = kHalfCols * kElem;       // from the first half of a row to the second
     static constexpr int kStageBytes = kItemRows * kRowPitch;
-    // Mask bytes of this many consecutive items are collected before they leave, so that a row's words go
-    // out as one longer run instead of 32-byte pieces.  Measured: it helps where the kernel waits for memory
-    // (Algorithm 1 alone) and costs more than it gives where it waits for the integer pipe (full search).
-    static constexpr int kMaskItems = DT == kF32 ? 4 : (METHOD == kMethodApprox ? 1 : 2);
-    // stages | mask bytes [items][half][4][32] | kept [2][32] | queue [128] | barriers
-    static constexpr int kWarpBytes = kStages * kStageBytes + kMaskItems * 256 + 256 + 128 + 128;
+    // stages | mask bytes [half][4][32] | kept [2][32] | queue [128] | barriers
+    static constexpr int kWarpBytes = kStages * kStageBytes + 256 + 256 + 128 + 128;
     static constexpr int kSmemBytes = kWarps * kWarpBytes + (DT == kBF16 ? kLaneLutBytes : 0);
     static_assert(kSmemBytes <= 232448, "at most 227 KB of shared memory per CTA");
     static_assert(kWarpBytes % 128 == 0, "stages stay 128-byte aligned");
@@ -243,7 +239,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned char* stages = smem_raw + (size_t)warp * G::kWarpBytes;
     unsigned char* mbytes = stages + G::kStages * G::kStageBytes;
-    uint32_t* kbuf = reinterpret_cast<uint32_t*>(mbytes + G::kMaskItems * 256);
+    uint32_t* kbuf = reinterpret_cast<uint32_t*>(mbytes + 256);
     unsigned char* queue = reinterpret_cast<unsigned char*>(kbuf + kHalves * 32);
     uint64_t* bars = reinterpret_cast<uint64_t*>(queue + 128);
     uint4* lut = reinterpret_cast<uint4*>(smem_raw + (size_t)G::kWarps * G::kWarpBytes);
@@ -283,7 +279,12 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     uint32_t worst = 0;                                                  // largest magnitude pattern seen (per 16-bit lane for bf16)
     const uint32_t lt = (1u << lane) - 1u;
     bool alive = true;
-    int mfirst = -1;                                                     // first slot of the mask-byte buffer in use
+    // the matrix in process: the fields every item needs
+    int p_cols = 0, p_wpr = 0, p_rows = 0;
+    uint32_t* p_mask = nullptr;
+    // an item's mask words: 4 rows x 16 words, lane -> word (lane & 15) of rows (lane >> 4) and (lane >> 4) + 2
+    const int mw = lane & 15, mr = lane >> 4;
+    const unsigned char* msrc = mbytes + (mw >> 3) * 128 + mr * 32 + (mw & 7) * 4;
     unsigned long long viol = 0;                                         // kMethodRows: non-zero entries pruned by this lane
 
     for (int it = 0; it < n_items && alive; ++it) {
@@ -292,7 +293,19 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         unsigned char* stage = stages + s * G::kStageBytes;
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bars[s], parity))) { status |= kDevInternal; alive = false; }
         int qn = 0;
-        // ---- steps A and B on both block rows -----------------------------------------------------
+        if (cur.k != acc_k) {                                   // a new matrix starts: flush the objective partial
+            if (acc_k >= 0) {
+                acc += (double)facc;
+                for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+                if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
+            }
+            acc = 0.0; facc = 0.f; acc_k = cur.k;
+            const DevProblem& P = tab[cur.k].p;
+            p_cols = (int)P.cols; p_wpr = P.wpr; p_rows = (int)P.rows; p_mask = P.mask;
+        }
+        // does the item lie inside the matrix? (warp-uniform; otherwise the copy zero-filled the rest)
+        const bool inside_cols = cur.cj < p_cols / kItemCols, inside = inside_cols && cur.bi < p_rows / kItemRows;
+        // ---- steps A and B on both halves ---------------------------------------------------------
 #pragma unroll
         for (int h = 0; h < kHalves; ++h) {
             Rel24 rel;
@@ -303,9 +316,9 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                 // N of 4 along rows: kept iff fewer than N entries of the row are heavier
                 const int nk = n_keep & 0xFF;
                 k = nk == 2 ? ~maj3(rel.hr1, rel.hr2, rel.hr3) : (nk == 1 ? ~(rel.hr1 | rel.hr2 | rel.hr3) : ~(rel.hr1 & rel.hr2 & rel.hr3));
-                const int c0 = cur.cj * kItemCols + h * kHalfCols + lane * 8, nc = (int)tab[cur.k].p.cols;
-                const uint32_t inside = c0 >= nc ? 0u : (c0 + 4 >= nc ? 0xFFFFu : 0xFFFFFFFFu);
-                viol += (unsigned)__popc(~k & nonzero & inside);
+                const int c0 = cur.cj * kItemCols + h * kHalfCols + lane * 8;
+                const uint32_t in_cols = c0 >= p_cols ? 0u : (c0 + 4 >= p_cols ? 0xFFFFu : 0xFFFFFFFFu);
+                viol += (unsigned)__popc(~k & nonzero & in_cols);
             } else {
                 k = cover_2_4(rel);
             }
@@ -353,52 +366,38 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             __syncwarp();
         }
         // ---- outputs ---------------------------------------------------------------------------
-        const TmaEntry& e = tab[cur.k];
-        if (cur.k != acc_k) {                                   // a new matrix starts: flush the objective partial
-            if (acc_k >= 0) {
-                acc += (double)facc;
-                for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-                if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
-            }
-            acc = 0.0; facc = 0.f; acc_k = cur.k;
-        }
         // blocks past the last column (zero-filled by the copy) contribute nothing
-        const int cols = (int)e.p.cols;
-        uint32_t colmask[kHalves];
+        uint32_t colmask[kHalves] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+        if (!inside_cols) {
 #pragma unroll
-        for (int h = 0; h < kHalves; ++h) {
-            const int col0 = cur.cj * kItemCols + h * kHalfCols + lane * 8;
-            colmask[h] = col0 >= cols ? 0u : (col0 + 4 >= cols ? 0xFFFFu : 0xFFFFFFFFu);
+            for (int h = 0; h < kHalves; ++h) {
+                const int col0 = cur.cj * kItemCols + h * kHalfCols + lane * 8;
+                colmask[h] = col0 >= p_cols ? 0u : (col0 + 4 >= p_cols ? 0xFFFFu : 0xFFFFFFFFu);
+            }
         }
-        const int slot = cur.cj & (G::kMaskItems - 1);
-        if (mfirst < 0) mfirst = slot;
         if (METHOD == kMethodRows && HAS_OUT && (n_keep & 0x100)) {       // mean absorption requested
 #pragma unroll
             for (int h = 0; h < kHalves; ++h)
-                facc += back_end_absorb<DT>(stage + h * G::kHalfBytes, mbytes + slot * 256 + h * 128, lane, kbuf[h * 32 + lane] & colmask[h], n_keep & 0xFF);
+                facc += back_end_absorb<DT>(stage + h * G::kHalfBytes, mbytes + h * 128, lane, kbuf[h * 32 + lane] & colmask[h], n_keep & 0xFF);
         } else {
 #pragma unroll
             for (int h = 0; h < kHalves; ++h)
-                facc += back_end<DT, HAS_OUT>(stage + h * G::kHalfBytes, mbytes + slot * 256 + h * 128, lut, lane, kbuf[h * 32 + lane] & colmask[h]);
+                facc += back_end<DT, HAS_OUT>(stage + h * G::kHalfBytes, mbytes + h * 128, lut, lane, kbuf[h * 32 + lane] & colmask[h]);
         }
         if constexpr (HAS_OUT) fence_proxy_async_smem();
         __syncwarp();
         if constexpr (HAS_OUT) {
-            if (lane == 0) { tma_store_2d(&e.out, cur.cj * kTmaBoxUnits, cur.bi * kItemRows, stage); tma_commit(); }
+            if (lane == 0) { tma_store_2d(&tab[cur.k].out, cur.cj * kTmaBoxUnits, cur.bi * kItemRows, stage); tma_commit(); }
         }
-        // mask words leave once the buffer holds the last item of an aligned group, of the block row or of this warp
-        if (slot == G::kMaskItems - 1 || cur.cj == cur.cchunks - 1 || it == n_items - 1) {
-            const long long rows = e.p.rows;                            // the 1-D pruning takes any number of rows
-            constexpr int kItemWords = kItemCols / 32, kRowWords = kItemWords * G::kMaskItems;
-            const int word0 = (cur.cj - slot) * kItemWords;
-#pragma unroll
-            for (int t = 0; t < 2 * G::kMaskItems; ++t) {               // 4 rows x (16 words per item: 8 of either half)
-                const int idx = lane + 32 * t, r = idx / kRowWords, wq = idx % kRowWords, q = wq / kItemWords, hw = wq % kItemWords;
-                const long long row = (long long)cur.bi * kItemRows + r;
-                const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + q * 256 + (hw >> 3) * 128 + r * 32 + (hw & 7) * 4);
-                if (q >= mfirst && q <= slot && word0 + wq < e.p.wpr && row < rows) e.p.mask[row * e.p.wpr + word0 + wq] = w;
+        {   // mask words: 64 bytes per row
+            const uint32_t w0 = *reinterpret_cast<const uint32_t*>(msrc), w1 = *reinterpret_cast<const uint32_t*>(msrc + 64);
+            const int word = cur.cj * (kItemCols / 32) + mw, row = cur.bi * kItemRows + mr;
+            uint32_t* dst = p_mask + (long long)row * p_wpr + word;
+            if (inside) { dst[0] = w0; dst[2 * (long long)p_wpr] = w1; }
+            else if (word < p_wpr) {                                    // the 1-D pruning takes any number of rows
+                if (row < p_rows) dst[0] = w0;
+                if (row + 2 < p_rows) dst[2 * (long long)p_wpr] = w1;
             }
-            mfirst = -1;
         }
         cur.advance(tab, count);
         if ((it & 31) == 31) { acc += (double)facc; facc = 0.f; }           // keep the fp32 partial short
