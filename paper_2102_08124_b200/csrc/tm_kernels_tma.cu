@@ -1,7 +1,8 @@
 // Bandwidth kernels of the approximate 2:4 search (TM_APPROX / TM_APPROX_COVER, M = 4).
 //
-// Every warp runs its own software pipeline over a contiguous range of work items (4 rows x 512
-// columns of one matrix: one block row, 128 blocks, in two halves of 256 columns):
+// Every warp runs its own software pipeline over work items (4 rows x 512 columns of one matrix: one
+// block row, 128 blocks, in two halves of 256 columns) -- a contiguous range for the full search,
+// every n-th item for the variants that only wait for memory:
 //   1. lane 0 keeps the bulk-tensor (TMA) load of the next item in flight into the other of the warp's
 //      two private shared-memory stages;
 //   2. each lane reads its two 4x4 blocks of either block row with 128-bit shared loads and runs steps
@@ -25,6 +26,7 @@
 #include "tm_tma_items.cuh"
 
 #include <cstring>
+#include <type_traits>
 
 namespace tmask {
 
@@ -249,9 +251,15 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     }
 
     const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
+    // A fixed deal of the items, so the objective's partial sums are reproducible.  Where the kernel waits for memory
+    // (Algorithm 1 alone, the 1-D pruning) the warps take the items round-robin -- gw, gw + nwarps, ... -- so that the
+    // whole grid works on one dense window of the matrix (3 % faster there); the full search, which also waits for the
+    // integer pipe, is indifferent to the order and 2 % faster with the plain cursor of a contiguous range.
+    constexpr bool kRoundRobin = METHOD != kMethodApprox;
     const long long per = (total_items + nwarps - 1) / nwarps;
-    const long long begin = gw * per, end = min(total_items, begin + per);
-    const int n_items = (int)max(0ll, end - begin);
+    const long long first = kRoundRobin ? gw : gw * per;
+    const int n_items = kRoundRobin ? (gw < total_items ? (int)((total_items - gw + nwarps - 1) / nwarps) : 0)
+                                    : (int)max(0ll, min(total_items, first + per) - first);
     const TmaEntry* tab = table ? table : &single;
 
     if (lane == 0) {
@@ -260,8 +268,8 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     }
     __syncwarp();
 
-    Cursor ld, cur;                        // next item to request / item in process
-    ld.seek(tab, count, begin);
+    typename std::conditional<kRoundRobin, StrideCursor, Cursor>::type ld, cur;      // next item to request / item in process
+    if constexpr (kRoundRobin) ld.seek(tab, count, first, (int)nwarps); else ld.seek(tab, count, first);
     cur = ld;
     int loaded = 0;
     auto issue_next = [&](int s) {         // all lanes track the cursor, lane 0 issues the copy

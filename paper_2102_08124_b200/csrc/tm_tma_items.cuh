@@ -40,6 +40,40 @@ struct Cursor {
     }
 };
 
+// The same walk in steps of `stride` items (the warps of a launch take the items round-robin, so that at any
+// moment the whole grid works on one dense window of the matrix).  Inside a matrix a step is an addition;
+// only the step that leaves a matrix goes through the item index.
+struct StrideCursor {
+    int k, bi, cj, cchunks, brows, dbi, dcj, stride;
+    __device__ __forceinline__ void enter(const TmaEntry* tab, int count) {
+        while (k < count && (tab[k].brows == 0 || tab[k].cchunks == 0)) ++k;   // empty matrices have no items
+        if (k < count) { cchunks = tab[k].cchunks; brows = tab[k].brows; } else { cchunks = 1; brows = 1; }
+        dbi = stride / cchunks; dcj = stride - dbi * cchunks;
+    }
+    __device__ __forceinline__ void seek(const TmaEntry* tab, int count, long long item, int stride_) {
+        stride = stride_;
+        k = 0;
+        while (k + 1 < count && tab[k + 1].p.item_begin <= item) ++k;
+        enter(tab, count);
+        const long long local = item - tab[k < count ? k : count - 1].p.item_begin;
+        bi = (int)(local / cchunks); cj = (int)(local - (long long)bi * cchunks);
+    }
+    __device__ __forceinline__ void advance(const TmaEntry* tab, int count) {
+        cj += dcj; bi += dbi;
+        if (cj >= cchunks) { cj -= cchunks; ++bi; }
+        if (bi >= brows) {
+            long long over = (long long)(bi - brows) * cchunks + cj;             // items past the end of matrix k
+            for (;;) {
+                ++k; enter(tab, count);
+                if (k >= count) { bi = 0; cj = 0; break; }
+                const long long n = (long long)brows * cchunks;
+                if (over < n) { bi = (int)(over / cchunks); cj = (int)(over - (long long)bi * cchunks); break; }
+                over -= n;
+            }
+        }
+    }
+};
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
