@@ -501,8 +501,9 @@ int tm_nm_mask_1d(const tm_problem* prob_host, int N, int M, int flags, unsigned
             if (tmask::tma_entry_bytes() <= sizeof(entry) && tmask::tma_build_entries(&dp, 1, entry, &total, 4)) {
                 tmask::TmaLaunch t;
                 t.entries_host = entry; t.entries_dev = nullptr; t.count = 1; t.total_items = total; t.partials = op; t.status = status_dev;
-                t.dtype = p.dtype; t.method = tmask::kMethodRows; t.M = 4; t.has_out = p.masked_w_out != nullptr;
-                t.stream = static_cast<cudaStream_t>(cuda_stream); t.n_keep = N | ((flags & TM_NM1D_ABSORB_MEAN) ? 0x100 : 0); t.vpartials = vp;
+                t.dtype = p.dtype; t.M = 4; t.has_out = p.masked_w_out != nullptr;
+                t.method = (flags & TM_NM1D_ABSORB_MEAN) && t.has_out ? tmask::kMethodRowsAbsorb : tmask::kMethodRows;
+                t.stream = static_cast<cudaStream_t>(cuda_stream); t.n_keep = N; t.vpartials = vp;
                 const int wpc = tmask::tma_warps_per_cta(t.dtype, 4, t.method);
                 const long long want = (total + wpc - 1) / wpc;
                 const int cap = d->sms < tmask::aux_partial_slots() / wpc ? d->sms : tmask::aux_partial_slots() / wpc;

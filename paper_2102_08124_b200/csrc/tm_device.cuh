@@ -9,6 +9,7 @@ constexpr int kMethodExact = 0;
 constexpr int kMethodApprox = 1;
 constexpr int kMethodCover = 2;
 constexpr int kMethodRows = 3;       // internal: plain N:M along rows (no column constraint), M = 4
+constexpr int kMethodRowsAbsorb = 4; // internal: the same with the mean of the pruned weights absorbed into the kept ones
 constexpr int kF32 = 0;
 constexpr int kBF16 = 1;
 constexpr int kDevNonFinite = 1;

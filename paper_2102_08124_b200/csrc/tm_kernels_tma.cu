@@ -37,12 +37,15 @@ constexpr int kHalves = 2;                 // processed as two halves of 256 col
 constexpr int kItemCols = 512;
 constexpr int kHalfCols = kItemCols / kHalves;
 
-// Warps per CTA (one CTA per SM) and stages per warp.  The search is bound by integer issue and wants many
-// warps: for bf16, 24 warps at 80 registers per thread fill the shared memory with two stages each (a
-// deeper ring with fewer warps measured no faster, also for Algorithm 1 alone).
+// Warps per CTA (one CTA per SM) and stages per warp.  The full search is bound by integer issue and wants many
+// warps: for bf16, 24 warps at 80 registers per thread fill the shared memory with two stages each (a deeper ring
+// with fewer warps measured no faster).  Algorithm 1 alone and the 1-D pruning only wait for memory, and the memory
+// system is at its best with about 96 KB of stages per SM: 12 warps for bf16 (0.387 ms on the 12288 x 49152 matrix
+// against 0.418 / 0.427 / 0.449 ms with 10 / 14 / 16 warps), 6 for fp32.
 template <int DT, int METHOD> struct Geometry {
     static constexpr int kElem = DT == kF32 ? 4 : 2;
-    static constexpr int kWarps = DT == kF32 ? 12 : 24;
+    static constexpr bool kHeavy = METHOD == kMethodApprox || METHOD == kMethodRowsAbsorb;      // bound by arithmetic, not by memory
+    static constexpr int kWarps = kHeavy ? (DT == kF32 ? 12 : 24) : (DT == kF32 ? 6 : 12);
     static constexpr int kStages = 2;
     static constexpr int kRowPitch = kItemCols * kElem;        // bytes between rows inside a stage
     static constexpr int kHalfBytes = kHalfCols * kElem;       // from the first half of a row to the second
@@ -237,6 +240,7 @@ __global__ void __launch_bounds__(Geometry<DT, METHOD>::kWarps * 32, 1)
 tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict__ table, int count, long long total_items,
              double* __restrict__ partials, int* __restrict__ status_out, int n_keep, unsigned long long* __restrict__ vpartials) {
     using G = Geometry<DT, METHOD>;
+    constexpr bool kRows = METHOD == kMethodRows || METHOD == kMethodRowsAbsorb;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned char* stages = smem_raw + (size_t)warp * G::kWarpBytes;
@@ -255,7 +259,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     // (Algorithm 1 alone, the 1-D pruning) the warps take the items round-robin -- gw, gw + nwarps, ... -- so that the
     // whole grid works on one dense window of the matrix (3 % faster there); the full search, which also waits for the
     // integer pipe, is indifferent to the order and 2 % faster with the plain cursor of a contiguous range.
-    constexpr bool kRoundRobin = METHOD != kMethodApprox;
+    constexpr bool kRoundRobin = !G::kHeavy;
     const long long per = (total_items + nwarps - 1) / nwarps;
     const long long first = kRoundRobin ? gw : gw * per;
     const int n_items = kRoundRobin ? (gw < total_items ? (int)((total_items - gw + nwarps - 1) / nwarps) : 0)
@@ -318,11 +322,11 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         for (int h = 0; h < kHalves; ++h) {
             Rel24 rel;
             uint32_t nonzero = 0;
-            front_end<DT, METHOD == kMethodRows>(stage + h * G::kHalfBytes, lane, rel, worst, nonzero);
+            front_end<DT, kRows>(stage + h * G::kHalfBytes, lane, rel, worst, nonzero);
             uint32_t k;
-            if constexpr (METHOD == kMethodRows) {
+            if constexpr (kRows) {
                 // N of 4 along rows: kept iff fewer than N entries of the row are heavier
-                const int nk = n_keep & 0xFF;
+                const int nk = n_keep;
                 k = nk == 2 ? ~maj3(rel.hr1, rel.hr2, rel.hr3) : (nk == 1 ? ~(rel.hr1 | rel.hr2 | rel.hr3) : ~(rel.hr1 & rel.hr2 & rel.hr3));
                 const int c0 = cur.cj * kItemCols + h * kHalfCols + lane * 8;
                 const uint32_t in_cols = c0 >= p_cols ? 0u : (c0 + 4 >= p_cols ? 0xFFFFu : 0xFFFFFFFFu);
@@ -383,10 +387,10 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                 colmask[h] = col0 >= p_cols ? 0u : (col0 + 4 >= p_cols ? 0xFFFFu : 0xFFFFFFFFu);
             }
         }
-        if (METHOD == kMethodRows && HAS_OUT && (n_keep & 0x100)) {       // mean absorption requested
+        if constexpr (METHOD == kMethodRowsAbsorb && HAS_OUT) {
 #pragma unroll
             for (int h = 0; h < kHalves; ++h)
-                facc += back_end_absorb<DT>(stage + h * G::kHalfBytes, mbytes + h * 128, lane, kbuf[h * 32 + lane] & colmask[h], n_keep & 0xFF);
+                facc += back_end_absorb<DT>(stage + h * G::kHalfBytes, mbytes + h * 128, lane, kbuf[h * 32 + lane] & colmask[h], n_keep);
         } else {
 #pragma unroll
             for (int h = 0; h < kHalves; ++h)
@@ -425,7 +429,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     else { if (nonfinite_bf16x2(worst)) status |= kDevNonFinite; }
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(0xFFFFFFFFu, status, o);
     if (lane == 0 && status && status_out) atomicOr(status_out, status);
-    if constexpr (METHOD == kMethodRows) {
+    if constexpr (kRows) {
         for (int o = 16; o; o >>= 1) viol += __shfl_xor_sync(0xFFFFFFFFu, viol, o);
         if (lane == 0 && vpartials) vpartials[gw] = viol;
     }
@@ -467,12 +471,13 @@ cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntr
 size_t tma_entry_bytes() { return sizeof(TmaEntry); }
 int tma_warps_per_cta(int dtype, int M, int method) {
     if (M == 8) return tma48_warps_per_cta(dtype);
-    if (dtype == kF32) return method == kMethodApprox ? Geometry<kF32, kMethodApprox>::kWarps : (method == kMethodRows ? Geometry<kF32, kMethodRows>::kWarps : Geometry<kF32, kMethodCover>::kWarps);
-    return method == kMethodApprox ? Geometry<kBF16, kMethodApprox>::kWarps : (method == kMethodRows ? Geometry<kBF16, kMethodRows>::kWarps : Geometry<kBF16, kMethodCover>::kWarps);
+    const bool heavy = method == kMethodApprox || method == kMethodRowsAbsorb;
+    if (dtype == kF32) return heavy ? Geometry<kF32, kMethodApprox>::kWarps : Geometry<kF32, kMethodCover>::kWarps;
+    return heavy ? Geometry<kBF16, kMethodApprox>::kWarps : Geometry<kBF16, kMethodCover>::kWarps;
 }
 
 bool tma_eligible(const DevProblem& p, int N, int M, int method) {
-    if (method == kMethodRows) { if (M != 4 || N < 1 || N > 3) return false; }
+    if (method == kMethodRows || method == kMethodRowsAbsorb) { if (M != 4 || N < 1 || N > 3) return false; }
     else if (!((N == 2 && M == 4) || (N == 4 && M == 8)) || (method != kMethodApprox && method != kMethodCover)) return false;
     const size_t elem = p.dtype == kF32 ? 4 : 2;
     if ((uintptr_t)p.W % 16 || ((size_t)p.ld * elem) % 16) return false;
@@ -506,12 +511,12 @@ cudaError_t launch_tma(const TmaLaunch& a) {
     if (a.total_items > 0) {
 #define TM_DISPATCH(DT, METHOD)                                                                                   \
     err = a.has_out ? launch_one<DT, METHOD, true>(a, host[0], table) : launch_one<DT, METHOD, false>(a, host[0], table)
-        if (a.dtype == kF32) { if (a.method == kMethodApprox) TM_DISPATCH(kF32, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kF32, kMethodRows); else TM_DISPATCH(kF32, kMethodCover); }
-        else { if (a.method == kMethodApprox) TM_DISPATCH(kBF16, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kBF16, kMethodRows); else TM_DISPATCH(kBF16, kMethodCover); }
+        if (a.dtype == kF32) { if (a.method == kMethodApprox) TM_DISPATCH(kF32, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kF32, kMethodRows); else if (a.method == kMethodRowsAbsorb) TM_DISPATCH(kF32, kMethodRowsAbsorb); else TM_DISPATCH(kF32, kMethodCover); }
+        else { if (a.method == kMethodApprox) TM_DISPATCH(kBF16, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kBF16, kMethodRows); else if (a.method == kMethodRowsAbsorb) TM_DISPATCH(kBF16, kMethodRowsAbsorb); else TM_DISPATCH(kBF16, kMethodCover); }
 #undef TM_DISPATCH
         if (err != cudaSuccess) return err;
     }
-    if (a.method == kMethodRows) return cudaSuccess;       // the caller sums objective and violation partials together
+    if (a.method == kMethodRows || a.method == kMethodRowsAbsorb) return cudaSuccess;       // the caller sums objective and violation partials together
     reduce_tma_kernel<<<a.count, 256, 0, a.stream>>>(host[0], table, a.partials, (long long)a.ctas * wpc);
     return cudaGetLastError();
 }

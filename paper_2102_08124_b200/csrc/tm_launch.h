@@ -32,8 +32,8 @@ struct TmaLaunch {
     int ctas;
     int dtype, method, M;
     bool has_out;               // masked_w_out present (all problems of one launch agree)
-    int n_keep = 2;             // kMethodRows only: entries kept per group of four (1..3); | 0x100: mean absorption into masked_w_out
-    unsigned long long* vpartials = nullptr;   // kMethodRows only (count == 1): ctas * warps pattern-violation partials; the caller reduces
+    int n_keep = 2;             // kMethodRows / kMethodRowsAbsorb: entries kept per group of four (1..3)
+    unsigned long long* vpartials = nullptr;   // kMethodRows / kMethodRowsAbsorb (count == 1): ctas * warps pattern-violation partials; the caller reduces
     cudaStream_t stream;
 };
 size_t tma_entry_bytes();
