@@ -307,7 +307,7 @@ def run_survey(args):
                 step()
             torch.cuda.synchronize()
             t0 = time.perf_counter(); step(); torch.cuda.synchronize(); once = time.perf_counter() - t0
-            steps = max(3, min(200, int(0.5 / max(once, 1e-5))))
+            steps = args.survey_steps or max(3, min(200, int(0.5 / max(once, 1e-5))))
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             for _ in range(steps):
@@ -337,7 +337,7 @@ def run_survey_neighbours(args):
             fn()
         torch.cuda.synchronize()
         t0 = time.perf_counter(); fn(); torch.cuda.synchronize(); once = time.perf_counter() - t0
-        steps = max(min_steps, min(200, int(0.3 / max(once, 1e-5))))
+        steps = args.survey_steps or max(min_steps, min(200, int(0.3 / max(once, 1e-5))))
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
@@ -400,6 +400,7 @@ def main():
     ap.add_argument("--skip-clocks", action="store_true", help="no nvidia-smi sampling and no extended warm-up")
     ap.add_argument("--survey", action="store_true", help="secondary table: all named workloads and methods, one JSON line each")
     ap.add_argument("--config", type=int, default=0, help="with --survey: only this workload (1..5)")
+    ap.add_argument("--survey-steps", type=int, default=0, help="with --survey: timed calls per case (default: about 0.5 s worth, at most 200)")
     args = ap.parse_args()
     if args.survey:
         if not args.config:

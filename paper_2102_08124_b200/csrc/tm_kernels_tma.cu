@@ -470,7 +470,7 @@ cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntr
 
 size_t tma_entry_bytes() { return sizeof(TmaEntry); }
 int tma_warps_per_cta(int dtype, int M, int method) {
-    if (M == 8) return tma48_warps_per_cta(dtype);
+    if (M == 8) return tma48_warps_per_cta(dtype, method);
     const bool heavy = method == kMethodApprox || method == kMethodRowsAbsorb;
     if (dtype == kF32) return heavy ? Geometry<kF32, kMethodApprox>::kWarps : Geometry<kF32, kMethodCover>::kWarps;
     return heavy ? Geometry<kBF16, kMethodApprox>::kWarps : Geometry<kBF16, kMethodCover>::kWarps;

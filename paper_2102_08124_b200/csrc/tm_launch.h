@@ -42,7 +42,7 @@ bool tma_eligible(const DevProblem& p, int N, int M, int method);
 bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M);
 cudaError_t tma_reduce(const void* entries_host, const void* entries_dev, int count, const double* partials, long long stride, cudaStream_t stream);
 // 4:8 variant (tm_kernels_tma48.cu), reached through launch_tma()
-int tma48_warps_per_cta(int dtype);
+int tma48_warps_per_cta(int dtype, int method);
 cudaError_t launch_tma48(const TmaLaunch& a);
 cudaError_t launch_tma(const TmaLaunch& a);
 
