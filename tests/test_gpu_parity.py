@@ -184,6 +184,21 @@ def test_batched_mixed_dtypes_and_strides(method):
     _batched_parity(mats[:4], 2, 4, method, strided=True)
 
 
+def test_batched_cover_deals_items_round_robin():
+    """Algorithm 1 alone takes the work items of a call round-robin over the warps of the grid, so one step of a warp may leave
+    a matrix, skip several small ones and land in the middle of another.  Many matrices of a few items each (fp32 and bf16 in one
+    call, ragged last items, one matrix of a single block; more items than warps, so every warp steps), then the 54 matrices of the ResNet-50-shaped model."""
+    mats = []
+    for k in range(240):                       # about 1700 items for the 888 warps of the fp32 launch
+        mats.append(workloads.normal_f32(4 * (1 + k % 5), 4 * (1 + (k * 37) % 331), 0.05, 300 + k))
+    for k in range(120):                       # about 3600 items for the 1776 warps of the bf16 launch
+        mats.append(workloads.normal_bf16(32 + 4 * (k % 9), 8 * (120 + (k * 29) % 140), 0.02, 600 + k))
+    mats.append(workloads.normal_f32(4, 4, 1.0, 399))
+    _batched_parity(mats, 2, 4, tm.TM_APPROX_COVER)
+    _batched_parity(mats, 2, 4, tm.TM_APPROX)
+    _batched_parity(workloads.config2(), 2, 4, tm.TM_APPROX_COVER)
+
+
 def test_prepared_batch_object():
     mats = [workloads.normal_f32(32, 264, 0.05, 61), workloads.normal_bf16(16, 520, 0.02, 62)]
     batch = tm.TmBatch([to_device(m) for m in mats])
