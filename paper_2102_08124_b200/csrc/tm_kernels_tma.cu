@@ -1,4 +1,5 @@
-// Bandwidth kernels of the approximate 2:4 search (TM_APPROX / TM_APPROX_COVER, M = 4).
+// Bandwidth kernels of the 2:4 search (TM_APPROX / TM_APPROX_COVER and, with the 90-pattern scorer in place of
+// steps A to C, TM_EXACT; M = 4).
 //
 // Every warp runs its own software pipeline over work items (4 rows x 512 columns of one matrix: one
 // block row, 128 blocks, in two halves of 256 columns) -- a contiguous range for the full search,
@@ -22,6 +23,7 @@
 #include "tm_core24.cuh"
 #include "tm_launch.h"
 #include "tm_pair_bf16.cuh"
+#include "tm_solvers.cuh"
 #include "tm_tma.cuh"
 #include "tm_tma_items.cuh"
 
@@ -44,8 +46,10 @@ constexpr int kHalfCols = kItemCols / kHalves;
 // against 0.418 / 0.427 / 0.449 ms with 10 / 14 / 16 warps), 6 for fp32.
 template <int DT, int METHOD> struct Geometry {
     static constexpr int kElem = DT == kF32 ? 4 : 2;
-    static constexpr bool kHeavy = METHOD == kMethodApprox || METHOD == kMethodRowsAbsorb;      // bound by arithmetic, not by memory
-    static constexpr int kWarps = kHeavy ? (DT == kF32 ? 12 : 24) : (DT == kF32 ? 6 : 12);
+    static constexpr bool kHeavy = METHOD == kMethodApprox || METHOD == kMethodRowsAbsorb || METHOD == kMethodExact;      // bound by arithmetic, not by memory
+    // the exact scorer wants registers: 20 warps (96 registers a thread) measured best for bf16 (1.12 ms on the 12288 x 49152
+    // matrix against 1.16 / 1.20 ms with 16 / 12 warps)
+    static constexpr int kWarps = METHOD == kMethodExact ? (DT == kF32 ? 12 : 20) : (kHeavy ? (DT == kF32 ? 12 : 24) : (DT == kF32 ? 6 : 12));
     static constexpr int kStages = 2;
     static constexpr int kRowPitch = kItemCols * kElem;        // bytes between rows inside a stage
     static constexpr int kHalfBytes = kHalfCols * kElem;       // from the first half of a row to the second
@@ -322,8 +326,33 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         for (int h = 0; h < kHalves; ++h) {
             Rel24 rel;
             uint32_t nonzero = 0;
-            front_end<DT, kRows>(stage + h * G::kHalfBytes, lane, rel, worst, nonzero);
             uint32_t k;
+            if constexpr (METHOD == kMethodExact) {
+                // the optimum of Eq. 1 for either of the lane's two blocks: all 90 patterns, exact integer sums
+                k = 0;
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    const unsigned char* blk = stage + h * G::kHalfBytes + lane * (8 * G::kElem) + b * (4 * G::kElem);
+                    uint32_t u[16];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if constexpr (DT == kBF16) {
+                            const uint2 v = *reinterpret_cast<const uint2*>(blk + i * G::kRowPitch);
+                            u[4 * i] = (v.x << 16) & 0x7FFFFFFFu; u[4 * i + 1] = v.x & 0x7FFF0000u;
+                            u[4 * i + 2] = (v.y << 16) & 0x7FFFFFFFu; u[4 * i + 3] = v.y & 0x7FFF0000u;
+                        } else {
+                            const uint4 v = *reinterpret_cast<const uint4*>(blk + i * G::kRowPitch);
+                            u[4 * i] = v.x & 0x7FFFFFFFu; u[4 * i + 1] = v.y & 0x7FFFFFFFu; u[4 * i + 2] = v.z & 0x7FFFFFFFu; u[4 * i + 3] = v.w & 0x7FFFFFFFu;
+                        }
+                    }
+                    bool bad = false;
+#pragma unroll
+                    for (int p = 0; p < 16; ++p) bad |= (u[p] >> 23) == 0xFFu;
+                    if (bad) status |= kDevNonFinite;
+                    k |= (uint32_t)exact_2_4(u, DT == kBF16 ? 16 : 0) << (16 * b);
+                }
+            } else {
+            front_end<DT, kRows>(stage + h * G::kHalfBytes, lane, rel, worst, nonzero);
             if constexpr (kRows) {
                 // N of 4 along rows: kept iff fewer than N entries of the row are heavier
                 const int nk = n_keep;
@@ -333,6 +362,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                 viol += (unsigned)__popc(~k & nonzero & in_cols);
             } else {
                 k = cover_2_4(rel);
+            }
             }
             if constexpr (METHOD == kMethodApprox) {
                 LineFill f = line_fill(k);
@@ -472,12 +502,14 @@ size_t tma_entry_bytes() { return sizeof(TmaEntry); }
 int tma_warps_per_cta(int dtype, int M, int method) {
     if (M == 8) return tma48_warps_per_cta(dtype, method);
     const bool heavy = method == kMethodApprox || method == kMethodRowsAbsorb;
+    if (method == kMethodExact) return dtype == kF32 ? Geometry<kF32, kMethodExact>::kWarps : Geometry<kBF16, kMethodExact>::kWarps;
     if (dtype == kF32) return heavy ? Geometry<kF32, kMethodApprox>::kWarps : Geometry<kF32, kMethodCover>::kWarps;
     return heavy ? Geometry<kBF16, kMethodApprox>::kWarps : Geometry<kBF16, kMethodCover>::kWarps;
 }
 
 bool tma_eligible(const DevProblem& p, int N, int M, int method) {
     if (method == kMethodRows || method == kMethodRowsAbsorb) { if (M != 4 || N < 1 || N > 3) return false; }
+    else if (method == kMethodExact) { if (N != 2 || M != 4) return false; }
     else if (!((N == 2 && M == 4) || (N == 4 && M == 8)) || (method != kMethodApprox && method != kMethodCover)) return false;
     const size_t elem = p.dtype == kF32 ? 4 : 2;
     if ((uintptr_t)p.W % 16 || ((size_t)p.ld * elem) % 16) return false;
@@ -511,8 +543,8 @@ cudaError_t launch_tma(const TmaLaunch& a) {
     if (a.total_items > 0) {
 #define TM_DISPATCH(DT, METHOD)                                                                                   \
     err = a.has_out ? launch_one<DT, METHOD, true>(a, host[0], table) : launch_one<DT, METHOD, false>(a, host[0], table)
-        if (a.dtype == kF32) { if (a.method == kMethodApprox) TM_DISPATCH(kF32, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kF32, kMethodRows); else if (a.method == kMethodRowsAbsorb) TM_DISPATCH(kF32, kMethodRowsAbsorb); else TM_DISPATCH(kF32, kMethodCover); }
-        else { if (a.method == kMethodApprox) TM_DISPATCH(kBF16, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kBF16, kMethodRows); else if (a.method == kMethodRowsAbsorb) TM_DISPATCH(kBF16, kMethodRowsAbsorb); else TM_DISPATCH(kBF16, kMethodCover); }
+        if (a.dtype == kF32) { if (a.method == kMethodExact) TM_DISPATCH(kF32, kMethodExact); else if (a.method == kMethodApprox) TM_DISPATCH(kF32, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kF32, kMethodRows); else if (a.method == kMethodRowsAbsorb) TM_DISPATCH(kF32, kMethodRowsAbsorb); else TM_DISPATCH(kF32, kMethodCover); }
+        else { if (a.method == kMethodExact) TM_DISPATCH(kBF16, kMethodExact); else if (a.method == kMethodApprox) TM_DISPATCH(kBF16, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kBF16, kMethodRows); else if (a.method == kMethodRowsAbsorb) TM_DISPATCH(kBF16, kMethodRowsAbsorb); else TM_DISPATCH(kBF16, kMethodCover); }
 #undef TM_DISPATCH
         if (err != cudaSuccess) return err;
     }

@@ -260,8 +260,8 @@ __device__ __forceinline__ uint64_t exact_2_4_scored(const uint32_t (&u)[16], in
     return best_code;
 }
 
-__device__ __noinline__ uint64_t exact_2_4_wide(const uint32_t (&u)[16], int Emin) { return exact_2_4_scored<Wide>(u, Emin); }
-__device__ __noinline__ uint64_t exact_2_4_int64(const uint32_t (&u)[16], int Emin) { return exact_2_4_scored<long long>(u, Emin); }
+static __device__ __noinline__ uint64_t exact_2_4_wide(const uint32_t (&u)[16], int Emin) { return exact_2_4_scored<Wide>(u, Emin); }
+static __device__ __noinline__ uint64_t exact_2_4_int64(const uint32_t (&u)[16], int Emin) { return exact_2_4_scored<long long>(u, Emin); }
 
 // Fast scorer.  A row keeps one of six column pairs {a,b} (index b(b-1)/2 + a, the order of
 // kRowChoice).  value(row i, pair) = (q_a + q_b) * 2^16 + (nibble << 4i): the mask code rides in the
