@@ -259,6 +259,13 @@ hamming_reduce_kernel(const unsigned long long* __restrict__ partials, int n, un
 // run of 64 values (128 bytes of bf16) written with 16-byte stores, and its four metadata words in one go.
 // Shared tile: the kept pair of (column c, block row br) at word ((c & 3) * 32 + (c >> 2)) * pitch + br * kVW:
 // lanes of a warp (columns four apart) fall into different banks.
+// Metadata nibble idx0 | idx1 << 2 of a keep nibble with exactly two bits set (never zero), 0 for any other nibble:
+// sixteen 4-bit entries in one 64-bit word.
+__device__ __forceinline__ uint32_t pair_nibble(uint32_t m) {
+    constexpr unsigned long long kTable = (4ull << 12) | (8ull << 20) | (9ull << 24) | (12ull << 36) | (13ull << 40) | (14ull << 48);
+    return (uint32_t)(kTable >> (4 * m)) & 0xFu;
+}
+
 template <int DT>
 __global__ void __launch_bounds__(256)
 compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __restrict__ meta, void* __restrict__ values_t,
@@ -278,7 +285,7 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
         const long long c0 = tc * 128 + lane * 4;
         for (int k = threadIdx.x; k < 128 * 4; k += 256) (&tile_mt[0][0])[k] = 0;
         __syncthreads();
-#pragma unroll 1
+#pragma unroll
         for (int it = 0; it < 4; ++it) {
             const int br = it * 8 + warp;                // block row inside the tile
             const long long r0 = tr * 128 + br * 4;
@@ -302,12 +309,12 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint32_t m = (mbits >> (4 * i)) & 0xFu;
-                uint32_t a = 0, b = 0, nib = 0;
-                if (__popc(m) == 2) {
-                    const int i0 = __ffs(m) - 1, i1 = 31 - __clz(m);
+                uint32_t a = 0, b = 0;
+                const uint32_t nib = pair_nibble(m);
+                if (nib) {
+                    const int i0 = nib & 3, i1 = nib >> 2;
                     a = i0 == 0 ? v[i][0] : (i0 == 1 ? v[i][1] : v[i][2]);
                     b = i1 == 1 ? v[i][1] : (i1 == 2 ? v[i][2] : v[i][3]);
-                    nib = (uint32_t)(i0 | (i1 << 2));
                 } else if (active) bad = true;
                 row_nibbles |= nib << (4 * i);
                 if (active) {
@@ -325,12 +332,12 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const uint32_t m = ((mbits >> j) & 1u) | (((mbits >> (4 + j)) & 1u) << 1) | (((mbits >> (8 + j)) & 1u) << 2) | (((mbits >> (12 + j)) & 1u) << 3);
-                uint32_t a = 0, b = 0, nib = 0;
-                if (__popc(m) == 2) {
-                    const int i0 = __ffs(m) - 1, i1 = 31 - __clz(m);
+                uint32_t a = 0, b = 0;
+                const uint32_t nib = pair_nibble(m);
+                if (nib) {
+                    const int i0 = nib & 3, i1 = nib >> 2;
                     a = i0 == 0 ? v[0][j] : (i0 == 1 ? v[1][j] : v[2][j]);
                     b = i1 == 1 ? v[1][j] : (i1 == 2 ? v[2][j] : v[3][j]);
-                    nib = (uint32_t)(i0 | (i1 << 2));
                 } else if (active) bad = true;
                 uint32_t* slot = tile_t + (j * 32 + lane) * kPitch + br * kVW;
                 if constexpr (DT == kF32) { slot[0] = a; slot[1] = b; } else slot[0] = a | (b << 16);
