@@ -18,6 +18,20 @@ struct alignas(128) TmaEntry {
 };
 static_assert(sizeof(TmaEntry) == 384 || sizeof(TmaEntry) == 512, "descriptor records stay 128-byte aligned in tables");
 
+// The matrix that holds work item `item`: the last record whose first item is not beyond it (first items never
+// decrease along the table).  Called by all 32 lanes of a warp with the same arguments: every lane tests its own
+// records, so a table of a hundred matrices costs three independent loads per lane instead of a hundred dependent ones.
+__device__ __forceinline__ int find_matrix(const TmaEntry* tab, int count, long long item) {
+    const int lane = threadIdx.x & 31;
+    int n = 0;
+    for (int base = 1; base < count; base += 32) {
+        const int k = base + lane;
+        const bool reached = k < count && tab[k].p.item_begin <= item;
+        n += __popc(__ballot_sync(0xFFFFFFFFu, reached));
+    }
+    return n;
+}
+
 // Walks the work items of a table of problems in order: problem k, block row bi, column chunk cj.
 struct Cursor {
     int k, bi, cj, cchunks, brows;
@@ -26,8 +40,7 @@ struct Cursor {
         if (k < count) { cchunks = tab[k].cchunks; brows = tab[k].brows; } else { cchunks = 1; brows = 1; }
     }
     __device__ __forceinline__ void seek(const TmaEntry* tab, int count, long long item) {
-        k = 0;
-        while (k + 1 < count && tab[k + 1].p.item_begin <= item) ++k;
+        k = find_matrix(tab, count, item);
         load(tab, count);
         const long long local = item - tab[k < count ? k : count - 1].p.item_begin;
         bi = (int)(local / cchunks); cj = (int)(local - (long long)bi * cchunks);
@@ -52,8 +65,7 @@ struct StrideCursor {
     }
     __device__ __forceinline__ void seek(const TmaEntry* tab, int count, long long item, int stride_) {
         stride = stride_;
-        k = 0;
-        while (k + 1 < count && tab[k + 1].p.item_begin <= item) ++k;
+        k = find_matrix(tab, count, item);
         enter(tab, count);
         const long long local = item - tab[k < count ? k : count - 1].p.item_begin;
         bi = (int)(local / cchunks); cj = (int)(local - (long long)bi * cchunks);
