@@ -109,6 +109,14 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
     constexpr int kLanesPerWord = 32 / M;          // lanes whose blocks share one mask word
     constexpr int kWordsPerItem = M;               // 32 blocks * M columns / 32 bits
 
+    if (begin < end) {          // the warp's first problem: every lane tests its own table entries (independent loads)
+        int n = 0;
+        for (int base = 1; base < count; base += 32) {
+            const int q = base + lane;
+            n += __popc(__ballot_sync(0xFFFFFFFFu, q < count && tab[q].item_begin <= begin));
+        }
+        k = n;
+    }
     for (long long item = begin; item < end; ++item) {
         const DevProblem& P = find_problem(tab, count, item, k);
         if (k != acc_k) {
