@@ -109,6 +109,19 @@ TM_HD uint32_t fill_accept(const Rel24& r, uint32_t kept, uint32_t cand) {
     return cand & ~(row_blocked | col_blocked);
 }
 
+// The candidates of blocks that have exactly one: such a candidate has no rival in its row or column, so the scan
+// takes it as it stands (and the block has none left afterwards).
+TM_HD uint32_t lone_candidates(uint32_t cand) {
+#if defined(__CUDA_ARCH__)
+    uint32_t less_one;
+    asm("add.u16x2 %0, %1, %2;" : "=r"(less_one) : "r"(cand), "r"(0xFFFFFFFFu));      // cand - 1 in either half
+#else
+    const uint32_t less_one = ((cand - 1u) & 0xFFFFu) | ((cand - 0x10000u) & 0xFFFF0000u);
+#endif
+    const uint32_t several = cand & less_one;                          // a half is non-zero iff it holds two or more
+    return cand & (((several & 0xFFFFu) ? 0u : 0xFFFFu) | ((several >> 16) ? 0u : 0xFFFF0000u));
+}
+
 // Steps A and B for one pair of blocks, without cross-lane votes (host tests, simple kernels).
 TM_HD uint32_t cover_and_fill_2_4(const Rel24& r, LineFill& f) {
     uint32_t kept = cover_2_4(r);
