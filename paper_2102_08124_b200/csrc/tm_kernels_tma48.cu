@@ -325,6 +325,13 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             int rounds = 0;
             while (__any_sync(0xFFFFFFFFu, cand != 0)) {
                 if (++rounds > 16) { status |= kDevInternal; break; }      // a block lacks at most sixteen entries
+                if (rounds == 4) {      // after three rounds a block that still has candidates has, as a rule, exactly one: it has
+                                        // no rival in its row or column and is taken as it stands
+                    if ((cand & (cand - 1)) == 0) kept |= cand;
+                    L = line_short(kept);
+                    cand = open_candidates8(kept, L);
+                    if (!__any_sync(0xFFFFFFFFu, cand != 0)) break;
+                }
                 kept |= fill_accept8(rel, kept, cand);
                 L = line_short(kept);
                 cand = open_candidates8(kept, L);
