@@ -274,6 +274,14 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
     constexpr int kPitch = 32 * kVW + 1;
     __shared__ uint32_t tile_t[128 * kPitch];
     __shared__ uint32_t tile_mt[128][4];                // transposed metadata words of every column (32 rows each)
+    // bf16: the kept pair of four 16-bit values held in two words leaves with one byte permute; entry m of the table is
+    // that permute's selector for keep nibble m (halfwords idx0, idx1) with the metadata nibble above it, 0 for a nibble
+    // that does not keep exactly two
+    __shared__ uint32_t pair_tab[16];
+    if (threadIdx.x < 16) {
+        const uint32_t nib = pair_nibble(threadIdx.x), i0 = nib & 3u, i1 = nib >> 2;
+        pair_tab[threadIdx.x] = nib ? ((2 * i0) | ((2 * i0 + 1) << 4) | ((2 * i1) << 8) | ((2 * i1 + 1) << 12) | (nib << 16)) : 0u;
+    }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long tiles_c = (P.cols + 127) / 128, tiles_r = (P.rows + 127) / 128;
     const long long wpr_t = (P.rows + 31) / 32, half_c = P.cols / 2, half_r = P.rows / 2;
@@ -291,6 +299,7 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
             const long long r0 = tr * 128 + br * 4;
             const bool active = r0 < P.rows && c0 < P.cols;
             uint32_t v[4][4] = {}, mbits = 0;            // mbits bit 4i+j = mask of (row i, column j)
+            uint2 raw[4] = {};                           // bf16: the row's four values as loaded
             if (active) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
@@ -298,8 +307,7 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
                         const uint4 a = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(P.W) + (r0 + i) * P.ld + c0));
                         v[i][0] = a.x; v[i][1] = a.y; v[i][2] = a.z; v[i][3] = a.w;
                     } else {
-                        const uint2 a = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(P.W) + (r0 + i) * P.ld + c0));
-                        v[i][0] = a.x & 0xFFFFu; v[i][1] = a.x >> 16; v[i][2] = a.y & 0xFFFFu; v[i][3] = a.y >> 16;
+                        raw[i] = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(P.W) + (r0 + i) * P.ld + c0));
                     }
                     mbits |= ((__ldg(P.mask + (r0 + i) * P.wpr + (c0 >> 5)) >> (c0 & 31)) & 0xFu) << (4 * i);
                 }
@@ -309,18 +317,24 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const uint32_t m = (mbits >> (4 * i)) & 0xFu;
-                uint32_t a = 0, b = 0;
-                const uint32_t nib = pair_nibble(m);
-                if (nib) {
-                    const int i0 = nib & 3, i1 = nib >> 2;
-                    a = i0 == 0 ? v[i][0] : (i0 == 1 ? v[i][1] : v[i][2]);
-                    b = i1 == 1 ? v[i][1] : (i1 == 2 ? v[i][2] : v[i][3]);
-                } else if (active) bad = true;
-                row_nibbles |= nib << (4 * i);
-                if (active) {
-                    if constexpr (DT == kF32) *reinterpret_cast<uint2*>(reinterpret_cast<uint32_t*>(values) + (r0 + i) * half_c + (c0 >> 1)) = make_uint2(a, b);
-                    else *reinterpret_cast<uint32_t*>(reinterpret_cast<uint16_t*>(values) + (r0 + i) * half_c + (c0 >> 1)) = a | (b << 16);
+                uint32_t nib;
+                if constexpr (DT == kF32) {
+                    uint32_t a = 0, b = 0;
+                    nib = pair_nibble(m);
+                    if (nib) {
+                        const int i0 = nib & 3, i1 = nib >> 2;
+                        a = i0 == 0 ? v[i][0] : (i0 == 1 ? v[i][1] : v[i][2]);
+                        b = i1 == 1 ? v[i][1] : (i1 == 2 ? v[i][2] : v[i][3]);
+                    }
+                    if (active) *reinterpret_cast<uint2*>(reinterpret_cast<uint32_t*>(values) + (r0 + i) * half_c + (c0 >> 1)) = make_uint2(a, b);
+                } else {
+                    const uint32_t e = pair_tab[m];
+                    nib = e >> 16;
+                    const uint32_t pair = nib ? __byte_perm(raw[i].x, raw[i].y, e) : 0u;
+                    if (active) *reinterpret_cast<uint32_t*>(reinterpret_cast<uint16_t*>(values) + (r0 + i) * half_c + (c0 >> 1)) = pair;
                 }
+                if (!nib && active) bad = true;
+                row_nibbles |= nib << (4 * i);
             }
 #pragma unroll
             for (int i = 0; i < 4; ++i) {                // eight lanes share a metadata word of a row
@@ -331,16 +345,29 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
             // column form into the shared tile
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const uint32_t m = ((mbits >> j) & 1u) | (((mbits >> (4 + j)) & 1u) << 1) | (((mbits >> (8 + j)) & 1u) << 2) | (((mbits >> (12 + j)) & 1u) << 3);
-                uint32_t a = 0, b = 0;
-                const uint32_t nib = pair_nibble(m);
-                if (nib) {
-                    const int i0 = nib & 3, i1 = nib >> 2;
-                    a = i0 == 0 ? v[0][j] : (i0 == 1 ? v[1][j] : v[2][j]);
-                    b = i1 == 1 ? v[1][j] : (i1 == 2 ? v[2][j] : v[3][j]);
-                } else if (active) bad = true;
+                // bit j of the four row nibbles, gathered by a multiplication (bits 0, 4, 8, 12 land on 9, 10, 11, 12)
+                const uint32_t m = ((((mbits >> j) & 0x1111u) * 0x249u) >> 9) & 0xFu;
                 uint32_t* slot = tile_t + (j * 32 + lane) * kPitch + br * kVW;
-                if constexpr (DT == kF32) { slot[0] = a; slot[1] = b; } else slot[0] = a | (b << 16);
+                uint32_t nib;
+                if constexpr (DT == kF32) {
+                    uint32_t a = 0, b = 0;
+                    nib = pair_nibble(m);
+                    if (nib) {
+                        const int i0 = nib & 3, i1 = nib >> 2;
+                        a = i0 == 0 ? v[0][j] : (i0 == 1 ? v[1][j] : v[2][j]);
+                        b = i1 == 1 ? v[1][j] : (i1 == 2 ? v[2][j] : v[3][j]);
+                    }
+                    slot[0] = a; slot[1] = b;
+                } else {
+                    // the column's four values as two words (rows 0,1 and rows 2,3), then the same table
+                    const uint32_t sel = (j & 1) ? 0x7632u : 0x5410u;
+                    const uint32_t c01 = j < 2 ? __byte_perm(raw[0].x, raw[1].x, sel) : __byte_perm(raw[0].y, raw[1].y, sel);
+                    const uint32_t c23 = j < 2 ? __byte_perm(raw[2].x, raw[3].x, sel) : __byte_perm(raw[2].y, raw[3].y, sel);
+                    const uint32_t e = pair_tab[m];
+                    nib = e >> 16;
+                    slot[0] = nib ? __byte_perm(c01, c23, e) : 0u;
+                }
+                if (!nib && active) bad = true;
                 if (nib) atomicOr(&tile_mt[lane * 4 + j][it], nib << (4 * warp));
             }
         }
