@@ -253,7 +253,7 @@ hamming_reduce_kernel(const unsigned long long* __restrict__ partials, int n, un
 }
 
 // ---- 2:4 compression ---------------------------------------------------------------------------
-// CTA tile: 128 rows x 128 columns = 32 x 32 blocks of 4x4; a warp takes block rows w, w+8, w+16, w+24 of the
+// CTA tile: 128 rows x 128 columns = 32 x 32 blocks of 4x4; a warp takes block rows 4w .. 4w+3 of the
 // tile, lane = block column.  The row form (values, meta) is written straight from registers, 128 bytes per
 // row and warp.  The column form is collected in shared memory so that every column of the tile leaves as one
 // run of 64 values (128 bytes of bf16) written with 16-byte stores, and its four metadata words in one go.
@@ -273,7 +273,9 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
     constexpr int kVW = DT == kF32 ? 2 : 1;             // words per kept pair
     constexpr int kPitch = 32 * kVW + 1;
     __shared__ uint32_t tile_t[128 * kPitch];
-    __shared__ uint32_t tile_mt[128][4];                // transposed metadata words of every column (32 rows each)
+    // transposed metadata: word k (block rows 8k .. 8k+7) of column 4*lane + j at [k][j][lane]; a warp owns one 16-bit
+    // half of its words (its four block rows), so no two warps ever write the same bytes
+    __shared__ uint32_t tile_mt[4][4][32];
     // bf16: the kept pair of four 16-bit values held in two words leaves with one byte permute; entry m of the table is
     // that permute's selector for keep nibble m (halfwords idx0, idx1) with the metadata nibble above it, 0 for a nibble
     // that does not keep exactly two
@@ -282,6 +284,7 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
         const uint32_t nib = pair_nibble(threadIdx.x), i0 = nib & 3u, i1 = nib >> 2;
         pair_tab[threadIdx.x] = nib ? ((2 * i0) | ((2 * i0 + 1) << 4) | ((2 * i1) << 8) | ((2 * i1 + 1) << 12) | (nib << 16)) : 0u;
     }
+    __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long tiles_c = (P.cols + 127) / 128, tiles_r = (P.rows + 127) / 128;
     const long long wpr_t = (P.rows + 31) / 32, half_c = P.cols / 2, half_r = P.rows / 2;
@@ -291,11 +294,10 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
     for (long long t = blockIdx.x; t < tiles_r * tiles_c; t += gridDim.x) {
         const long long tr = t / tiles_c, tc = t - tr * tiles_c;
         const long long c0 = tc * 128 + lane * 4;
-        for (int k = threadIdx.x; k < 128 * 4; k += 256) (&tile_mt[0][0])[k] = 0;
-        __syncthreads();
+        uint32_t col_nibbles[4] = {0, 0, 0, 0};      // nibble `it` = metadata of column j in block row 4 * warp + it
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
-            const int br = it * 8 + warp;                // block row inside the tile
+            const int br = warp * 4 + it;                // block row inside the tile
             const long long r0 = tr * 128 + br * 4;
             const bool active = r0 < P.rows && c0 < P.cols;
             uint32_t v[4][4] = {}, mbits = 0;            // mbits bit 4i+j = mask of (row i, column j)
@@ -368,9 +370,12 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
                     slot[0] = nib ? __byte_perm(c01, c23, e) : 0u;
                 }
                 if (!nib && active) bad = true;
-                if (nib) atomicOr(&tile_mt[lane * 4 + j][it], nib << (4 * warp));
+                col_nibbles[j] |= nib << (4 * it);
             }
         }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            reinterpret_cast<unsigned short*>(&tile_mt[warp >> 1][j][lane])[warp & 1] = (unsigned short)col_nibbles[j];
         __syncthreads();
         {   // 128 columns: two threads per column, each half of its 64 values and two of its four metadata words
             const int c = threadIdx.x >> 1, h = threadIdx.x & 1;
@@ -389,7 +394,7 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
                 }
 #pragma unroll
                 for (int k = 0; k < 2; ++k)
-                    if (tr * 4 + h * 2 + k < wpr_t) meta_t[col * wpr_t + tr * 4 + h * 2 + k] = tile_mt[c][h * 2 + k];
+                    if (tr * 4 + h * 2 + k < wpr_t) meta_t[col * wpr_t + tr * 4 + h * 2 + k] = tile_mt[h * 2 + k][c & 3][c >> 2];
             }
         }
         __syncthreads();
