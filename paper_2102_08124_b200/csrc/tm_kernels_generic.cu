@@ -92,9 +92,11 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
     const int lane = threadIdx.x & 31;
     const long long gw = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
     const long long nwarps = (long long)gridDim.x * kWarpsPerCta;
-    const long long per = (total_items + nwarps - 1) / nwarps;
-    const long long begin = gw * per;
-    const long long end = min(total_items, begin + per);
+    // even split: total / nwarps items each, the first warps one more
+    const long long order = gw;
+    const long long share = total_items / nwarps, surplus = total_items - share * nwarps;
+    const long long begin = order * share + (order < surplus ? order : surplus);
+    const long long end = begin + share + (order < surplus ? 1 : 0);
     const DevProblem* tab = table ? table : &single;
 
     // per-thread columns of the flow solver's state (only the exact instantiations that use it get dynamic shared memory)

@@ -260,14 +260,18 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
 
     const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
     // A fixed deal of the items, so the objective's partial sums are reproducible.  Where the kernel waits for memory
-    // (Algorithm 1 alone, the 1-D pruning) the warps take the items round-robin -- gw, gw + nwarps, ... -- so that the
+    // (Algorithm 1 alone, the 1-D pruning) the warps take the items round-robin -- first, first + nwarps, ... -- so that the
     // whole grid works on one dense window of the matrix (3 % faster there); the full search, which also waits for the
     // integer pipe, is indifferent to the order and 2 % faster with the plain cursor of a contiguous range.
     constexpr bool kRoundRobin = !G::kHeavy;
-    const long long per = (total_items + nwarps - 1) / nwarps;
-    const long long first = kRoundRobin ? gw : gw * per;
-    const int n_items = kRoundRobin ? (gw < total_items ? (int)((total_items - gw + nwarps - 1) / nwarps) : 0)
-                                    : (int)max(0ll, min(total_items, first + per) - first);
+    int n_items;
+    long long first;
+    if constexpr (kRoundRobin) {       // the same order as even_share(): surplus items fall on different SMs
+        first = (long long)warp * gridDim.x + blockIdx.x;
+        n_items = first < total_items ? (int)((total_items - first + nwarps - 1) / nwarps) : 0;
+    } else {
+        first = even_share(total_items, G::kWarps, n_items);
+    }
     const TmaEntry* tab = table ? table : &single;
 
     if (lane == 0) {

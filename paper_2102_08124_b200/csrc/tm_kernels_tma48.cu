@@ -254,9 +254,8 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     }
 
     const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
-    const long long per = (total_items + nwarps - 1) / nwarps;
-    const long long begin = gw * per, end = min(total_items, begin + per);
-    const int n_items = (int)max(0ll, end - begin);
+    int n_items;
+    const long long begin = even_share(total_items, G::kWarps, n_items);
     const TmaEntry* tab = table ? table : &single;
 
     if (lane == 0) {

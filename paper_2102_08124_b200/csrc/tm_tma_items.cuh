@@ -18,6 +18,18 @@ struct alignas(128) TmaEntry {
 };
 static_assert(sizeof(TmaEntry) == 384 || sizeof(TmaEntry) == 512, "descriptor records stay 128-byte aligned in tables");
 
+// Even split of `total` work items over the warps of the grid: every warp gets total / nwarps items and the first
+// total % nwarps warps one more -- "first" in an order that runs across the CTAs before it runs down their warps, so
+// that the surplus items fall on as many different SMs as possible (an SM's warps share its issue slots: what counts
+// is the SM's total).  Returns the warp's first item and sets its item count.
+__device__ __forceinline__ long long even_share(long long total, int warps_per_cta, int& n_items) {
+    const long long nwarps = (long long)gridDim.x * warps_per_cta;
+    const long long order = (long long)(threadIdx.x >> 5) * gridDim.x + blockIdx.x;
+    const long long q = total / nwarps, rem = total - q * nwarps;
+    n_items = (int)(q + (order < rem ? 1 : 0));
+    return order * q + (order < rem ? order : rem);
+}
+
 // The matrix that holds work item `item`: the last record whose first item is not beyond it (first items never
 // decrease along the table).  Called by all 32 lanes of a warp with the same arguments: every lane tests its own
 // records, so a table of a hundred matrices costs three independent loads per lane instead of a hundred dependent ones.
