@@ -127,6 +127,30 @@ def test_exact_2_4_bf16_narrow_blocks_take_the_32_bit_scorer():
     assert_parity(V, 2, 4, tm.TM_EXACT)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_exact_2_4_on_the_bandwidth_kernel(dtype):
+    """16-byte aligned matrices take the staged kernel for the exact 2:4 search too: several 512-column items and a ragged
+    last one, mask only, in place, and (bf16) Inf and NaN patterns, which the scorer must order by bit pattern."""
+    rows, cols = 44, 1336 if dtype == "f32" else 1336 + 8
+    W = workloads.normal_f32(rows, cols, 0.02, 71) if dtype == "f32" else workloads.normal_bf16(rows, cols, 0.02, 71)
+    assert_parity(W, 2, 4, tm.TM_EXACT)
+    want = orc.find_mask(W, 2, 4, orc.EXACT)
+    got = gpu_find_mask(W, 2, 4, tm.TM_EXACT, want_masked=False, want_objective=False)
+    assert got["masked"] is None and np.array_equal(got["mask"], want["mask"])
+    Wd = to_device(W)
+    fn = tm.tm_find_mask_bf16 if dtype == "bf16" else tm.tm_find_mask
+    mask, masked, obj = fn(Wd, 2, 4, tm.TM_EXACT, masked_w_out=Wd)        # in place
+    torch.cuda.synchronize()
+    assert np.array_equal(to_host_bits(Wd), want["masked"].view(np.uint16 if dtype == "bf16" else np.uint32))
+    assert np.array_equal(to_host_bits(mask), want["mask"])
+    V = W.copy()
+    if dtype == "bf16":
+        V[1, 3] = 0x7F80; V[2, 5] = 0xFF80; V[5, 28] = 0x7FC0; V[5, 29] = 0x7F81; V[6, 29] = 0xFFFF; V[43, cols - 2] = 0x7FA0
+    else:
+        V[1, 3] = np.inf; V[5, 28] = np.nan; V[43, cols - 2] = -np.inf
+    assert_parity(V, 2, 4, tm.TM_EXACT, rel=None)
+
+
 @pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
 def test_optional_outputs_and_in_place(N, M):
     W = workloads.normal_f32(4 * M, 45 * M, 0.02, 13)
