@@ -126,9 +126,14 @@ int build_plan(const tm_problem* probs, int count, int N, int M, int method, voi
 
     // group 0: generic; groups 1..4: bandwidth path by (dtype, masked output present)
     std::vector<DevProblem> group[5];
+    // A lane of the staged kernel scores its four blocks of an item one after the other: a small exact call is spread
+    // wider, and finished sooner, by the generic kernel (one block per lane).
+    long long call_weights = 0;
+    for (int k = 0; k < count; ++k) call_weights += (long long)probs[k].rows * probs[k].cols;
+    const bool staged = !(method == TM_EXACT && call_weights < (1ll << 20));
     for (int k = 0; k < count; ++k) {
         DevProblem d = to_dev(probs[k], M, 0);
-        const int g = tmask::tma_eligible(d, N, M, method) ? 1 + 2 * d.dtype + (d.masked ? 1 : 0) : 0;
+        const int g = staged && tmask::tma_eligible(d, N, M, method) ? 1 + 2 * d.dtype + (d.masked ? 1 : 0) : 0;
         group[g].push_back(d);
     }
     int used = 0;

@@ -131,7 +131,7 @@ def test_exact_2_4_bf16_narrow_blocks_take_the_32_bit_scorer():
 def test_exact_2_4_on_the_bandwidth_kernel(dtype):
     """16-byte aligned matrices take the staged kernel for the exact 2:4 search too: several 512-column items and a ragged
     last one, mask only, in place, and (bf16) Inf and NaN patterns, which the scorer must order by bit pattern."""
-    rows, cols = 44, 1336 if dtype == "f32" else 1336 + 8
+    rows, cols = 204, 5144 if dtype == "f32" else 5144 + 8             # above a million weights: smaller exact calls stay on the generic kernel
     W = workloads.normal_f32(rows, cols, 0.02, 71) if dtype == "f32" else workloads.normal_bf16(rows, cols, 0.02, 71)
     assert_parity(W, 2, 4, tm.TM_EXACT)
     want = orc.find_mask(W, 2, 4, orc.EXACT)
