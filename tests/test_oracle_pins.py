@@ -355,6 +355,56 @@ def test_completion_invariants(N, M, kind):
         assert saw_swap
 
 
+@pytest.mark.parametrize("N,M,kind", [(2, 4, "normal"), (2, 4, "ties"), (4, 8, "laplace"), (4, 8, "ties"), (3, 6, "ties"), (1, 4, "ties")])
+def test_step_b_is_the_heavy_to_light_greedy_fill(N, M, kind):
+    """Step B checked as a certificate, without running it again: an entry outside Algorithm 1's kept set is taken by the
+    fill exactly when, counting that kept set and the taken entries heavier than it, its row and its column both still hold
+    fewer than N.  By induction from the heaviest entry down, only one set satisfies this for every entry."""
+    for block in rand_blocks(300, M, 95 + M, kind):
+        r = orc.block_approx(block, N, M)
+        A, B = r["after_a"].astype(bool), r["after_b"].astype(bool)
+        mag = np.abs(block.astype(np.float64))
+        filled = B & ~A
+        for i in range(M):
+            for j in range(M):
+                if A[i, j]:
+                    continue
+                p = i * M + j
+                heavier = np.zeros((M, M), bool)
+                for q in np.flatnonzero(filled):
+                    qi, qj = divmod(int(q), M)
+                    if (mag[qi, qj], q) > (mag[i, j], p):
+                        heavier[qi, qj] = True
+                H = A | heavier
+                takes = H[i, :].sum() < N and H[:, j].sum() < N
+                assert bool(filled[i, j]) == bool(takes), (i, j)
+
+
+@pytest.mark.parametrize("N,M,kind", [(2, 4, "normal"), (2, 4, "ties"), (4, 8, "laplace"), (4, 8, "ties"), (3, 6, "ties")])
+def test_step_c_single_swap_takes_the_lightest_eligible_entry(N, M, kind):
+    """Blocks that need exactly one swap, checked against the rule itself: the entry that leaves is the lightest kept entry
+    (r', c') for which some short row is free in column c' and some short column is free in row r'; the two that enter are
+    the heaviest such free entries of column c' and of row r'."""
+    seen = 0
+    for block in rand_blocks(600, M, 97 + M, kind):
+        r = orc.block_approx(block, N, M)
+        if r["n_swap"] != 1:
+            continue
+        seen += 1
+        B, K = r["after_b"].astype(bool), r["kept"].astype(bool)
+        mag = np.abs(block.astype(np.float64))
+        key = lambda i, j: (mag[i, j], i * M + j)
+        DR = [i for i in range(M) if B[i].sum() < N]; DC = [j for j in range(M) if B[:, j].sum() < N]
+        elig = [(i, j) for i in range(M) for j in range(M) if B[i, j]
+                and any(not B[rr, j] for rr in DR) and any(not B[i, cc] for cc in DC)]
+        x = min(elig, key=lambda e: key(*e))
+        a = max(((rr, x[1]) for rr in DR if not B[rr, x[1]]), key=lambda e: key(*e))
+        b = max(((x[0], cc) for cc in DC if not B[x[0], cc]), key=lambda e: key(*e))
+        want = B.copy(); want[x] = False; want[a] = True; want[b] = True
+        assert np.array_equal(K, want)
+    assert seen > 20
+
+
 def _py_approx(block, N, M):
     """Steps A, B, C re-stated with Python sets (independent of the C code)."""
     mag = np.abs(block.astype(np.float64))
