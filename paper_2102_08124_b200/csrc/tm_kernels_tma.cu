@@ -194,7 +194,7 @@ __device__ __forceinline__ float back_end(unsigned char* stage, unsigned char* m
 // n_keep entries of every group, so the divisor is the same for the whole call.  The objective stays the sum of
 // the kept magnitudes before absorption.
 template <int DT>
-__device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned char* mrow /* [4][32] */, int lane, uint32_t kept, int n_keep) {
+__device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned char* mrow /* [4][32] */, const uint4* lut, int lane, uint32_t kept, int n_keep) {
     constexpr int kPitch = kItemCols * (DT == kF32 ? 4 : 2);
     float s4 = 0.f;
     const uint32_t mb4 = mask_bytes_2_4(kept);
@@ -203,8 +203,9 @@ __device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned 
     for (int i = 0; i < 4; ++i) {
         const uint32_t mb = (mb4 >> (8 * i)) & 0xFFu;
         uint32_t raw[8];
+        uint4 r = make_uint4(0, 0, 0, 0);
         if constexpr (DT == kBF16) {
-            const uint4 r = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 16);
+            r = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 16);
             raw[0] = r.x << 16; raw[1] = r.x & 0xFFFF0000u; raw[2] = r.y << 16; raw[3] = r.y & 0xFFFF0000u;
             raw[4] = r.z << 16; raw[5] = r.z & 0xFFFF0000u; raw[6] = r.w << 16; raw[7] = r.w & 0xFFFF0000u;
         } else {
@@ -213,6 +214,7 @@ __device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned 
             raw[0] = ra.x; raw[1] = ra.y; raw[2] = ra.z; raw[3] = ra.w; raw[4] = rb.x; raw[5] = rb.y; raw[6] = rb.z; raw[7] = rb.w;
         }
         uint32_t o[8];
+        float v8[8];
 #pragma unroll
         for (int g = 0; g < 2; ++g) {                    // block A, block B: one group of four each
             double psum = 0.0;
@@ -224,12 +226,37 @@ __device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned 
             for (int j = 0; j < 4; ++j) {
                 const bool k = (mb >> (4 * g + j)) & 1u;
                 const float v = (float)((double)__uint_as_float(raw[4 * g + j]) + mu);
-                o[4 * g + j] = k ? (DT == kF32 ? __float_as_uint(v) : float_to_bf16_bits(v)) : 0u;
-                s4 += k ? fabsf(__uint_as_float(raw[4 * g + j])) : 0.f;
+                v8[4 * g + j] = v;
+                if constexpr (DT == kF32) {
+                    o[4 * g + j] = k ? __float_as_uint(v) : 0u;
+                    s4 += k ? fabsf(__uint_as_float(raw[4 * g + j])) : 0.f;
+                }
             }
         }
         if constexpr (DT == kBF16) {
-            *reinterpret_cast<uint4*>(stage + i * kPitch + lane * 16) = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), o[4] | (o[5] << 16), o[6] | (o[7] << 16));
+            // pairs rounded to bf16 by the packed conversion (nearest even, as the oracle rounds); a NaN keeps its payload
+            // bits there, so a row that holds one takes the integer form; pruned entries are cleared by the lane masks
+            const uint4 mm = lut[mb];
+            const uint32_t rw[4] = {r.x, r.y, r.z, r.w}, m4[4] = {mm.x, mm.y, mm.z, mm.w};
+            const float chk = ((v8[0] + v8[1]) + (v8[2] + v8[3])) + ((v8[4] + v8[5]) + (v8[6] + v8[7]));
+            uint32_t pk[4];
+            if (chk == chk) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[c]) : "f"(v8[2 * c + 1]), "f"(v8[2 * c]));
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) pk[c] = float_to_bf16_bits(v8[2 * c]) | (float_to_bf16_bits(v8[2 * c + 1]) << 16);
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                pk[c] &= m4[c];
+                const uint32_t ab = abs_bf16x2(rw[c] & m4[c]);
+                unsigned short lo, hi;
+                asm("mov.b32 {%0,%1}, %2;" : "=h"(lo), "=h"(hi) : "r"(ab));
+                asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(s4) : "h"(lo));
+                asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(s4) : "h"(hi));
+            }
+            *reinterpret_cast<uint4*>(stage + i * kPitch + lane * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         } else {
             *reinterpret_cast<uint4*>(stage + i * kPitch + lane * 32) = make_uint4(o[0], o[1], o[2], o[3]);
             *reinterpret_cast<uint4*>(stage + i * kPitch + lane * 32 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
@@ -431,7 +458,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         if constexpr (METHOD == kMethodRowsAbsorb && HAS_OUT) {
 #pragma unroll
             for (int h = 0; h < kHalves; ++h)
-                facc += back_end_absorb<DT>(stage + h * G::kHalfBytes, mbytes + h * 128, lane, kbuf[h * 32 + lane] & colmask[h], n_keep);
+                facc += back_end_absorb<DT>(stage + h * G::kHalfBytes, mbytes + h * 128, lut, lane, kbuf[h * 32 + lane] & colmask[h], n_keep);
         } else {
 #pragma unroll
             for (int h = 0; h < kHalves; ++h)

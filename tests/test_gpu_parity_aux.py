@@ -70,6 +70,39 @@ def test_nm_1d_groups_of_four_edge_values(dtype, N):
             assert abs(float(obj.item()) - want["objective"]) <= 1e-6 * abs(want["objective"]) + 1e-300
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N", [1, 2, 3])
+def test_nm_1d_mean_absorption_edge_values(dtype, N):
+    """Mean absorption on the bandwidth kernel where the rounding matters: sums that land between two bf16 values or on a
+    tie, results that round up to Inf, subnormal results, zeros of both signs, and rows that hold Inf or NaN."""
+    rows, cols = 12, 1544
+    rng = np.random.Generator(np.random.PCG64(70 + N))
+    W = workloads.normal_f32(rows, cols, 0.02, 71)
+    W[rng.random(W.shape) < 0.2] = 0.0
+    W[rng.random(W.shape) < 0.05] = -0.0
+    W[:, 64:128] = rng.choice(np.array([1.0, 1.00390625, 1.0078125, -1.0, 0.99609375], np.float32), size=(rows, 64))   # one bf16 step apart
+    W[:, 128:192] = rng.choice(np.array([3.3e38, -3.3e38, 3.38e38, 1e38], np.float32), size=(rows, 64))               # sums overflow
+    W[:, 192:256] = rng.choice(np.array([1e-39, -2e-39, 9.2e-41, 1.2e-38], np.float32), size=(rows, 64))              # subnormal range
+    if dtype == "bf16":
+        W = workloads.f32_to_bf16_bits(W)
+    for nonfinite in (False, True):
+        if nonfinite:
+            if dtype == "bf16":
+                W[2, 5] = 0x7F80; W[3, 300] = 0xFFC1; W[3, 301] = 0x7FC0; W[7, 900] = 0x7F81; W[11, 1543] = 0xFF80
+            else:
+                W[2, 5] = np.inf; W[3, 300] = np.nan; W[3, 301] = -np.nan; W[11, 1543] = -np.inf
+        want = orc.nm_mask_1d(W, N, 4, absorb_mean=True)
+        mask, masked, obj, viol, status = tm.tm_nm_mask_1d(to_device(W), N, 4, absorb_mean=True)
+        torch.cuda.synchronize()
+        assert np.array_equal(to_host_bits(mask), want["mask"])
+        got, exp = to_host_bits(masked), want["masked"].view(np.uint16 if dtype == "bf16" else np.uint32)
+        # a NaN that went through the fp64 addition carries the sign and payload its processor chose: NaN must meet NaN, all else bit for bit
+        is_nan = (lambda a: (a & 0x7FFF) > 0x7F80) if dtype == "bf16" else (lambda a: (a & 0x7FFFFFFF) > 0x7F800000)
+        assert np.array_equal(is_nan(got), is_nan(exp))
+        assert np.array_equal(got[~is_nan(exp)], exp[~is_nan(exp)])
+        assert int(viol.item()) == want["violations"]
+
+
 def test_nm_1d_strided_rows_and_unaligned_pitch():
     base = to_device(_case("bf16", 12, 100, 7))                  # 200-byte pitch: rows are only 8-byte aligned
     W = base[:, :92]                                             # a strided view
