@@ -223,6 +223,36 @@ def test_batched_cover_deals_items_round_robin():
     _batched_parity(workloads.config2(), 2, 4, tm.TM_APPROX_COVER)
 
 
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_shapes_dtypes_methods_and_batches(seed):
+    """Seeded random calls: 2:4 and 4:8, every method, fp32 and bf16 in one call, one to thirty matrices of up to 300 block
+    rows and 6000 columns, values with and without ties, contiguous rows or rows inside a wider buffer."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+
+    def matrix(M, big):
+        rows = M * int(rng.integers(1, 300 if big else 40)); cols = M * int(rng.integers(1, 1500 if big else 700))
+        bf16 = rng.random() < 0.5
+        if bf16 and rng.random() < 0.7:
+            cols = 8 * max(1, cols // 8)
+        kind = int(rng.integers(0, 3))
+        if kind == 0:
+            W = workloads.normal_f32(rows, cols, 0.02, int(rng.integers(1 << 30)))
+        elif kind == 1:
+            W = (rng.integers(-3, 4, size=(rows, cols)) * 0.25).astype(np.float32)
+        else:
+            W = workloads.laplace_f32(rows, cols, 0.05, int(rng.integers(1 << 30)))
+        return workloads.f32_to_bf16_bits(W) if bf16 else W
+
+    for _ in range(24):
+        N, M = (2, 4) if rng.random() < 0.7 else (4, 8)
+        method = METHODS[int(rng.integers(0, 3))]
+        count = int(rng.choice([1, 1, 2, 5, 30]))
+        mats = [matrix(M, count <= 2 and rng.random() < 0.3) for _ in range(count)]
+        if method == tm.TM_EXACT and M == 8:
+            mats = [np.ascontiguousarray(m[: 4 * M, : 40 * M]) for m in mats]      # the flow solver is slow on the CPU side
+        _batched_parity(mats, N, M, method, strided=rng.random() < 0.3)
+
+
 def test_prepared_batch_object():
     mats = [workloads.normal_f32(32, 264, 0.05, 61), workloads.normal_bf16(16, 520, 0.02, 62)]
     batch = tm.TmBatch([to_device(m) for m in mats])
