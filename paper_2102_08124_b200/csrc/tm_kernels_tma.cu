@@ -234,8 +234,8 @@ __device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned 
             }
         }
         if constexpr (DT == kBF16) {
-            // pairs rounded to bf16 by the packed conversion (nearest even, as the oracle rounds); a NaN keeps its payload
-            // bits there, so a row that holds one takes the integer form; pruned entries are cleared by the lane masks
+            // pairs rounded to bf16 by the packed conversion (nearest even); the rounding rule of this library lets a NaN keep
+            // its payload bits, so a row that holds one takes the integer form; pruned entries are cleared by the lane masks
             const uint4 mm = lut[mb];
             const uint32_t rw[4] = {r.x, r.y, r.z, r.w}, m4[4] = {mm.x, mm.y, mm.z, mm.w};
             const float chk = ((v8[0] + v8[1]) + (v8[2] + v8[3])) + ((v8[4] + v8[5]) + (v8[6] + v8[7]));
