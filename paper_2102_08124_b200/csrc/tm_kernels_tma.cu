@@ -80,11 +80,21 @@ __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, 
         for (int i = 0; i < 4; ++i) v[i] = *reinterpret_cast<const uint4*>(stage + i * kPitch + lane * 16);
         PairKeys pk;
         interleave_keys<true>(v, pk);
-        uint32_t m[4];
+        // Inf / NaN watch.  The OR of the sixteen words can only show an all-ones exponent where some magnitude has the top
+        // exponent bit set (|w| >= 2): for ordinary weights this cheap test settles it; otherwise the packed maximum
+        // decides exactly.  `worst` stays as it is once it holds an Inf or NaN, so the warp keeps to the integer form.
+        uint32_t any_bits = worst;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) m[i] = max_u16x2(max_u16x2(pk.x[i][0], pk.x[i][1]), max_u16x2(pk.x[i][2], pk.x[i][3]));
-        worst = max_u16x2(worst, max_u16x2(max_u16x2(m[0], m[1]), max_u16x2(m[2], m[3])));
-        if (__any_sync(0xFFFFFFFFu, nonfinite_bf16x2(worst))) {        // Inf or NaN met: integer keys, bit-pattern order
+        for (int i = 0; i < 4; ++i) any_bits |= (pk.x[i][0] | pk.x[i][1]) | (pk.x[i][2] | pk.x[i][3]);
+        bool integer_form = false;
+        if (__any_sync(0xFFFFFFFFu, nonfinite_bf16x2(any_bits))) {
+            uint32_t m[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) m[i] = max_u16x2(max_u16x2(pk.x[i][0], pk.x[i][1]), max_u16x2(pk.x[i][2], pk.x[i][3]));
+            worst = max_u16x2(worst, max_u16x2(max_u16x2(m[0], m[1]), max_u16x2(m[2], m[3])));
+            integer_form = __any_sync(0xFFFFFFFFu, nonfinite_bf16x2(worst));
+        }
+        if (integer_form) {                                            // Inf or NaN met: integer keys, bit-pattern order
             interleave_keys<false>(v, pk);
             relations_bf16<false>(pk, rel);
         }
