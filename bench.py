@@ -33,7 +33,7 @@ ROWS = FULL_ROWS
 N_KEEP, M_BLOCK = 2, 4
 BYTES_PER_WEIGHT = 2 + 2 + 1.0 / 8          # read W, write masked W, write one mask bit (bf16)
 # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture on the 2048-row case (see profiles/), per weight
-TRAFFIC_PER_WEIGHT = (201.43e6 + 162.05e6) / (2048 * 49152)
+TRAFFIC_PER_WEIGHT = (201.40e6 + 162.26e6) / (2048 * 49152)
 TRAFFIC_SOURCE = "ncu --set full on the 2048 x 49152 case, scaled by rows (profiles/tma24_kernel_approx_2_4_bf16_2048x49152_full.md)"
 METRIC = "transposable-mask weights/s (2:4 approx, bf16, 1 GPU: achieved HBM GB/s vs peak in `roofline`)"
 WORKLOAD = "%dx49152 bf16, N(0,0.02) quantised to 256 levels (frequent ties), 2:4 approximate, per-step recompute"
