@@ -130,10 +130,19 @@ __device__ __forceinline__ void front_end(const unsigned char* stage, int lane, 
                 const uint32_t e = k[i], f = k[4 + i], g = k[8 + i], hh = k[12 + i];
                 rel.hc1 |= ((f >= e ? 0x1u : 0u) | (g >= f ? 0x10u : 0u) | (hh >= g ? 0x100u : 0u) | (e > hh ? 0x1000u : 0u)) << (i + shift);
                 rel.hc2 |= ((g >= e ? 0x1u : 0u) | (hh >= f ? 0x10u : 0u)) << (i + shift);
-                worst = max(worst, max(max(a, b), max(c, d)));
             }
         }
         complete_relations(rel);
+        {   // Inf / NaN watch (for the status flag): the OR of the magnitudes shows an all-ones exponent only if some
+            // |w| >= 2; the exact maximum is taken only then
+            uint32_t any_bits = 0;
+#pragma unroll
+            for (int p = 0; p < 16; ++p) any_bits |= ka[p] | kb[p];
+            if (any_bits >= 0x7F800000u) {
+#pragma unroll
+                for (int p = 0; p < 16; ++p) worst = max(worst, max(ka[p], kb[p]));
+            }
+        }
         if constexpr (NZ) {
             nonzero = 0;
 #pragma unroll
