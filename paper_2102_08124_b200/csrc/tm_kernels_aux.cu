@@ -187,11 +187,12 @@ violations_stream_kernel(const AuxProblem P, unsigned long long* __restrict__ vi
     const int lane = threadIdx.x & 31;
     const long long gw = (long long)blockIdx.x * kAuxWarps + (threadIdx.x >> 5), nwarps = (long long)gridDim.x * kAuxWarps;
     const long long units = P.cols / kUnit, chunks = (units + 127) / 128, total = P.rows * chunks;
-    const long long per = (total + nwarps - 1) / nwarps, begin = gw * per, end = min(total, begin + per);
     const unsigned char* mbytes = reinterpret_cast<const unsigned char*>(P.mask);
     unsigned long long viol = 0;
-    long long r = begin < end ? begin / chunks : 0, chunk = begin < end ? begin - r * chunks : 0;
-    for (long long item = begin; item < end; ++item) {
+    // items dealt round-robin: the grid reads one dense window of the matrix at a time
+    const long long dr = nwarps / chunks, dc = nwarps - dr * chunks;
+    long long r = gw / chunks, chunk = gw - r * chunks;
+    for (long long item = gw; item < total; item += nwarps) {
         constexpr int kWords = DT == kF32 ? 8 : 4;
         uint32_t w[4][kWords], given[4];
 #pragma unroll
@@ -224,7 +225,8 @@ violations_stream_kernel(const AuxProblem P, unsigned long long* __restrict__ vi
             }
             viol += (unsigned)__popc(nz & ~given[s]);
         }
-        if (++chunk == chunks) { chunk = 0; ++r; }
+        r += dr; chunk += dc;
+        if (chunk >= chunks) { chunk -= chunks; ++r; }
     }
     for (int o = 16; o; o >>= 1) viol += __shfl_xor_sync(0xFFFFFFFFu, viol, o);
     if (lane == 0) viol_partials[gw] = viol;
