@@ -237,9 +237,22 @@ __global__ void __launch_bounds__(kAuxWarps * 32)
 hamming_kernel(const uint32_t* __restrict__ a, const uint32_t* __restrict__ b, long long words, unsigned long long* __restrict__ partials) {
     const int lane = threadIdx.x & 31;
     const long long gw = (long long)blockIdx.x * kAuxWarps + (threadIdx.x >> 5), nwarps = (long long)gridDim.x * kAuxWarps;
-    const long long per = ((words + nwarps - 1) / nwarps + 31) / 32 * 32, begin = gw * per, end = min(words, begin + per);
     unsigned long long n = 0;
-    for (long long i = begin + lane; i < end; i += 32) n += __popc(__ldg(a + i) ^ __ldg(b + i));
+    if ((((uintptr_t)a | (uintptr_t)b) & 15) == 0) {
+        // 16 bytes per lane and load, the warps of the grid side by side (one dense window of both masks at a time)
+        const long long quads = words / 4;
+        const uint4* a4 = reinterpret_cast<const uint4*>(a);
+        const uint4* b4 = reinterpret_cast<const uint4*>(b);
+#pragma unroll 2
+        for (long long i = gw * 32 + lane; i < quads; i += nwarps * 32) {
+            const uint4 x = __ldg(a4 + i), y = __ldg(b4 + i);
+            n += __popc(x.x ^ y.x) + __popc(x.y ^ y.y) + __popc(x.z ^ y.z) + __popc(x.w ^ y.w);
+        }
+        if (gw == 0 && quads * 4 + lane < words) n += __popc(__ldg(a + quads * 4 + lane) ^ __ldg(b + quads * 4 + lane));
+    } else {
+        const long long per = ((words + nwarps - 1) / nwarps + 31) / 32 * 32, begin = gw * per, end = min(words, begin + per);
+        for (long long i = begin + lane; i < end; i += 32) n += __popc(__ldg(a + i) ^ __ldg(b + i));
+    }
     for (int o = 16; o; o >>= 1) n += __shfl_xor_sync(0xFFFFFFFFu, n, o);
     if (lane == 0) partials[gw] = n;
 }
