@@ -54,6 +54,11 @@ def test_mask_hamming():
         want = int(np.unpackbits((a ^ b).view(np.uint8)).sum())
         got = tm.tm_mask_hamming(torch.from_numpy(a.view(np.int32)).cuda(), torch.from_numpy(b.view(np.int32)).cuda())
         assert int(got.item()) == want
+        if n > 40:                                                   # masks that start off a 16-byte boundary
+            ad, bd = torch.from_numpy(a.view(np.int32)).cuda()[1:], torch.from_numpy(b.view(np.int32)).cuda()[3:n - 2 + 3 - 1]
+            m = min(ad.numel(), bd.numel())
+            got = tm.tm_mask_hamming(ad[:m], bd[:m])
+            assert int(got.item()) == int(np.unpackbits((a[1:1 + m] ^ b[3:3 + m]).view(np.uint8)).sum())
 
 
 @pytest.mark.gpu
