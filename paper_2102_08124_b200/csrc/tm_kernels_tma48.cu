@@ -18,6 +18,8 @@
 #include "tm_tma.cuh"
 #include "tm_tma_items.cuh"
 
+#include <type_traits>
+
 namespace tmask {
 
 namespace {
@@ -254,8 +256,17 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     }
 
     const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
+    // Algorithm 1 alone takes its items round-robin over the warps of the grid (one dense window of the matrix at a time),
+    // the full search contiguous ranges (see the 2:4 kernel)
+    constexpr bool kRoundRobin = METHOD != kMethodApprox;
     int n_items;
-    const long long begin = even_share(total_items, G::kWarps, n_items);
+    long long begin;
+    if constexpr (kRoundRobin) {
+        begin = (long long)warp * gridDim.x + blockIdx.x;
+        n_items = begin < total_items ? (int)((total_items - begin + nwarps - 1) / nwarps) : 0;
+    } else {
+        begin = even_share(total_items, G::kWarps, n_items);
+    }
     const TmaEntry* tab = table ? table : &single;
 
     if (lane == 0) {
@@ -264,8 +275,8 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     }
     __syncwarp();
 
-    Cursor ld, cur;
-    ld.seek(tab, count, begin);
+    typename std::conditional<kRoundRobin, StrideCursor, Cursor>::type ld, cur;
+    if constexpr (kRoundRobin) ld.seek(tab, count, begin, (int)nwarps); else ld.seek(tab, count, begin);
     cur = ld;
     int loaded = 0;
     auto issue_next = [&]() {              // all lanes track the cursor, lane 0 issues the copy
