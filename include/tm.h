@@ -48,7 +48,8 @@
  * pointer owned by the caller, calls are asynchronous on the stated stream, and nothing is
  * synchronised.  Host-detectable errors are returned (nothing is launched); conditions only the
  * device can see are OR-ed into a device status word (TM_DEV_* bits) that the caller reads after
- * its own synchronisation -- the outputs are fully written and deterministic even then.
+ * its own synchronisation -- with TM_DEV_NONFINITE or TM_DEV_BADMASK the outputs are fully written and
+ * deterministic; TM_DEV_INTERNAL means the call failed (see the bit's comment).
  * There is no CPU fallback: without a CUDA device every compute entry point returns TM_ERR_CUDA.
  */
 #ifndef TM_H_
@@ -83,10 +84,13 @@ extern "C" {
 #define TM_ERR_CUDA 7       /* a CUDA runtime call failed (no device, launch error, allocation failure) */
 #define TM_ERR_WORKSPACE 8  /* workspace NULL, misaligned (256 bytes) or smaller than tm_workspace_bytes() */
 #define TM_ERR_TOO_LARGE 9  /* more matrices than the built-in scratch of tm_find_mask_batched_static() can serve */
+#define TM_ERR_CAPTURE 10   /* cuda_stream is being captured and the call would have to copy descriptor tables from host memory */
 
 /* device status bits */
 #define TM_DEV_NONFINITE 1  /* an Inf or NaN was met in W (it is ordered by its bit pattern) */
-#define TM_DEV_INTERNAL 2   /* an iteration cap was hit (cannot happen; outputs fall back to a valid mask) */
+#define TM_DEV_INTERNAL 2   /* a bound inside a kernel was hit (not expected to happen).  An iteration cap of a per-block search leaves
+                               that block with the mask reached so far; a bulk copy that did not land within its bounded wait makes
+                               the warp stop, and the outputs of its remaining work items stay UNWRITTEN: treat the call as failed */
 #define TM_DEV_BADMASK 4    /* tm_compress_2_4: a group of four did not hold exactly two kept entries (zeros were emitted) */
 
 typedef struct tm_problem {
@@ -126,7 +130,12 @@ int tm_device_status(int* status_host);
  * workspace_dev: device scratch of at least tm_workspace_bytes(...) bytes, 256-byte aligned, owned
  * by the caller, reusable across calls on the same stream (calls on different streams need
  * different workspaces).  status_dev: device int, OR-ed with TM_DEV_* bits; may be NULL.
- * cuda_stream: a cudaStream_t (NULL = legacy default stream).  Never allocates, never synchronises.
+ * cuda_stream: a cudaStream_t (NULL = legacy default stream).  Never allocates.  With count == 1 the
+ * descriptors travel as kernel arguments and the call only enqueues work; with count > 1 it first copies
+ * the descriptor tables from (pageable) host memory into the workspace, and the runtime may hold the
+ * calling thread until earlier work of cuda_stream has drained before that copy is staged.  For the same
+ * reason only count == 1 calls can be recorded by a stream capture: a count > 1 call on a capturing
+ * stream returns TM_ERR_CAPTURE and enqueues nothing -- capture tm_plan_run() instead.
  * All matrices share N, M and method; dtypes may differ.
  */
 int tm_find_mask_batched(const tm_problem* probs_host, int count, int N, int M, int method,
@@ -175,10 +184,18 @@ int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols,
  *
  * The call allocates nothing on the device and frees nothing.  The first call on a device looks the
  * scratch array's device address up (once per device, with that device current); make that first call
- * before any stream capture begins.  All calls on one device share the one array, which keeps whatever
- * the previous call left in it: each call clears the objective partials it is about to use, but two
- * calls that overlap on the GPU (different streams, no dependency between them) race on it and corrupt
- * each other's objectives -- order them, or use tm_find_mask_batched() with separate workspaces.
+ * before any stream capture begins.  Like tm_find_mask_batched(), a call with count > 1 copies its
+ * descriptor tables from host memory and is refused (TM_ERR_CAPTURE) on a capturing stream.
+ *
+ * All calls on one device share the one array, which keeps whatever the previous call left in it; each
+ * call clears the objective partials it is about to use.  Calls that can overlap on the GPU (different
+ * streams with no dependency between them, or several host threads) MUST be ordered by the caller: the
+ * array holds not only the objective partials but, for count > 1, the descriptor table and the tensor
+ * maps with the output pointers, at fixed offsets, and every call rewrites them.  A second call can
+ * therefore replace the descriptors a running kernel is still reading -- wrong masks and masked weights,
+ * and accesses through foreign or half-written descriptors, i.e. memory safety is at stake, not only the
+ * objective.  Only count == 1 calls (descriptors passed as kernel arguments) confine such a race to the
+ * objective value.  Where calls cannot be ordered use tm_find_mask_batched() with separate workspaces.
  * Results are bit-identical to tm_find_mask_batched() on the same inputs.
  */
 #define TM_STATIC_MAX_MATRICES 16

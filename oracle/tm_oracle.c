@@ -161,8 +161,10 @@ static int complete_fill(const uint32_t* u, int N, int M, uint8_t* kept) {
  * x = (r', c') for which a short row r with (r, c') free and a short column c with (r', c) free
  * exist; un-keep x and keep the heaviest such (r, c') and the heaviest such (r', c).
  * Each swap adds one kept entry.  Returns the number of swaps, or -1 if no eligible entry exists
- * or the cap M*M is exceeded (neither can happen; the tests assert it). */
-static int complete_swap(const uint32_t* u, int N, int M, uint8_t* kept) {
+ * or the cap M*M is exceeded (neither can happen; the tests assert it).  If trace is not NULL it
+ * receives a copy of kept[] after every swap (M*M bytes each, room for N*N/4 + 1 of them): an
+ * observation point for the pins, the steps themselves do not look at it. */
+static int complete_swap(const uint32_t* u, int N, int M, uint8_t* kept, uint8_t* trace) {
     int n = M * M, order[TMO_MAXE], swaps = 0;
     sort_entries(u, n, order);
     for (;;) {
@@ -180,7 +182,11 @@ static int complete_swap(const uint32_t* u, int N, int M, uint8_t* kept) {
                 if (rk[r] < N && !kept[r * M + c2] && (a < 0 || lighter(u, a, r * M + c2))) a = r * M + c2;
             for (int c = 0; c < M; ++c)            /* heaviest free (r2, c) in a short column */
                 if (ck[c] < N && !kept[r2 * M + c] && (b < 0 || lighter(u, b, r2 * M + c))) b = r2 * M + c;
-            if (a >= 0 && b >= 0) { kept[x] = 0; kept[a] = 1; kept[b] = 1; swaps++; done = 1; }
+            if (a >= 0 && b >= 0) {
+                kept[x] = 0; kept[a] = 1; kept[b] = 1; done = 1;
+                if (trace && swaps <= N * N / 4) memcpy(trace + (size_t)swaps * (size_t)n, kept, (size_t)n);
+                swaps++;
+            }
         }
         if (!done) return -1;
     }
@@ -320,8 +326,20 @@ int tmo_block_approx(const uint32_t* u, int N, int M, uint8_t* kept, uint8_t* af
     if (after_a) memcpy(after_a, kept, (size_t)(M * M));
     int nb = complete_fill(u, N, M, kept);
     if (after_b) memcpy(after_b, kept, (size_t)(M * M));
-    int nc = complete_swap(u, N, M, kept);
+    int nc = complete_swap(u, N, M, kept, NULL);
     if (n_fill) *n_fill = nb;
+    if (n_swap) *n_swap = nc;
+    return nc < 0 ? TMO_ERR_ARG : TMO_OK;
+}
+
+/* The same search, also handing back the kept set after every swap of step C (swap_trace: room for
+ * N*N/4 + 1 sets of M*M bytes), so that the pins can check a sequence of swaps one rule application at a time. */
+int tmo_block_approx_trace(const uint32_t* u, int N, int M, uint8_t* kept, uint8_t* after_b, uint8_t* swap_trace, int* n_swap) {
+    if (!check_nm(N, M) || !swap_trace) return TMO_ERR_ARG;
+    alg1_cover(u, N, M, kept, NULL);
+    complete_fill(u, N, M, kept);
+    if (after_b) memcpy(after_b, kept, (size_t)(M * M));
+    int nc = complete_swap(u, N, M, kept, swap_trace);
     if (n_swap) *n_swap = nc;
     return nc < 0 ? TMO_ERR_ARG : TMO_OK;
 }
@@ -351,7 +369,7 @@ int tmo_block_exact_mcf(const uint32_t* u, int N, int M, uint8_t* kept, int* n_n
 static void solve_block(const uint32_t* u, int N, int M, int method, uint8_t* kept) {
     switch (method) {
     case TMO_APPROX_COVER: alg1_cover(u, N, M, kept, NULL); break;
-    case TMO_APPROX: alg1_cover(u, N, M, kept, NULL); complete_fill(u, N, M, kept); complete_swap(u, N, M, kept); break;
+    case TMO_APPROX: alg1_cover(u, N, M, kept, NULL); complete_fill(u, N, M, kept); complete_swap(u, N, M, kept, NULL); break;
     case TMO_EXACT_ENUM: exact_enumerate(u, N, M, kept); break;
     case TMO_EXACT_MCF: exact_mcf(u, N, M, kept, NULL, NULL, NULL); break;
     default: /* TMO_EXACT: the definition by enumeration where that is feasible, else Fig. 3's flow */

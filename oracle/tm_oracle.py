@@ -41,6 +41,7 @@ def _load():
         lib.tmo_find_mask.restype = i32
         lib.tmo_block_cover.argtypes = [vp, i32, i32, vp, vp, vp]
         lib.tmo_block_approx.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+        lib.tmo_block_approx_trace.argtypes = [vp, i32, i32, vp, vp, vp, vp]
         lib.tmo_block_exact_enum.argtypes = [vp, i32, i32, vp, vp]
         lib.tmo_block_exact_bruteforce.argtypes = [vp, i32, i32, vp, vp]
         lib.tmo_block_exact_mcf.argtypes = [vp, i32, i32, vp, vp, vp, vp]
@@ -92,6 +93,18 @@ def block_approx(block, N, M):
     assert rc == 0, "completion failed"
     return dict(kept=kept.reshape(M, M), after_a=a.reshape(M, M), after_b=b.reshape(M, M),
                 n_fill=nf.value, n_swap=ns.value)
+
+
+def block_approx_trace(block, N, M):
+    """Algorithm 1 + completion -> (after_b, [kept set after every swap of step C]); the last one is the result."""
+    u = _block_u(block, M)
+    kept = np.zeros(M * M, np.uint8); b = np.zeros(M * M, np.uint8); ns = ctypes.c_int(0)
+    trace = np.zeros((N * N // 4 + 1, M * M), np.uint8)
+    rc = _load().tmo_block_approx_trace(_ptr(u), N, M, _ptr(kept), _ptr(b), _ptr(trace), ctypes.byref(ns))
+    assert rc == 0, "completion failed"
+    states = [trace[k].reshape(M, M).copy() for k in range(ns.value)]
+    assert ns.value == 0 or np.array_equal(states[-1], kept.reshape(M, M))
+    return b.reshape(M, M), states
 
 
 def block_exact_enum(block, N, M):

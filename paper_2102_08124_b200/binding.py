@@ -11,6 +11,7 @@ TM_EXACT, TM_APPROX, TM_APPROX_COVER = 0, 1, 2
 TM_F32, TM_BF16 = 0, 1
 TM_DEV_NONFINITE, TM_DEV_INTERNAL, TM_DEV_BADMASK = 1, 2, 4
 TM_NM1D_ABSORB_MEAN = 1
+TM_ERR_TOO_LARGE, TM_ERR_CAPTURE = 9, 10
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libtm.so")
@@ -160,6 +161,30 @@ def _problem_array(Ws: Sequence, masks, maskeds, objectives):
     return arr
 
 
+def _batch_outputs(Ws: Sequence, masks, maskeds, objectives, workspace, status, want_masked: bool):
+    """Checks the matrices of a batched call and creates whichever output tensors the caller did not pass."""
+    import torch
+    dev = Ws[0].device
+    for W in Ws:
+        if not (W.is_cuda and W.dim() == 2 and (W.shape[1] <= 1 or W.stride(1) == 1) and W.device == dev):
+            raise TmError(2, "every W must be a 2-D CUDA tensor with unit column stride on one device")
+    if masks is None:
+        masks = [torch.empty((W.shape[0], tm_mask_words_per_row(W.shape[1])), dtype=torch.int32, device=dev) for W in Ws]
+    if maskeds is None and want_masked:
+        maskeds = [torch.empty_strided(W.shape, W.stride(), dtype=W.dtype, device=dev) for W in Ws]
+    if maskeds is not None:
+        for W, Y in zip(Ws, maskeds):                      # the ABI has one leading dimension per matrix
+            if Y is not None and (Y.shape != W.shape or Y.stride() != W.stride() or Y.dtype != W.dtype):
+                raise TmError(2, "masked_w_out must have the shape, strides and dtype of W")
+    if objectives is None:
+        objectives = torch.empty((len(Ws),), dtype=torch.float64, device=dev)
+    if status is None:
+        status = torch.zeros((1,), dtype=torch.int32, device=dev)
+    if workspace is None:
+        workspace = torch.empty((tm_workspace_bytes(len(Ws)),), dtype=torch.uint8, device=dev)
+    return dev, masks, maskeds, objectives, status, workspace
+
+
 class TmBatch:
     """A list of matrices with their output tensors, marshalled once into the C descriptor array.
 
@@ -167,27 +192,9 @@ class TmBatch:
     masks of the same weight buffers every few iterations prepares the batch once and calls run() each time."""
 
     def __init__(self, Ws: Sequence, masks=None, maskeds=None, objectives=None, workspace=None, status=None, want_masked: bool = True):
-        import torch
         if len(Ws) == 0:
             raise TmError(2, "empty batch")
-        dev = Ws[0].device
-        for W in Ws:
-            if not (W.is_cuda and W.dim() == 2 and (W.shape[1] <= 1 or W.stride(1) == 1) and W.device == dev):
-                raise TmError(2, "every W must be a 2-D CUDA tensor with unit column stride on one device")
-        if masks is None:
-            masks = [torch.empty((W.shape[0], tm_mask_words_per_row(W.shape[1])), dtype=torch.int32, device=dev) for W in Ws]
-        if maskeds is None and want_masked:
-            maskeds = [torch.empty_strided(W.shape, W.stride(), dtype=W.dtype, device=dev) for W in Ws]
-        if maskeds is not None:
-            for W, Y in zip(Ws, maskeds):                      # the ABI has one leading dimension per matrix
-                if Y is not None and (Y.shape != W.shape or Y.stride() != W.stride() or Y.dtype != W.dtype):
-                    raise TmError(2, "masked_w_out must have the shape, strides and dtype of W")
-        if objectives is None:
-            objectives = torch.empty((len(Ws),), dtype=torch.float64, device=dev)
-        if status is None:
-            status = torch.zeros((1,), dtype=torch.int32, device=dev)
-        if workspace is None:
-            workspace = torch.empty((tm_workspace_bytes(len(Ws)),), dtype=torch.uint8, device=dev)
+        dev, masks, maskeds, objectives, status, workspace = _batch_outputs(Ws, masks, maskeds, objectives, workspace, status, want_masked)
         self.Ws, self.masks, self.maskeds, self.objectives, self.status, self.workspace = list(Ws), masks, maskeds, objectives, status, workspace
         self.device = dev
         self.count = len(Ws)
@@ -254,30 +261,14 @@ def tm_find_mask_batched(Ws: Sequence, N: int, M: int, method: int, masks=None, 
     """One launch for a list of 2-D CUDA tensors (fp32 and/or bf16; rows may be strided, stride(1) == 1).
 
     Returns (masks, maskeds, objectives float64[count], status int32[1], workspace uint8[...]).  Runs on
-    `stream` (a torch.cuda.Stream) or on torch's current stream; nothing is synchronised."""
+    `stream` (a torch.cuda.Stream) or on torch's current stream.  With more than one matrix the descriptor tables
+    are copied from host memory first (the runtime may wait for the stream's earlier work to do so), and such a
+    call is refused on a capturing stream: capture tm_plan_run() instead."""
     import torch
     lib = load_library()
     if len(Ws) == 0:
         return [], [], None, status, workspace
-    dev = Ws[0].device
-    for W in Ws:
-        if not (W.is_cuda and W.dim() == 2 and (W.shape[1] <= 1 or W.stride(1) == 1) and W.device == dev):
-            raise TmError(2, "every W must be a 2-D CUDA tensor with unit column stride on one device")
-    if masks is None:
-        masks = [torch.empty((W.shape[0], tm_mask_words_per_row(W.shape[1])), dtype=torch.int32, device=dev) for W in Ws]
-    if maskeds is None and want_masked:
-        maskeds = [torch.empty_strided(W.shape, W.stride(), dtype=W.dtype, device=dev) for W in Ws]
-    if maskeds is not None:
-        for W, Y in zip(Ws, maskeds):                      # the ABI has one leading dimension per matrix
-            if Y is not None and (Y.shape != W.shape or Y.stride() != W.stride() or Y.dtype != W.dtype):
-                raise TmError(2, "masked_w_out must have the shape, strides and dtype of W")
-    if objectives is None:
-        objectives = torch.empty((len(Ws),), dtype=torch.float64, device=dev)
-    if status is None:
-        status = torch.zeros((1,), dtype=torch.int32, device=dev)
-    need = tm_workspace_bytes(len(Ws))
-    if workspace is None:
-        workspace = torch.empty((need,), dtype=torch.uint8, device=dev)
+    dev, masks, maskeds, objectives, status, workspace = _batch_outputs(Ws, masks, maskeds, objectives, workspace, status, want_masked)
     arr = _problem_array(Ws, masks, maskeds, objectives)
     with torch.cuda.device(dev):
         s = stream if stream is not None else torch.cuda.current_stream(dev)
@@ -294,7 +285,10 @@ def tm_find_mask_batched_static(Ws: Sequence, N: int, M: int, method: int, masks
     framework's memory pool, a pre-allocated real-time loop): the library's built-in scratch replaces the
     workspace, at most TM_STATIC_MAX_MATRICES matrices per call.  Every output tensor is passed in (masks:
     list of int32 [rows, wpr]; maskeds: list of tensors shaped like W, or None; objectives: float64[count];
-    status: int32[1]); this function creates no tensor.  Calls that overlap on the GPU race on the scratch."""
+    status: int32[1]); this function creates no tensor.  The caller must order the calls on a device: calls that
+    overlap on the GPU share the scratch, which for more than one matrix also holds the descriptor tables and
+    tensor maps, so an unordered second call can redirect the loads and stores of a running one (wrong outputs,
+    out-of-range accesses).  Only single-matrix calls confine such a race to the objective value."""
     import torch
     lib = load_library()
     dev = Ws[0].device if len(Ws) else torch.device("cuda")

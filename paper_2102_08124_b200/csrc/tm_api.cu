@@ -1,5 +1,6 @@
 // C ABI of the transposable N:M mask search (see include/tm.h): argument validation, work
 // partitioning and kernel dispatch.  Nothing here computes masks on the host.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -24,10 +25,12 @@ size_t table_bytes(int count) { return align_up(sizeof(DevProblem) * (size_t)at_
 size_t entry_bytes(int count) { return align_up(tmask::tma_entry_bytes() * (size_t)at_least_one(count)); }
 size_t partial_bytes(int count) { return align_up(sizeof(double) * (size_t)at_least_one(count) * kPartialSlots); }
 
+// `ready` and `scratch` are published with release stores after the fields they guard are written (under the mutex)
+// and read with acquire loads outside it.
 struct DeviceState {
-    bool ready = false;
+    std::atomic<bool> ready{false};
     int sms = 0;
-    void* scratch = nullptr;          // workspace of the plain calls: [status | table | partials]
+    std::atomic<void*> scratch{nullptr};   // workspace of the plain calls: [status | table | partials]
     size_t scratch_bytes = 0;
     // staging of tm_find_mask_host
     void* stage_w = nullptr; void* stage_masked = nullptr; void* stage_mask = nullptr; void* stage_ws = nullptr; double* stage_obj = nullptr;
@@ -41,11 +44,11 @@ int current_device(DeviceState** st) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return TM_ERR_CUDA; }
     DeviceState& d = g_dev[dev];
-    if (!d.ready) {
+    if (!d.ready.load(std::memory_order_acquire)) {
         std::lock_guard<std::mutex> lock(g_mutex);
-        if (!d.ready) {
+        if (!d.ready.load(std::memory_order_relaxed)) {
             if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
-            d.ready = true;
+            d.ready.store(true, std::memory_order_release);
         }
     }
     *st = &d;
@@ -178,8 +181,16 @@ int build_plan(const tm_problem* probs, int count, int N, int M, int method, voi
 }
 
 // Copies the descriptor tables of multi-matrix groups into the workspace (pageable sources: the runtime
-// stages the bytes before cudaMemcpyAsync returns, so the plan may die right after).
+// stages the bytes before cudaMemcpyAsync returns -- waiting for the stream's earlier work if it has to -- so the
+// plan may die right after).  Such a copy cannot be recorded by a stream capture (a replay would read host memory
+// that is long gone): a call that needs one while its stream is capturing is refused.
 int upload_plan(const Plan& plan, cudaStream_t stream) {
+    bool needed = false;
+    for (const PlanGroup& pg : plan.groups) needed |= pg.n > 1;
+    if (!needed) return TM_OK;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    if (cap != cudaStreamCaptureStatusNone) return TM_ERR_CAPTURE;
     for (const PlanGroup& pg : plan.groups) {
         if (pg.n <= 1) continue;
         cudaError_t e = pg.tma
@@ -211,14 +222,15 @@ int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, 
 }
 
 int ensure_scratch(DeviceState& d) {
-    if (d.scratch) return TM_OK;
+    if (d.scratch.load(std::memory_order_acquire)) return TM_OK;
     std::lock_guard<std::mutex> lock(g_mutex);
-    if (d.scratch) return TM_OK;
+    if (d.scratch.load(std::memory_order_relaxed)) return TM_OK;
     const size_t bytes = tm_workspace_bytes(nullptr, 1);
     void* p = nullptr;
     if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
     if (cudaMemset(p, 0, kHeaderBytes) != cudaSuccess) { cudaGetLastError(); cudaFree(p); return TM_ERR_CUDA; }
-    d.scratch = p; d.scratch_bytes = bytes;
+    d.scratch_bytes = bytes;
+    d.scratch.store(p, std::memory_order_release);
     return TM_OK;
 }
 
@@ -235,7 +247,8 @@ int plain_call(const void* W, int dtype, int64_t rows, int64_t cols, int N, int 
     DeviceState* d = nullptr;
     if ((rc = current_device(&d)) != TM_OK) return rc;
     if ((rc = ensure_scratch(*d)) != TM_OK) return rc;
-    return run(&p, 1, N, M, method, d->scratch, d->scratch_bytes, static_cast<int*>(d->scratch), nullptr, *d);
+    void* scratch = d->scratch.load(std::memory_order_acquire);
+    return run(&p, 1, N, M, method, scratch, d->scratch_bytes, static_cast<int*>(scratch), nullptr, *d);
 }
 
 int grow(void** p, size_t* have, size_t want) {
@@ -253,8 +266,7 @@ int grow(void** p, size_t* have, size_t want) {
 static __device__ __align__(256) unsigned char g_static_scratch[TM_STATIC_SCRATCH_BYTES];
 
 struct StaticScratch {
-    bool ready = false;
-    void* ptr = nullptr;
+    std::atomic<void*> ptr{nullptr};       // published once the look-up has succeeded
 };
 StaticScratch g_static[kMaxDevices];
 
@@ -262,16 +274,16 @@ int static_scratch_address(void** out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return TM_ERR_CUDA; }
     StaticScratch& s = g_static[dev];
-    if (!s.ready) {
+    void* p = s.ptr.load(std::memory_order_acquire);
+    if (!p) {
         std::lock_guard<std::mutex> lock(g_mutex);
-        if (!s.ready) {
-            void* p = nullptr;
+        p = s.ptr.load(std::memory_order_relaxed);
+        if (!p) {
             if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return TM_ERR_CUDA; }
-            s.ptr = p;
-            s.ready = true;
+            s.ptr.store(p, std::memory_order_release);
         }
     }
-    *out = s.ptr;
+    *out = p;
     return TM_OK;
 }
 
@@ -302,10 +314,11 @@ int tm_device_status(int* status_host) {
     int rc = current_device(&d);
     if (rc != TM_OK) return rc;
     *status_host = 0;
-    if (!d->scratch) return TM_OK;
+    void* scratch = d->scratch.load(std::memory_order_acquire);
+    if (!scratch) return TM_OK;
     if (cudaStreamSynchronize(nullptr) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
-    if (cudaMemcpy(status_host, d->scratch, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
-    if (cudaMemset(d->scratch, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    if (cudaMemcpy(status_host, scratch, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    if (cudaMemset(scratch, 0, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
     return TM_OK;
 }
 
@@ -591,6 +604,7 @@ const char* tm_status_string(int code) {
     case TM_ERR_CUDA: return "CUDA runtime error (no device, launch or allocation failure)";
     case TM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case TM_ERR_TOO_LARGE: return "too many matrices for the built-in scratch (TM_STATIC_MAX_MATRICES per call)";
+    case TM_ERR_CAPTURE: return "the stream is being captured and the call would have to copy descriptor tables from host memory (use tm_plan_run)";
     default: return "unknown status";
     }
 }

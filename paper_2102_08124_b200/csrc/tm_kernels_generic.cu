@@ -216,11 +216,10 @@ cudaError_t launch_nm(const LaunchArgs& a) {
     case kMethodExact: {
         // the flow solver (everything but 2:4) keeps its state in shared memory
         constexpr size_t smem = (N == 2 && M == 4) ? 0 : (size_t)flow_shared_bytes_per_thread(M) * kWarpsPerCta * 32;
-        static bool configured = false;    // per instantiation
-        if (smem > 48 * 1024 && !configured) {
-            cudaError_t e = cudaFuncSetAttribute(generic_kernel<N, M, kMethodExact>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        static PerDeviceOnce configured;   // per instantiation
+        if (smem > 48 * 1024) {
+            const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(generic_kernel<N, M, kMethodExact>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });
             if (e != cudaSuccess) return e;
-            configured = true;
         }
         generic_kernel<N, M, kMethodExact><<<grid, block, smem, a.stream>>>(a.single, a.table, a.count, a.total_items, a.partials, a.status);
         break;

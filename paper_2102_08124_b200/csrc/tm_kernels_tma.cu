@@ -357,7 +357,8 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         const int s = it % G::kStages;
         const uint32_t parity = (uint32_t)((it / G::kStages) & 1);
         unsigned char* stage = stages + s * G::kStageBytes;
-        if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bars[s], parity))) { status |= kDevInternal; alive = false; }
+        // a copy that never landed: stop before anything is computed on, or stored from, the unfilled stage
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bars[s], parity))) { status |= kDevInternal; alive = false; break; }
         int qn = 0;
         if (cur.k != acc_k) {                                   // a new matrix starts: flush the objective partial
             if (acc_k >= 0) {
@@ -543,12 +544,9 @@ cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntr
     using G = Geometry<DT, METHOD>;
     const size_t smem = G::kSmemBytes;
     auto kern = tma24_kernel<DT, METHOD, HAS_OUT>;
-    static bool configured = false;        // per instantiation
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDeviceOnce configured;       // per instantiation
+    const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });
+    if (e != cudaSuccess) return e;
     kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status, a.n_keep, a.vpartials);
     return cudaGetLastError();
 }

@@ -407,12 +407,9 @@ cudaError_t launch_one48(const TmaLaunch& a, const TmaEntry& single, const TmaEn
     using G = Geo48<DT, METHOD>;
     const size_t smem = (size_t)G::kWarps * G::kWarpBytes + (DT == kBF16 ? kLaneLutBytes : 0);
     auto kern = tma48_kernel<DT, METHOD, HAS_OUT>;
-    static bool configured = false;        // per instantiation
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDeviceOnce configured;       // per instantiation
+    const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });
+    if (e != cudaSuccess) return e;
     kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status);
     return cudaGetLastError();
 }

@@ -1,8 +1,27 @@
 // Host-side launch interface between the C ABI (tm_api.cu) and the kernel translation units.
 #pragma once
+#include <atomic>
+
 #include "tm_device.cuh"
 
 namespace tmask {
+
+// Function attributes (the dynamic shared-memory limit) belong to a device, not to the process: one flag per
+// device (up to 64, the library's limit) and kernel instantiation.  Two threads that meet an unset flag both set
+// the attribute, which is harmless.
+struct PerDeviceOnce {
+    std::atomic<unsigned long long> done{0};
+    template <class Fn> cudaError_t run(Fn&& fn) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        const unsigned long long bit = 1ull << (dev & 63);
+        if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
+        if ((e = fn()) != cudaSuccess) return e;
+        done.fetch_or(bit, std::memory_order_release);
+        return cudaSuccess;
+    }
+};
 
 struct LaunchArgs {
     DevProblem single;          // used when table == nullptr (count == 1)

@@ -405,6 +405,42 @@ def test_step_c_single_swap_takes_the_lightest_eligible_entry(N, M, kind):
     assert seen > 20
 
 
+def _swap_rule(S, block, N, M):
+    """One application of step C's rule to the kept set S (bool [M, M]) with a short row: the set it must produce."""
+    mag = np.abs(block.astype(np.float64))
+    key = lambda i, j: (mag[i, j], i * M + j)
+    DR = [i for i in range(M) if S[i].sum() < N]; DC = [j for j in range(M) if S[:, j].sum() < N]
+    elig = [(i, j) for i in range(M) for j in range(M) if S[i, j]
+            and any(not S[rr, j] for rr in DR) and any(not S[i, cc] for cc in DC)]
+    x = min(elig, key=lambda e: key(*e))
+    a = max(((rr, x[1]) for rr in DR if not S[rr, x[1]]), key=lambda e: key(*e))
+    b = max(((x[0], cc) for cc in DC if not S[x[0], cc]), key=lambda e: key(*e))
+    want = S.copy(); want[x] = False; want[a] = True; want[b] = True
+    return want
+
+
+@pytest.mark.parametrize("N,M,kind", [(4, 8, "laplace"), (4, 8, "ties"), (4, 8, "normal"), (3, 6, "ties"), (2, 4, "ties")])
+def test_step_c_every_swap_of_a_sequence_follows_the_rule(N, M, kind):
+    """Blocks that need several swaps: the kept set after every single swap (handed out by the oracle's trace entry) must
+    be what one application of the rule makes of the set before it, and the last one is the result.  The rule is applied
+    here to the oracle's intermediate states, so a wrong second or third swap cannot hide behind a right first one."""
+    multi = swaps_seen = 0
+    for block in rand_blocks(3000 if M == 8 else 800, M, 131 + M, kind):
+        after_b, states = orc.block_approx_trace(block, N, M)
+        assert len(states) == int(N * M - after_b.sum())                     # one swap per missing entry
+        S = after_b.astype(bool)
+        for nxt in states:
+            assert np.array_equal(_swap_rule(S, block, N, M), nxt.astype(bool))
+            S = nxt.astype(bool)
+            swaps_seen += 1
+        assert (S.sum(axis=0) == N).all() and (S.sum(axis=1) == N).all()
+        assert np.array_equal(S, orc.block_approx(block, N, M)["kept"].astype(bool))
+        multi += len(states) >= 2
+    assert swaps_seen > 20
+    if M == 8:
+        assert multi > 10                                                    # sequences of two or more swaps were really seen
+
+
 def _py_approx(block, N, M):
     """Steps A, B, C re-stated with Python sets (independent of the C code)."""
     mag = np.abs(block.astype(np.float64))

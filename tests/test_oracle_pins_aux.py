@@ -2,6 +2,7 @@
 transposable mask exists for): checked against numpy's sort, the paper's Eq. 3, closed forms and round trips."""
 from __future__ import annotations
 
+from fractions import Fraction
 from math import comb
 
 import numpy as np
@@ -80,6 +81,81 @@ def test_mean_absorption_preserves_the_group_sum(N, M):
     gb = workloads.f32_to_bf16_bits(np.array([[1.0, 3.0, -3.0, 4.0, 0.5, 0.25, 100.0, 0.001]], np.float32))
     outb = workloads.bf16_bits_to_f32(orc.nm_mask_1d(gb, 2, 4, absorb_mean=True)["masked"])
     assert outb[0, :4].tolist() == [0.0, 0.0, -1.0, 6.0] and outb[0, 5] == 0.0 and outb[0, 7] == 0.0
+
+
+def _bf16_nearest_even(x: Fraction) -> int:
+    """Bit pattern of the bf16 number nearest to the positive rational x (ties to the even pattern), worked out with
+    exact fractions: no float arithmetic, no bit tricks shared with the oracle.  Normal range only."""
+    assert x > 0
+    e = 0
+    while Fraction(2) ** (e + 1) <= x: e += 1
+    while Fraction(2) ** e > x: e -= 1
+    ulp = Fraction(2) ** (e - 7)                      # bf16: 8 significant bits
+    lo = (x // ulp) * ulp
+    hi = lo + ulp
+    def pattern(v):
+        ee = e if v < Fraction(2) ** (e + 1) else e + 1
+        frac = int(v / (Fraction(2) ** (ee - 7))) - 128
+        return ((ee + 127) << 7) | frac
+    if x - lo < hi - x: return pattern(lo)
+    if x - lo > hi - x: return pattern(hi)
+    return pattern(lo) if pattern(lo) % 2 == 0 else pattern(hi)
+
+
+def _bf16(v: float) -> int:
+    b = workloads.f32_to_bf16_bits(np.array([v], np.float32))
+    assert workloads.bf16_bits_to_f32(b)[0] == np.float32(v), "test value must be exact in bf16"
+    return int(b[0])
+
+
+@pytest.mark.parametrize("case", ["below", "above", "tie_even_low", "tie_odd_low", "carry", "exact"])
+def test_mean_absorption_rounds_bf16_to_nearest_even(case):
+    """Groups (p1, p2, k1, k2) with |p| < |k|: the pruned mean mu = (p1 + p2) / 2 is added to the kept entries, and the
+    sum -- exact in fp64 and in fp32 for these values -- must be rounded to bf16 to nearest, ties to even.  Expected
+    patterns come from exact fractions.  Truncation, round-half-up or a missing carry each fail one of the cases."""
+    u = 2.0 ** -7                                                   # bf16 spacing in [1, 2)
+    k1 = {"below": 1.0, "above": 1.0, "tie_even_low": 1.0, "tie_odd_low": 1.0 + u, "carry": 2.0 - u, "exact": 1.0}[case]
+    # mu chosen so that k1 + mu lies a quarter, three quarters or exactly half an ulp above k1 (all exact in fp32)
+    mu = {"below": u / 4, "above": 3 * u / 4, "tie_even_low": u / 2, "tie_odd_low": u / 2, "carry": u / 2, "exact": u}[case]
+    k2 = 1.5
+    g = np.array([[mu, mu, k1, k2]], np.float32)                    # the two light entries are pruned: their mean is mu
+    gb = np.array([[_bf16(mu), _bf16(mu), _bf16(k1), _bf16(k2)]], np.uint16)
+    res = orc.nm_mask_1d(gb, 2, 4, absorb_mean=True)
+    assert orc.unpack_mask(res["mask"], 4).tolist() == [[0, 0, 1, 1]]
+    want1 = _bf16_nearest_even(Fraction(k1) + Fraction(mu)); want2 = _bf16_nearest_even(Fraction(k2) + Fraction(mu))
+    assert [int(v) for v in res["masked"][0]] == [0, 0, want1, want2]
+    if case == "tie_even_low": assert want1 == _bf16(1.0)          # halfway between 1 and 1 + u: the even pattern is the lower one
+    if case == "tie_odd_low": assert want1 == _bf16(1.0 + 2 * u)   # halfway between 1 + u and 1 + 2u: the even one is the upper
+    if case == "carry": assert want1 == _bf16(2.0)                 # the rounding carries into the exponent
+    if case == "below": assert want1 == _bf16(1.0)
+    if case == "above": assert want1 == _bf16(1.0 + u)
+    # the same group in fp32 keeps the unrounded sum
+    assert orc.nm_mask_1d(g, 2, 4, absorb_mean=True)["masked"][0].tolist() == [0.0, 0.0, float(np.float32(k1 + mu)), float(np.float32(k2 + mu))]
+
+
+def test_mean_absorption_keeps_nan_a_nan_in_bf16():
+    gb = np.array([[_bf16(0.25), _bf16(0.5), 0x7FC1, _bf16(1.0)]], np.uint16)          # a NaN counts as the heaviest
+    out = orc.nm_mask_1d(gb, 2, 4, absorb_mean=True)["masked"][0]
+    assert out[0] == 0 and out[1] == 0
+    assert (int(out[2]) & 0x7F80) == 0x7F80 and (int(out[2]) & 0x7F) != 0             # still a NaN, not an Inf
+    assert int(out[3]) == _bf16(1.375)                                                # 1 + (0.25 + 0.5) / 2
+
+
+@pytest.mark.parametrize("N,M,group,want", [
+    # N kept of M.  mu = (sum of the pruned weights) / (number of pruned weights) -- the reading of Section 5's "mean of
+    # the pruned weights" taken by this build; spreading the pruned sum over the kept entries instead would give the
+    # values in the comments, which differ whenever N != M / 2.
+    (1, 4, [1.0, 2.0, 3.0, 8.0], [0.0, 0.0, 0.0, 10.0]),                                  # mean 6 / 3 = 2      (spread: 14)
+    (3, 4, [1.0, 2.0, 3.0, 8.0], [0.0, 3.0, 4.0, 9.0]),                                   # mean 1 / 1 = 1      (spread: 1/3 each)
+    (2, 8, [1.0, 2.0, 3.0, 4.0, 5.0, 6.0, 16.0, 32.0], [0.0] * 6 + [19.5, 35.5]),         # mean 21 / 6 = 3.5   (spread: 10.5)
+    (6, 8, [1.0, 3.0, 4.0, 5.0, 6.0, 7.0, 16.0, 32.0], [0.0, 0.0, 6.0, 7.0, 8.0, 9.0, 18.0, 34.0]),   # mean 4 / 2 = 2 (spread: 2/3)
+    (2, 4, [1.0, -5.0, 8.0, 16.0], [0.0, 0.0, 6.0, 14.0]),                                # mean (1 - 5) / 2 = -2: signs count
+])
+def test_mean_absorption_divides_by_the_number_of_pruned_weights(N, M, group, want):
+    g = np.array([group], np.float32)
+    assert orc.nm_mask_1d(g, N, M, absorb_mean=True)["masked"][0].tolist() == want
+    gb = workloads.f32_to_bf16_bits(g)                                                    # all values are exact in bf16
+    assert workloads.bf16_bits_to_f32(orc.nm_mask_1d(gb, N, M, absorb_mean=True)["masked"])[0].tolist() == want
 
 
 def _decompress(values, meta, cols):

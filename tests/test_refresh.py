@@ -43,6 +43,41 @@ def test_plan_equals_batched_call(N, M, method):
             assert np.array_equal(to_host_bits(masks[k]), to_host_bits(ref_masks[k]))
             assert np.array_equal(to_host_bits(maskeds[k]), to_host_bits(ref_maskeds[k]))
         assert np.array_equal(objs.cpu().numpy(), ref_obj.cpu().numpy())
+    # and, directly, the CPU oracle's answer on the same bytes
+    for k, m in enumerate(mats):
+        want = orc.find_mask(m, N, M, {tm.TM_APPROX: orc.APPROX, tm.TM_EXACT: orc.EXACT}[method])
+        assert np.array_equal(to_host_bits(masks[k]), want["mask"])
+        assert np.array_equal(to_host_bits(maskeds[k]), want["masked"].view(np.uint16 if m.dtype == np.uint16 else np.uint32))
+        assert abs(float(objs[k].item()) - want["objective"]) <= 1e-6 * abs(want["objective"])
+    tm.tm_plan_destroy(plan)
+
+
+@pytest.mark.gpu
+def test_multi_matrix_call_is_refused_on_a_capturing_stream():
+    """A call that must copy descriptor tables from host memory cannot be recorded: it returns TM_ERR_CAPTURE and
+    enqueues nothing; the prepared plan on the same buffers can be recorded and replayed."""
+    mats = [workloads.normal_bf16(16, 520, 0.02, 84), workloads.normal_bf16(16, 264, 0.02, 85)]
+    Ws = [to_device(m) for m in mats]
+    batch = tm.TmBatch(Ws)
+    batch.run(2, 4, tm.TM_APPROX)                                   # outside a capture: fine
+    plan = tm.tm_plan_create(Ws, 2, 4, tm.TM_APPROX)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    refused = None
+    with torch.cuda.graph(graph, stream=side):
+        try:
+            batch.run(2, 4, tm.TM_APPROX, stream=side)
+        except tm.TmError as e:
+            refused = e.code
+        tm.tm_plan_run(plan, stream=side)
+    assert refused == 10 and "captured" in tm.tm_status_string(10)
+    for t in plan.batch.masks:
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for k, m in enumerate(mats):
+        assert np.array_equal(to_host_bits(plan.batch.masks[k]), orc.find_mask(m, 2, 4, orc.APPROX, want_masked=False)["mask"])
     tm.tm_plan_destroy(plan)
 
 

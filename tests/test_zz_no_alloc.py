@@ -11,16 +11,21 @@ import torch
 
 import paper_2102_08124_b200 as tm
 import workloads
+from oracle import tm_oracle as orc
 from paper_2102_08124_b200 import binding
 
 pytestmark = pytest.mark.gpu
 
 
-def _device_tensors(M):
+def _host_matrices(M):
     # 132 bf16 columns give a row pitch that is not a multiple of 16 bytes (the generic kernel takes it);
     # the 4:8 search needs multiples of 8
-    mats = [workloads.normal_f32(64, 520, 0.02, 901), workloads.quantised_bf16(128, 1024, 0.02, 902),
+    return [workloads.normal_f32(64, 520, 0.02, 901), workloads.quantised_bf16(128, 1024, 0.02, 902),
             workloads.normal_bf16(16, 132 if M == 4 else 136, 0.02, 903), workloads.normal_f32(8, 8, 1.0, 904)]
+
+
+def _device_tensors(M):
+    mats = _host_matrices(M)
     out = []
     for m in mats:
         if m.dtype == np.uint16:
@@ -55,6 +60,14 @@ def test_static_scratch_entry_matches_the_workspace_entry(N, M, method):
             assert np.array_equal(masks[k].cpu().numpy(), ref_masks[k].cpu().numpy()), (round_, k)
             assert np.array_equal(_bits(maskeds[k]), _bits(ref_maskeds[k])), (round_, k)
         assert np.array_equal(obj.cpu().numpy(), ref_obj.cpu().numpy()), round_   # same kernels, same order: same bits
+    # and, directly, the CPU oracle's answer on the same bytes
+    oracle_method = {tm.TM_APPROX: orc.APPROX, tm.TM_EXACT: orc.EXACT}[method]
+    for k, m in enumerate(_host_matrices(M)):
+        want = orc.find_mask(m, N, M, oracle_method)
+        assert np.array_equal(masks[k].cpu().numpy().view(np.uint32), want["mask"]), k
+        assert np.array_equal(_bits(maskeds[k]).view(np.uint16 if m.dtype == np.uint16 else np.uint32),
+                              want["masked"].view(np.uint16 if m.dtype == np.uint16 else np.uint32)), k
+        assert abs(float(obj[k].item()) - want["objective"]) <= 1e-6 * abs(want["objective"])
 
 
 def test_static_scratch_entry_rejects_too_many_matrices():
