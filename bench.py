@@ -32,9 +32,10 @@ FULL_ROWS, COLS = 12288, 49152
 ROWS = FULL_ROWS
 N_KEEP, M_BLOCK = 2, 4
 BYTES_PER_WEIGHT = 2 + 2 + 1.0 / 8          # read W, write masked W, write one mask bit (bf16)
-# dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture on the 2048-row case (see profiles/), per weight
-TRAFFIC_PER_WEIGHT = (201.40e6 + 162.26e6) / (2048 * 49152)
-TRAFFIC_SOURCE = "ncu --set full on the 2048 x 49152 case, scaled by rows (profiles/tma24_kernel_approx_2_4_bf16_2048x49152_full.md)"
+# dram__bytes_read.sum + dram__bytes_write.sum of the search kernel, from an ncu capture (see profiles/); None until the
+# counters have been taken again for the kernel as it stands
+TRAFFIC_BYTES_PER_LAUNCH = None
+TRAFFIC_SOURCE = None
 METRIC = "transposable-mask weights/s (2:4 approx, bf16, 1 GPU: achieved HBM GB/s vs peak in `roofline`)"
 WORKLOAD = "%dx49152 bf16, N(0,0.02) quantised to 256 levels (frequent ties), 2:4 approximate, per-step recompute"
 
@@ -51,7 +52,7 @@ def measured_peak():
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,timestamp")
 
     def __init__(self, gpu_index: int):
         self.gpu = gpu_index
@@ -62,13 +63,18 @@ class ClockSampler:
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "100"],
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, since=None):
+        """Summary of the samples; `since` (a time.perf_counter() value) keeps only those taken after that moment."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        cut = None
+        if since is not None:
+            import datetime
+            cut = datetime.datetime.now() - datetime.timedelta(seconds=time.perf_counter() - since)
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -82,6 +88,13 @@ class ClockSampler:
                 f = [x.strip() for x in line.split(",")]
                 if len(f) < 9:
                     continue
+                if cut is not None and len(f) >= 10:
+                    try:
+                        import datetime
+                        if datetime.datetime.strptime(f[9], "%Y/%m/%d %H:%M:%S.%f") < cut:
+                            continue
+                    except ValueError:
+                        pass
                 try:
                     sm.append(float(f[1])); mx.append(float(f[2]))
                 except ValueError:
@@ -186,7 +199,10 @@ def run_gpu(args):
     sync()
     ms_cold = b0.elapsed_time(b1) / args.steps
 
-    # warm-up: at least W steps and long enough for the clock sampler (started first) to see the GPU under load
+    # Sustained measurement.  The clock sampler starts first; an extended warm-up (at least W steps, at least 0.6 s) lets
+    # the part settle at the clock it holds under load; then R blocks of exactly K steps are timed back to back with CUDA
+    # events on the launching stream (R chosen so that the timed region lasts about half a second and the sampler sees
+    # it), bracketed by a barrier and a synchronize.  The reported step time is the median block.
     sampler = ClockSampler(local_rank)
     if rank == 0 and not args.skip_clocks:
         sampler.start()
@@ -197,20 +213,25 @@ def run_gpu(args):
         if warm % 8 == 0:
             torch.cuda.synchronize()
     sync()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    repeats = args.repeats or max(10, min(200, int(0.5 / max(ms_cold * 1e-3 * args.steps, 1e-6))))
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
     sync()
-    start.record()
-    for _ in range(args.steps):
-        step()
-    end.record()
+    t_region = time.perf_counter()
+    marks[0].record()
+    for r in range(repeats):
+        for _ in range(args.steps):
+            step()
+        marks[r + 1].record()
     sync()
-    ms = start.elapsed_time(end) / args.steps
-    clocks = sampler.stop() if (rank == 0 and not args.skip_clocks) else None
+    region_s = time.perf_counter() - t_region
+    blocks_ms = sorted(marks[r].elapsed_time(marks[r + 1]) / args.steps for r in range(repeats))
+    ms = statistics.median(blocks_ms)
+    clocks = sampler.stop(since=t_region) if (rank == 0 and not args.skip_clocks) else None
     status = tm.tm_device_status()
-    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    t = torch.tensor([ms, blocks_ms[0], blocks_ms[-1]], dtype=torch.float64, device="cuda")
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max = float(t.item())
+    ms_max, ms_best, ms_worst = (float(v) for v in t.tolist())
 
     # end to end through the host-buffer entry point: pinned host input, results read back every step
     e2e = None
@@ -243,32 +264,116 @@ def run_gpu(args):
     weights = ROWS * COLS
     peak, peak_src = measured_peak()
     achieved = weights * BYTES_PER_WEIGHT / (ms * 1e-3) / 1e9
-    cpu_rows = min(768, ROWS)
-    cpu_value, cpu_dt = (None, 0.0) if args.skip_cpu else time_oracle(Wh, cpu_rows, 1)
+    cpu = None
+    if not args.skip_cpu and world == 1:
+        # the oracle as it stands on this machine's host cores: one thread (the plain definition) and all of them (its OpenMP
+        # loop over block rows), each on a bounded strip of the same matrix
+        cores = os.cpu_count() or 1
+        one_rows = min(768, ROWS)
+        one_value, one_dt = time_oracle(Wh, one_rows, 1)
+        from oracle import tm_oracle as orc
+        threads = orc.max_threads()
+        all_rows = min(ROWS, max(one_rows, 512 * threads))
+        all_value, all_dt = time_oracle(Wh, all_rows, threads)
+        cpu = {"value": all_value, "unit": "weights/s", "cores": threads, "kind": "oracle",
+               "sample": "first %d rows of the matrix (%d weights), %d OpenMP threads over block rows, %.1f s" % (all_rows, all_rows * COLS, threads, all_dt),
+               "single_thread": {"value": one_value, "unit": "weights/s", "cores": 1,
+                                 "sample": "first %d rows of the matrix (%d weights), %.1f s" % (one_rows, one_rows * COLS, one_dt)},
+               "host_cores": cores}
+    sm_mhz = clocks.get("sm_mhz") if clocks else None
     line = {
         "metric": METRIC, "value": world * weights / (ms_max * 1e-3), "unit": "weights/s", "n_gpus": world, "steps": args.steps,
-        "warmup": warm, "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "warmup": args.warmup, "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD % ROWS, "N": N_KEEP, "M": M_BLOCK, "method": "approx", "outputs": "mask+masked_w+objective",
                    "l2": "inputs (1.2 GB) larger than L2 (126 MB)", "device_status": status,
                    "objective": float(obj.item())},
+        "timing": {"blocks_of_K_steps": repeats, "timed_steps": repeats * args.steps, "region_s": region_s, "ms_per_step_median": ms,
+                   "ms_per_step_best_block": ms_best, "ms_per_step_worst_block": ms_worst, "warmup_steps_run": warm,
+                   "ms_x_sm_mhz": ms * sm_mhz if sm_mhz else None,
+                   "note": "value = median over the blocks; every block is exactly K steps, timed with CUDA events on the launching stream"},
         "e2e": e2e,
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": 2 * args.steps * repeats,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": TRAFFIC_PER_WEIGHT * weights if ROWS == FULL_ROWS else None, "traffic_source": TRAFFIC_SOURCE,
+                     "traffic": TRAFFIC_BYTES_PER_LAUNCH if ROWS == FULL_ROWS else None, "traffic_source": TRAFFIC_SOURCE,
                      "peak_source": peak_src, "algorithmic_bytes_per_launch": weights * BYTES_PER_WEIGHT,
                      "frac_of_8000": achieved / 8000.0,
                      "cold": {"ms_per_step": ms_cold, "achieved": weights * BYTES_PER_WEIGHT / (ms_cold * 1e-3) / 1e9,
                               "frac": weights * BYTES_PER_WEIGHT / (ms_cold * 1e-3) / 1e9 / peak,
-                              "note": "the same K steps timed right after W warm-up steps, before the sustained warm-up under the clock sampler"},
+                              "note": "K steps timed right after W warm-up steps, before the sustained warm-up under the clock sampler"},
                      "note": "duration = CUDA-event time of one step (search kernel + its tiny partial-zeroing and reduction launches)"},
-        "cpu_baseline": {"value": cpu_value, "unit": "weights/s", "cores": 1, "kind": "oracle",
-                         "sample": "first %d rows of the matrix (%d weights), %.1f s" % (cpu_rows, cpu_rows * COLS, cpu_dt)},
+        "cpu_baseline": cpu,
     }
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_dry(args):
+    """The multi-rank skeleton of run_gpu() without a GPU: gloo ranks, a host stand-in for the step, the same barrier,
+    max-over-ranks reduction and one JSON line from rank 0.  Used by the CPU test of the launcher."""
+    import torch
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    x = np.ones(1 << 16, np.float32)
+
+    def sync():
+        if world > 1:
+            dist.barrier()
+
+    for _ in range(max(args.warmup, 3)):
+        x += 1.0
+    sync()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        x += 1.0
+    ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    sync()
+    t = torch.tensor([ms], dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    if rank == 0:
+        print(json.dumps({"metric": "dry run of the launcher (no GPU work)", "value": world * x.size / (float(t.item()) * 1e-3), "unit": "elements/s",
+                          "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(t.item()), "scaling": "weak",
+                          "gpu_launches": 0}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def launch_ranks(args, argv):
+    """`--gpus N` with N > 1 outside a torchrun environment: start N ranks of this script on this node (one per GPU,
+    rendezvous on 127.0.0.1) and hand their output through; rank 0 prints the line."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus), "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + argv
+    return subprocess.call(cmd)
+
+
+def _block_sums(x, M):
+    r, c = x.shape
+    return x.reshape(r // M, M, c // M, M).sum(axis=(1, 3))
+
+
+def quality_numbers(W, cover_bits, approx_bits, exact_bits, M):
+    """Per-block quality of the approximation against the optimum (Section 4.1 quotes "within a factor of 1.2" for
+    Algorithm 1; the Lemma bounds the factor by 2): pruned-mass ratio W(P) / W* of the cover and of the completed mask,
+    kept-mass gap 1 - kept(approx) / kept(exact); mean and maximum over the blocks with W* > 0."""
+    mag = np.abs(W.astype(np.float64))
+    total = _block_sums(mag, M)
+    kept_e, kept_a, kept_c = (_block_sums(mag * b, M) for b in (exact_bits, approx_bits, cover_bits))
+    w_star, w_cover, w_approx = total - kept_e, total - kept_c, total - kept_a
+    ok = w_star > 0
+    return {"blocks": int(ok.sum()),
+            "cover_ratio_mean": float((w_cover[ok] / w_star[ok]).mean()), "cover_ratio_max": float((w_cover[ok] / w_star[ok]).max()),
+            "approx_ratio_mean": float((w_approx[ok] / w_star[ok]).mean()), "approx_ratio_max": float((w_approx[ok] / w_star[ok]).max()),
+            "kept_gap_mean": float((1 - kept_a[ok] / kept_e[ok]).mean()), "kept_gap_max": float((1 - kept_a[ok] / kept_e[ok]).max()),
+            "kept_gap_whole_matrix": float(1 - kept_a.sum() / kept_e.sum())}
 
 
 def run_survey(args):
@@ -320,6 +425,14 @@ def run_survey(args):
                               "frac_of_measured_hbm": gbs / peak, "steps": steps,
                               "resident_in_l2": bool(weights * bpw < 100e6), "status": int(status.item()),
                               "objective_sum": float(objs.sum().item())}), flush=True)
+        if name.startswith("config1") or name.startswith("config4"):
+            # quality of the approximation against the optimum, per block (masks from the GPU, sums on the host in fp64)
+            bits = {}
+            for mname in ("cover", "approx", "exact"):
+                batch.run(N, M, methods[mname]); torch.cuda.synchronize()
+                words = batch.masks[0].cpu().numpy().view(np.uint32)
+                bits[mname] = np.unpackbits(words.view(np.uint8), axis=1, bitorder="little")[:, :mats[0].shape[1]]
+            print(json.dumps({"workload": name, "N": N, "M": M, "quality": quality_numbers(mats[0], bits["cover"], bits["approx"], bits["exact"], M)}), flush=True)
         del Ws, batch, objs, status
         torch.cuda.empty_cache()
 
@@ -401,8 +514,14 @@ def main():
     ap.add_argument("--survey", action="store_true", help="secondary table: all named workloads and methods, one JSON line each")
     ap.add_argument("--config", type=int, default=0, help="with --survey: only this workload (1..5)")
     ap.add_argument("--survey-steps", type=int, default=0, help="with --survey: timed calls per case (default: about 0.5 s worth, at most 200)")
+    ap.add_argument("--repeats", type=int, default=0, help="timed blocks of K steps (default: about half a second worth, 10 to 200)")
+    ap.add_argument("--dry-run", action="store_true", help="launcher and multi-rank skeleton only: gloo on CPU, no GPU work")
     args = ap.parse_args()
-    if args.survey:
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.survey and args.impl != "reference":
+        raise SystemExit(launch_ranks(args, sys.argv[1:]))
+    if args.dry_run:
+        run_dry(args)
+    elif args.survey:
         if not args.config:
             run_survey(args)
             run_survey_neighbours(args)

@@ -59,3 +59,20 @@ def test_two_ranks_reproduce_the_unsharded_result(tmp_path):
     for m in metas:
         assert abs(m[2] - whole["objective"]) <= 1e-12 * whole["objective"]
         assert m[3] == float(world)                                # max over ranks
+
+
+def test_bench_starts_its_own_ranks():
+    """`bench.py --gpus 2` outside a torchrun environment starts two ranks itself (rendezvous on 127.0.0.1) and rank 0 prints
+    one line that counts both; here with the GPU step replaced by the host stand-in of --dry-run (gloo)."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "4", "--warmup", "3", "--dry-run"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                                      # rank 0 alone prints
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["steps"] == 4 and line["warmup"] == 3 and line["scaling"] == "weak"
