@@ -50,6 +50,9 @@ template <int K> TM_HD uint32_t rot_row(uint32_t x) {
 // result bit (i,j) = x bit ((i+k) mod 4, j), inside each 16-bit half
 template <int K> TM_HD uint32_t rot_col(uint32_t x) {
     constexpr uint32_t lo = K == 1 ? 0x0FFF0FFFu : (K == 2 ? 0x00FF00FFu : 0x000F000Fu);
+#if defined(__CUDA_ARCH__)
+    if constexpr (K == 2) { uint32_t r; asm("prmt.b32 %0, %1, %1, 0x2301;" : "=r"(r) : "r"(x)); return r; }   // bytes swapped inside either half
+#endif
     return ((x >> (4 * K)) & lo) | ((x << (16 - 4 * K)) & ~lo);
 }
 
@@ -75,14 +78,17 @@ struct LineFill {
     uint32_t row_full, col_full;
 };
 TM_HD LineFill line_fill(uint32_t kept) {
+    // Left shifts gather a line's four flags in its last entry (the top bit of the nibble, the last row); one right shift
+    // brings the verdict back down and a multiplication spreads it over the line.  (Left shifts can run on either of two
+    // pipes, right shifts only on the busier one.)
     LineFill f;
     {
-        const uint32_t a = kept, b = kept >> 1, c = kept >> 2, d = kept >> 3;
-        f.row_full = ((maj3(a, b, c) | (d & (a | b | c))) & 0x11111111u) * 15u;
+        const uint32_t a = kept, b = kept << 1, c = kept << 2, d = kept << 3;
+        f.row_full = (((maj3(a, b, c) | (d & (a | b | c))) >> 3) & 0x11111111u) * 15u;
     }
     {
-        const uint32_t a = kept, b = kept >> 4, c = kept >> 8, d = kept >> 12;
-        f.col_full = ((maj3(a, b, c) | (d & (a | b | c))) & 0x000F000Fu) * 0x1111u;
+        const uint32_t a = kept, b = kept << 4, c = kept << 8, d = kept << 12;
+        f.col_full = (((maj3(a, b, c) | (d & (a | b | c))) >> 12) & 0x000F000Fu) * 0x1111u;
     }
     return f;
 }
@@ -120,19 +126,6 @@ TM_HD uint32_t lone_candidates(uint32_t cand) {
 #endif
     const uint32_t several = cand & less_one;                          // a half is non-zero iff it holds two or more
     return cand & (((several & 0xFFFFu) ? 0u : 0xFFFFu) | ((several >> 16) ? 0u : 0xFFFF0000u));
-}
-
-// Steps A and B for one pair of blocks, without cross-lane votes (host tests, simple kernels).
-TM_HD uint32_t cover_and_fill_2_4(const Rel24& r, LineFill& f) {
-    uint32_t kept = cover_2_4(r);
-    f = line_fill(kept);
-    for (int round = 0; round < 4; ++round) {
-        const uint32_t cand = open_candidates(kept, f);
-        if (!cand) break;
-        kept |= fill_accept(r, kept, cand);
-        f = line_fill(kept);
-    }
-    return kept;
 }
 
 // Blocks (A: bit 0, B: bit 1) that still have a short row after step B, i.e. need step C.

@@ -418,22 +418,28 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             if constexpr (METHOD == kMethodApprox) {
                 LineFill f = line_fill(k);
                 uint32_t cand = open_candidates(k, f);
-                int rounds = 0;
-                while (__any_sync(0xFFFFFFFFu, cand != 0)) {
-                    if (++rounds > 4) { status |= kDevInternal; break; }    // a block lacks at most four entries
-                    if (rounds == 3) {      // after two rounds a block that still has candidates has, as a rule, exactly one:
-                                            // a third full round is needed by 3 % of the warps instead of 54 %
-                        k |= lone_candidates(cand);
-                        f = line_fill(k);
-                        cand = open_candidates(k, f);
-                        if (!__any_sync(0xFFFFFFFFu, cand != 0)) break;
-                    }
+                // two full rounds are needed by every warp of ordinary data (some block of its 64 has candidates left after
+                // the first): they run without asking; after them a block that still has candidates has, as a rule, one
+#pragma unroll
+                for (int round = 0; round < 2; ++round) {
                     k |= fill_accept(rel, k, cand);
                     f = line_fill(k);
                     cand = open_candidates(k, f);
                 }
+                if (__any_sync(0xFFFFFFFFu, cand != 0)) {
+                    k |= lone_candidates(cand);
+                    f = line_fill(k);
+                    cand = open_candidates(k, f);
+                    int rounds = 2;
+                    while (__any_sync(0xFFFFFFFFu, cand != 0)) {
+                        if (++rounds > 4) { status |= kDevInternal; break; }    // a block lacks at most four entries
+                        k |= fill_accept(rel, k, cand);
+                        f = line_fill(k);
+                        cand = open_candidates(k, f);
+                    }
+                }
                 const uint32_t sb = short_blocks(f);
-                if (__any_sync(0xFFFFFFFFu, sb != 0)) {
+                {   // some block of the 64 needs step C in all but a few warps: no vote first
 #pragma unroll
                     for (int b = 0; b < 2; ++b) {
                         const bool need = (sb >> b) & 1;
