@@ -101,9 +101,6 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
 
     // per-thread columns of the flow solver's state (only the exact instantiations that use it get dynamic shared memory)
     extern __shared__ __align__(16) unsigned char flow_smem[];
-    uint4* spot = reinterpret_cast<uint4*>(flow_smem) + threadIdx.x;
-    uint4* sdist = spot + 2 * M * (kWarpsPerCta * 32);
-    uint32_t* su = reinterpret_cast<uint32_t*>(flow_smem + 2 * (2 * M) * 16 * (kWarpsPerCta * 32)) + threadIdx.x;
 
     int k = 0, status = 0;
     double acc = 0.0;
@@ -145,7 +142,7 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
         uint64_t kept;
         if constexpr (METHOD == kMethodExact) {
             if constexpr (M == 4 && N == 2) kept = exact_2_4(u, P.dtype == kBF16 ? 16 : 0);
-            else kept = exact_ssp<N, M>(u, status, su, spot, sdist, kWarpsPerCta * 32);
+            else kept = exact_ssp<N, M, kWarpsPerCta * 32>(u, status, flow_smem, (int)threadIdx.x, active);
         } else {
             kept = cover_mask<N, M>(u);
             if constexpr (METHOD == kMethodApprox) {

@@ -36,6 +36,7 @@ template <int DT, int METHOD> struct Geo48 {
     static constexpr int kRowPitch = kCols8 * kElem;
     static constexpr int kStageBytes = kRows8 * kRowPitch;
     static constexpr int kWarpBytes = kStages * kStageBytes + 256 /* mask bytes [8][32] */ + 64 /* barriers */ + 64;
+    static constexpr int kLutBytes = DT == kBF16 ? kLaneLutBytes : 256 * 32;     // keep flags of a row as lane masks (bf16) or as 0/1 words (fp32)
 };
 
 __device__ __forceinline__ uint32_t max_u16x2_(uint32_t a, uint32_t b) {
@@ -158,6 +159,68 @@ __device__ __forceinline__ void relations48_f32(const unsigned char* blk, Rel48&
     complete_relations8(rel);
 }
 
+// ---- fp32, finite data: subtractions on the floating-point pipe ------------------------------------
+// The sign of |q| - |p| decides "q lighter than p" exactly (a difference of two finite floats is zero only for equal
+// operands and never changes sign in rounding; denormals are kept).  One subtraction per comparison runs on the
+// multiply-add pipe, one funnel shift pushes its sign bit into the relation word: half the logic-pipe work of a
+// compare-and-set pair.  A partner at a later position is heavier on ties, so for it the pushed bit is the complement
+// of the relation (turned by one constant per word at the end); a partner at an earlier position (the line wrapped
+// around) needs a strictly larger magnitude, and |p| - |q| gives the relation itself.
+__device__ __forceinline__ uint32_t push_sign(uint32_t acc, float d) { return __funnelshift_l(__float_as_uint(d), acc, 1); }
+
+__device__ __forceinline__ void relations48_f32_arith(const float (&f)[64], Rel48& rel) {
+#pragma unroll
+    for (int k = 1; k <= 4; ++k) {
+        uint32_t rw[2], cw[2] = {0, 0};
+        // rows: bit 8r + j of word w <- entry (4w + r, j) against (4w + r, j + k mod 8); k = 4: columns 0..3 only
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            uint32_t acc = 0;
+#pragma unroll
+            for (int r = 3; r >= 0; --r) {
+                const int i = 4 * w + r;
+                if (k == 4 && r != 3) acc <<= 4;
+#pragma unroll
+                for (int j = (k == 4 ? 3 : 7); j >= 0; --j) {
+                    const int jj = (j + k) & 7;
+                    const float a = fabsf(f[8 * i + jj]), b = fabsf(f[8 * i + j]);
+                    acc = push_sign(acc, (j + k <= 7) ? a - b : b - a);
+                }
+            }
+            const uint32_t later = k == 4 ? 0x0F0F0F0Fu : 0x01010101u * ((1u << (8 - k)) - 1u);      // partners that did not wrap
+            rw[w] = acc ^ later;
+        }
+        // columns: bit 8r + j of word w <- entry (4w + r, j) against (4w + r + k mod 8, j); k = 4: rows 0..3 only
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            if (k == 4 && w == 1) continue;
+            uint32_t acc = 0, later = 0;
+#pragma unroll
+            for (int r = 3; r >= 0; --r) {
+                const int i = 4 * w + r, ii = (i + k) & 7;
+                if (i + k <= 7) later |= 0xFFu << (8 * r);
+#pragma unroll
+                for (int j = 7; j >= 0; --j) {
+                    const float a = fabsf(f[8 * ii + j]), b = fabsf(f[8 * i + j]);
+                    acc = push_sign(acc, (i + k <= 7) ? a - b : b - a);
+                }
+            }
+            cw[w] = acc ^ later;
+        }
+        rel.hr[k] = (u64)rw[0] | ((u64)rw[1] << 32);
+        rel.hc[k] = (u64)cw[0] | ((u64)cw[1] << 32);
+    }
+    complete_relations8(rel);
+}
+
+// Keep flags of a row of eight fp32 entries as eight words of 0 or 1: entry e of the 256-entry table (two 16-byte halves).
+__device__ __forceinline__ void fill_keep_lut32(uint4* lut, int tid, int nthreads) {
+    for (int e = tid; e < 256; e += nthreads) {
+        lut[2 * e] = make_uint4(e & 1, (e >> 1) & 1, (e >> 2) & 1, (e >> 3) & 1);
+        lut[2 * e + 1] = make_uint4((e >> 4) & 1, (e >> 5) & 1, (e >> 6) & 1, (e >> 7) & 1);
+    }
+}
+
 // magnitude pattern of entry p of the lane's block, read back from the stage
 template <int DT>
 __device__ __forceinline__ uint32_t key_at(const unsigned char* blk, int p) {
@@ -202,7 +265,6 @@ __device__ __forceinline__ float back_end48(unsigned char* blk, unsigned char* m
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const uint32_t word = kw[i >> 2];
-        const int base = 8 * (i & 3);
         const uint32_t mb = (i & 3) == 0 ? (word & 0xFFu) : prmt(word, 0u, 0x4440 + (i & 3));      // the row's mask byte
         if constexpr (DT == kBF16) {
             const uint4 r = *reinterpret_cast<const uint4*>(blk + i * 512);
@@ -222,11 +284,12 @@ __device__ __forceinline__ float back_end48(unsigned char* blk, unsigned char* m
             if constexpr (HAS_OUT) *reinterpret_cast<uint4*>(blk + i * 512) = make_uint4(o[0], o[1], o[2], o[3]);
         } else {
             const uint4 ra = *reinterpret_cast<const uint4*>(blk + i * 1024), rb = *reinterpret_cast<const uint4*>(blk + i * 1024 + 16);
-            const uint32_t raw[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+            const uint4 ka = lut[2 * mb], kb = lut[2 * mb + 1];          // the row's keep flags as words of 0 or 1
+            const uint32_t raw[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w}, k01[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
             uint32_t o[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
-                o[q] = ((word >> (base + q)) & 1u) ? raw[q] : 0u;
+                o[q] = raw[q] * k01[q];                                  // the bits themselves or +0: an integer product, off the logic pipe
                 s8 += fabsf(__uint_as_float(o[q]));
             }
             if constexpr (HAS_OUT) {
@@ -250,10 +313,9 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     unsigned char* mbytes = stages + G::kStages * G::kStageBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(mbytes + 256);
     uint4* lut = reinterpret_cast<uint4*>(smem_raw + (size_t)G::kWarps * G::kWarpBytes);
-    if constexpr (DT == kBF16) {           // the only CTA-wide step: the lane-mask table
-        fill_lane_lut(lut, threadIdx.x, G::kWarps * 32);
-        __syncthreads();
-    }
+    // the only CTA-wide step: the table of keep flags
+    if constexpr (DT == kBF16) fill_lane_lut(lut, threadIdx.x, G::kWarps * 32); else fill_keep_lut32(lut, threadIdx.x, G::kWarps * 32);
+    __syncthreads();
 
     const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
     // Algorithm 1 alone takes its items round-robin over the warps of the grid (one dense window of the matrix at a time),
@@ -293,6 +355,9 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     int status = 0, acc_k = -1;
     float facc = 0.f; double acc = 0.0;
     uint32_t worst = 0;
+    // the matrix in process: the fields every item needs
+    int p_cols = 0, p_wpr = 0;
+    uint32_t* p_mask = nullptr;
 
     for (int it = 0; it < n_items; ++it) {
         const int s = it % G::kStages;
@@ -326,25 +391,45 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                 relations48_bf16<true>(R, rel);
             }
         } else {
-            relations48_f32(blk, rel, worst);
+            float f[64];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float4 a = *reinterpret_cast<const float4*>(blk + i * 1024), b = *reinterpret_cast<const float4*>(blk + i * 1024 + 16);
+                f[8 * i] = a.x; f[8 * i + 1] = a.y; f[8 * i + 2] = a.z; f[8 * i + 3] = a.w;
+                f[8 * i + 4] = b.x; f[8 * i + 5] = b.y; f[8 * i + 6] = b.z; f[8 * i + 7] = b.w;
+            }
+            // Inf / NaN watch on the multiply-add pipe: x * 0 + acc stays 0 for finite data and turns NaN otherwise
+            float watch = 0.f;
+#pragma unroll
+            for (int p = 0; p < 64; ++p) watch = fmaf(f[p], 0.f, watch);
+            if (__any_sync(0xFFFFFFFFu, watch != watch)) relations48_f32(blk, rel, worst);       // integer keys, bit-pattern order
+            else relations48_f32_arith(f, rel);
         }
         u64 kept = cover_4_8(rel);
         if constexpr (METHOD == kMethodApprox) {
             Short48 L = line_short(kept);
             u64 cand = open_candidates8(kept, L);
-            int rounds = 0;
-            while (__any_sync(0xFFFFFFFFu, cand != 0)) {
-                if (++rounds > 16) { status |= kDevInternal; break; }      // a block lacks at most sixteen entries
-                if (rounds == 4) {      // after three rounds a block that still has candidates has, as a rule, exactly one: it has
-                                        // no rival in its row or column and is taken as it stands
-                    if ((cand & (cand - 1)) == 0) kept |= cand;
-                    L = line_short(kept);
-                    cand = open_candidates8(kept, L);
-                    if (!__any_sync(0xFFFFFFFFu, cand != 0)) break;
-                }
+            // three full rounds are needed by every warp of ordinary data (some block of its 32 still has candidates):
+            // they run without asking
+#pragma unroll 1                                                           // one copy of the round's code: the loop body is large
+            for (int round = 0; round < 3; ++round) {
                 kept |= fill_accept8(rel, kept, cand);
                 L = line_short(kept);
                 cand = open_candidates8(kept, L);
+            }
+            if (__any_sync(0xFFFFFFFFu, cand != 0)) {
+                // a block that still has candidates has, as a rule, exactly one: it has no rival in its row or column and
+                // is taken as it stands
+                if ((cand & (cand - 1)) == 0) kept |= cand;
+                L = line_short(kept);
+                cand = open_candidates8(kept, L);
+                int rounds = 3;
+                while (__any_sync(0xFFFFFFFFu, cand != 0)) {
+                    if (++rounds > 16) { status |= kDevInternal; break; }  // a block lacks at most sixteen entries
+                    kept |= fill_accept8(rel, kept, cand);
+                    L = line_short(kept);
+                    cand = open_candidates8(kept, L);
+                }
             }
             int swaps = 0;
             while (__any_sync(0xFFFFFFFFu, L.row_short != 0)) {
@@ -357,9 +442,6 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                 }
             }
         }
-        const TmaEntry& e = tab[cur.k];
-        if (cur.cj * kCols8 + lane * 8 >= (int)e.p.cols) kept = 0;       // blocks past the last column (zero-filled by the copy)
-
         if (cur.k != acc_k) {                                              // a new matrix starts: flush the objective partial
             if (acc_k >= 0) {
                 acc += (double)facc;
@@ -367,18 +449,21 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                 if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
             }
             acc = 0.0; facc = 0.f; acc_k = cur.k;
+            const DevProblem& P = tab[cur.k].p;
+            p_cols = (int)P.cols; p_wpr = P.wpr; p_mask = P.mask;
         }
+        if (cur.cj * kCols8 + lane * 8 >= p_cols) kept = 0;               // blocks past the last column (zero-filled by the copy)
         facc += back_end48<DT, HAS_OUT>(blk, mbytes, lut, lane, kept);
         if constexpr (HAS_OUT) fence_proxy_async_smem();
         __syncwarp();
         if constexpr (HAS_OUT) {
-            if (lane == 0) { tma_store_2d(&e.out, cur.cj * kCols8, cur.bi * kRows8, stage); tma_commit(); }
+            if (lane == 0) { tma_store_2d(&tab[cur.k].out, cur.cj * kCols8, cur.bi * kRows8, stage); tma_commit(); }
         }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {                                      // 8 rows x 8 words of mask
             const int idx = lane + 32 * h, row = idx >> 3, word = cur.cj * 8 + (idx & 7);
             const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + row * 32 + (idx & 7) * 4);
-            if (word < e.p.wpr) e.p.mask[((long long)cur.bi * kRows8 + row) * e.p.wpr + word] = w;
+            if (word < p_wpr) p_mask[((long long)cur.bi * kRows8 + row) * p_wpr + word] = w;
         }
         // refill: the stage of the previous item is free once its store has been read
         if (loaded < n_items) {
@@ -405,7 +490,7 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
 template <int DT, int METHOD, bool HAS_OUT>
 cudaError_t launch_one48(const TmaLaunch& a, const TmaEntry& single, const TmaEntry* table) {
     using G = Geo48<DT, METHOD>;
-    const size_t smem = (size_t)G::kWarps * G::kWarpBytes + (DT == kBF16 ? kLaneLutBytes : 0);
+    const size_t smem = (size_t)G::kWarps * G::kWarpBytes + G::kLutBytes;
     auto kern = tma48_kernel<DT, METHOD, HAS_OUT>;
     static PerDeviceOnce configured;       // per instantiation
     const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });

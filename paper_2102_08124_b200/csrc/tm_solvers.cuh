@@ -480,54 +480,132 @@ __device__ __noinline__ uint64_t exact_flow_run(const uint32_t (&u)[M * M], int 
 // instruction stream for all lanes.  The scalar version above branches on the node it has just settled, so
 // the 32 lanes of a warp drift apart and execute one after the other; here every data-dependent choice is a
 // select or a predicated store, every loop is uniform (a vote ends it when no lane needs another turn), and
-// a settled node's row and column cases share one body.  A thread's magnitudes, potentials and distances
+// a settled node's row and column cases share one body.  A thread's edge costs, potentials and distances
 // are three strided columns (stride T entries); predecessors and column loads are packed four bits each
 // into registers.  Must be called by all 32 lanes; lanes with `enabled` false take part in the votes only.
-constexpr int flow_shared_bytes_per_thread(int M) { return M * M * 4 + 2 * (2 * M) * 16; }
+//
+// Two number formats share the routine.  Flow128 carries the full costs q_p * 2^64 + 2^p (recomputed from the
+// magnitudes at every use).  Flow64 carries q_p alone, precomputed: half the words in every load, sum and
+// comparison.  Without the tie term the optimum it finds is the wanted one only if it is the only one; that is
+// certified afterwards (tight_forest below), and a block without the certificate is solved again in full.
+// Shared-memory state.  A thread owns the 8-byte cells t, T + t, 2T + t, ... of the CTA's region (T threads; consecutive
+// threads touch consecutive cells, so 8-byte accesses do not collide) -- the same cells in either format, because warps
+// of a CTA can be in different formats at the same time.  cell(base, k, T) is the k-th cell of the thread whose first is base.
+constexpr int flow_cells_per_thread(int M) { return M * M + 2 * (2 * M); }                   // Flow64: a cell per cost, potential, distance
+constexpr int flow_shared_bytes_per_thread(int M) {                                         // Flow128: two cells per potential / distance, half a cell per magnitude
+    return 8 * (flow_cells_per_thread(M) > 4 * (2 * M) + M * M / 2 ? flow_cells_per_thread(M) : 4 * (2 * M) + M * M / 2);
+}
+typedef unsigned long long FlowCell;
+__device__ __forceinline__ FlowCell* cell(FlowCell* base, int k, int T) { return base + (size_t)k * T; }
 
-__device__ __forceinline__ __int128 ld128(const uint4* p) {
-    const uint4 v = *p;
-    return (__int128)(((unsigned __int128)(((unsigned long long)v.w << 32) | v.z) << 64) | (((unsigned long long)v.y << 32) | v.x));
-}
-__device__ __forceinline__ void st128(uint4* p, __int128 x) {
-    const unsigned long long lo = (unsigned long long)x, hi = (unsigned long long)((unsigned __int128)x >> 64);
-    *p = make_uint4((uint32_t)lo, (uint32_t)(lo >> 32), (uint32_t)hi, (uint32_t)(hi >> 32));
-}
 __device__ __forceinline__ __int128 edge_cost128(uint32_t u, int Emin, int p) {
     uint32_t sig; int E; split_float(u, sig, E);
     return ((__int128)((long long)sig << (sig ? E - Emin : 0)) << 64) + ((__int128)1 << p);
 }
 
-template <int N, int M>
+template <int M> struct Flow128 {
+    typedef __int128 V;
+    static constexpr bool kTieFree = false;
+    static constexpr int kPot = 0, kDist = 2 * (2 * M), kCost = 4 * (2 * M);                // first cell of each array
+    static constexpr int kCells = 2;                                                        // cells per potential / distance
+    static __device__ __forceinline__ V ld(FlowCell* base, int first, int n, int T) {
+        const FlowCell lo = *cell(base, first + 2 * n, T), hi = *cell(base, first + 2 * n + 1, T);
+        return (__int128)(((unsigned __int128)hi << 64) | lo);
+    }
+    static __device__ __forceinline__ void st(FlowCell* base, int first, int n, int T, V x) {
+        *cell(base, first + 2 * n, T) = (FlowCell)x; *cell(base, first + 2 * n + 1, T) = (FlowCell)((unsigned __int128)x >> 64);
+    }
+    static __device__ __forceinline__ V ldp(FlowCell* first, int T) { return (__int128)(((unsigned __int128)first[T] << 64) | first[0]); }
+    static __device__ __forceinline__ void stp(FlowCell* first, int T, V x) { first[0] = (FlowCell)x; first[T] = (FlowCell)((unsigned __int128)x >> 64); }
+    // what is kept per entry: the magnitude, two to a cell
+    static __device__ __forceinline__ void put_cost(FlowCell* base, int p, int T, uint32_t u, int) {
+        reinterpret_cast<uint32_t*>(cell(base, kCost + (p >> 1), T))[p & 1] = u;
+    }
+    static __device__ __forceinline__ V cost(FlowCell* base, int p, int T, int Emin) {
+        return edge_cost128(reinterpret_cast<const uint32_t*>(cell(base, kCost + (p >> 1), T))[p & 1], Emin, p);
+    }
+};
+template <int M> struct Flow64 {
+    typedef long long V;
+    static constexpr bool kTieFree = true;
+    static constexpr int kCost = 0, kPot = M * M, kDist = M * M + 2 * M;
+    static constexpr int kCells = 1;
+    static __device__ __forceinline__ V ld(FlowCell* base, int first, int n, int T) { return (V)*cell(base, first + n, T); }
+    static __device__ __forceinline__ void st(FlowCell* base, int first, int n, int T, V x) { *cell(base, first + n, T) = (FlowCell)x; }
+    static __device__ __forceinline__ V ldp(FlowCell* first, int) { return (V)*first; }
+    static __device__ __forceinline__ void stp(FlowCell* first, int, V x) { *first = (FlowCell)x; }
+    // q_p, at most 50 bits (24 significand bits, 26 binades); paths add 4 bits, potentials 5
+    static __device__ __forceinline__ void put_cost(FlowCell* base, int p, int T, uint32_t u, int Emin) {
+        uint32_t sig; int E; split_float(u, sig, E);
+        *cell(base, kCost + p, T) = (FlowCell)sig << (sig ? E - Emin : 0);
+    }
+    static __device__ __forceinline__ V cost(FlowCell* base, int p, int T, int) { return (V)*cell(base, kCost + p, T); }
+};
+
+// Is the bipartite graph of the marked entries (rows and columns as nodes, bit i*M+j an edge) free of cycles?  Leaves are
+// stripped until nothing changes: rows with a single edge lose it, then columns with a single edge; what survives lies on
+// a cycle.  Called by all 32 lanes (the loop ends on a vote).
+template <int M>
+__device__ __forceinline__ bool tight_forest(uint64_t edges) {
+    uint32_t row[M];
+#pragma unroll
+    for (int i = 0; i < M; ++i) row[i] = (uint32_t)(edges >> (i * M)) & ((1u << M) - 1u);
+    for (int it = 0; it < 2 * M; ++it) {
+        bool changed = false;
+        uint32_t once = 0, twice = 0;                                   // columns with at least one / at least two edges
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            const bool single = row[i] != 0 && (row[i] & (row[i] - 1)) == 0;
+            changed |= single;
+            row[i] = single ? 0u : row[i];
+            twice |= once & row[i]; once |= row[i];
+        }
+        const uint32_t leaf_cols = once & ~twice;
+        changed |= leaf_cols != 0;
+#pragma unroll
+        for (int i = 0; i < M; ++i) row[i] &= ~leaf_cols;
+        if (!__any_sync(0xFFFFFFFFu, changed)) break;
+    }
+    uint32_t left = 0;
+#pragma unroll
+    for (int i = 0; i < M; ++i) left |= row[i];
+    return left == 0;
+}
+
+// certified (Flow64 only): set to true when the optimum found is the only one, so that the tie rule has nothing to decide:
+// by complementary slackness every optimal flow agrees with this one outside the entries of reduced cost zero, and when
+// those entries form a forest the row and column totals fix the flow on them too.
+template <class A, int N, int M, int T>
 __device__ __noinline__ uint64_t exact_flow_warp(const uint32_t (&u)[M * M], int Emin, bool enabled, int& status,
-                                                 uint32_t* su, uint4* spot, uint4* sdist, int T) {
+                                                 FlowCell* base, bool* certified) {
+    typedef typename A::V V;
     constexpr int P = M - N;
     constexpr unsigned kFull = 0xFFFFFFFFu;
     uint64_t pruned = 0;
     uint32_t load = 0;                                                  // nibble j: pruned entries of column j
 #pragma unroll
-    for (int j = 0; j < M; ++j) st128(spot + (M + j) * T, 0);
+    for (int j = 0; j < M; ++j) A::st(base, A::kPot, M + j, T, 0);
 #pragma unroll
     for (int i = 0; i < M; ++i) {
 #pragma unroll
         for (int j = 0; j < M; ++j) {
-            su[(i * M + j) * T] = u[i * M + j];
+            A::put_cost(base, i * M + j, T, u[i * M + j], Emin);
             int heavier = 0;
 #pragma unroll
             for (int k = 0; k < M; ++k)
                 heavier += (k != j) && (u[i * M + k] > u[i * M + j] || (u[i * M + k] == u[i * M + j] && k > j));
             if (heavier >= N) { pruned |= 1ull << (i * M + j); load += 1u << (4 * j); }
-            if (heavier == N) st128(spot + i * T, -edge_cost128(u[i * M + j], Emin, i * M + j));   // reduced cost c + pot[row] - pot[col]: <= 0 pruned, >= 0 kept
+            if (heavier == N) A::st(base, A::kPot, i, T, -A::cost(base, i * M + j, T, Emin));   // reduced cost c + pot[row] - pot[col]: <= 0 pruned, >= 0 kept
         }
     }
     bool failed = false;
     for (int unit = 0; unit <= M * P; ++unit) {
         unsigned reach = 0, done = 0;
-        uint64_t pre = 0;                                               // nibble n: predecessor of node n
+        uint32_t pre_r = 0, pre_c = 0;                                  // nibble k: predecessor of row node k / column node k
 #pragma unroll
         for (int j = 0; j < M; ++j) {
             const bool over = enabled && !failed && (int)((load >> (4 * j)) & 15u) > P;
-            if (over) st128(sdist + (M + j) * T, 0);
+            if (over) A::st(base, A::kDist, M + j, T, 0);
             reach |= (over ? 1u : 0u) << (M + j);
         }
         const unsigned sources = reach;
@@ -540,10 +618,10 @@ __device__ __noinline__ uint64_t exact_flow_warp(const uint32_t (&u)[M * M], int
             if (!__any_sync(kFull, searching)) break;
             // settle the open node at the smallest distance
             const unsigned open = searching ? (reach & ~done) : 0u;
-            int v = -1; __int128 dv = 0;
+            int v = -1; V dv = 0;
 #pragma unroll
             for (int n = 0; n < 2 * M; ++n) {
-                const __int128 d = ld128(sdist + n * T);
+                const V d = A::ld(base, A::kDist, n, T);
                 const bool better = ((open >> n) & 1) && (v < 0 || d < dv);
                 v = better ? n : v; dv = better ? d : dv;
             }
@@ -551,35 +629,48 @@ __device__ __noinline__ uint64_t exact_flow_warp(const uint32_t (&u)[M * M], int
             const int vv = has ? v : 0;
             done |= has ? (1u << vv) : 0u;
             const bool iscol = vv >= M;
-            const bool hit = has && iscol && (int)((load >> (4 * (vv & (M - 1)))) & 15u) < P;
+            const int line = iscol ? vv - M : vv;                       // the settled node's column or row
+            const bool hit = has && iscol && (int)((load >> (4 * line)) & 15u) < P;
             target = hit ? vv : target;
             const bool relax = has && !hit;
-            // relax its M arcs: a column un-prunes one of its pruned entries, a row prunes one more of its kept ones
-            const __int128 base = dv + ld128(spot + vv * T);
+            // relax its M arcs: a column un-prunes one of its pruned entries, a row prunes one more of its kept ones.
+            // Arc k leads to row k (from a column) or to column k (from a row): everything that depends on k alone is a
+            // constant offset from what is worked out once per step.
+            const V from = dv + A::ld(base, A::kPot, vv, T);
+            const uint64_t flags = pruned >> (iscol ? line : line * M); // arc k's pruned flag at bit k*M (column) or k (row)
+            FlowCell* const costs = cell(base, A::kCost, T) + (size_t)(iscol ? line : line * M) * (A::kTieFree ? T : 0);
+            const unsigned reached = iscol ? reach : reach >> M, settled = iscol ? done : done >> M;
+            unsigned taken = 0, spread = 0;                             // arcs that reached or improved their node: bit k / bit 4k
 #pragma unroll
             for (int k = 0; k < M; ++k) {
-                const int nb = iscol ? k : M + k;
-                const int p = iscol ? k * M + (vv - M) : vv * M + k;
-                const bool is_pruned = (pruned >> p) & 1;
-                const bool elig = relax && (is_pruned == iscol) && !((done >> nb) & 1);
-                const __int128 c = edge_cost128(su[p * T], Emin, p);
-                const __int128 nd = base - ld128(spot + nb * T) + (iscol ? -c : c);
-                const bool better = elig && (!((reach >> nb) & 1) || nd < ld128(sdist + nb * T));
-                if (better) st128(sdist + nb * T, nd);
-                pre = better ? ((pre & ~(15ull << (4 * nb))) | ((uint64_t)vv << (4 * nb))) : pre;
-                reach |= (better ? 1u : 0u) << nb;
+                const bool is_pruned = ((iscol ? flags >> (k * M) : flags >> k) & 1) != 0;
+                const bool elig = relax && (is_pruned == iscol) && !((settled >> k) & 1);
+                const int p = iscol ? k * M + line : line * M + k;
+                const V c = A::kTieFree ? (V)*(iscol ? costs + (size_t)k * M * T : costs + (size_t)k * T) : A::cost(base, p, T, Emin);
+                FlowCell* const potk = iscol ? cell(base, A::kPot + A::kCells * k, T) : cell(base, A::kPot + A::kCells * (M + k), T);
+                FlowCell* const distk = iscol ? cell(base, A::kDist + A::kCells * k, T) : cell(base, A::kDist + A::kCells * (M + k), T);
+                const V nd = from - A::ldp(potk, T) + (iscol ? -c : c);
+                const bool better = elig && (!((reached >> k) & 1) || nd < A::ldp(distk, T));
+                if (better) A::stp(distk, T, nd);
+                taken |= (better ? 1u : 0u) << k;
+                spread |= (better ? 1u : 0u) << (4 * k);
             }
+            // their predecessor is the settled node
+            const uint32_t mask = spread * 15u, fill = spread * (uint32_t)vv;
+            pre_r = iscol ? ((pre_r & ~mask) | fill) : pre_r;
+            pre_c = iscol ? pre_c : ((pre_c & ~mask) | fill);
+            reach |= iscol ? taken : taken << M;
         }
         const bool ok = active && target >= 0;
         failed |= active && target < 0;
         // potentials: settled nodes closer than the target move by their distance, all others by the target's
         const int tt = ok ? target : M;
-        const __int128 D = ld128(sdist + tt * T);
+        const V D = A::ld(base, A::kDist, tt, T);
 #pragma unroll
         for (int n = 0; n < 2 * M; ++n) {
-            const __int128 d = ld128(sdist + n * T);
-            const __int128 add = (((done >> n) & 1) && d < D) ? d : D;
-            if (ok) st128(spot + n * T, ld128(spot + n * T) + add);
+            const V d = A::ld(base, A::kDist, n, T);
+            const V add = (((done >> n) & 1) && d < D) ? d : D;
+            if (ok) A::st(base, A::kPot, n, T, A::ld(base, A::kPot, n, T) + add);
         }
         // flip the arcs of the path back to its source column
         int v = tt;
@@ -588,7 +679,7 @@ __device__ __noinline__ uint64_t exact_flow_warp(const uint32_t (&u)[M * M], int
         for (int s = 0; s < 2 * M + 2; ++s) {
             const bool go = ok && !((sources >> v) & 1);
             if (!__any_sync(kFull, go)) break;
-            const int w = (int)((pre >> (4 * v)) & 15u);
+            const int w = (int)(((v >= M ? pre_c >> (4 * (v - M)) : pre_r >> (4 * v))) & 15u);
             const uint64_t bit = v >= M ? (1ull << ((w & (M - 1)) * M + (v - M))) : (1ull << (v * M + (w & (M - 1))));
             pruned = go ? (v >= M ? (pruned | bit) : (pruned & ~bit)) : pruned;     // row w -> column v-M prunes; column w-M -> row v un-prunes
             v = go ? w : v;
@@ -598,20 +689,44 @@ __device__ __noinline__ uint64_t exact_flow_warp(const uint32_t (&u)[M * M], int
         failed |= ok && !home;
     }
     if (failed) status |= kDevInternal;
+    if constexpr (A::kTieFree) {
+        // the entries of reduced cost zero under the final potentials
+        V pr[M], pc[M];
+#pragma unroll
+        for (int i = 0; i < M; ++i) { pr[i] = A::ld(base, A::kPot, i, T); pc[i] = A::ld(base, A::kPot, M + i, T); }
+        uint64_t tight = 0;
+#pragma unroll
+        for (int i = 0; i < M; ++i)
+#pragma unroll
+            for (int j = 0; j < M; ++j)
+                tight |= (A::cost(base, i * M + j, T, Emin) + pr[i] == pc[j]) ? (1ull << (i * M + j)) : 0ull;
+        const bool forest = tight_forest<M>(enabled ? tight : 0ull);
+        *certified = enabled && !failed && forest;
+    }
     const uint64_t all = (M == 8) ? ~0ull : ((1ull << (M * M)) - 1);
     return ~pruned & all;
 }
 
-// Called by all 32 lanes of a warp.
-template <int N, int M>
-__device__ __forceinline__ uint64_t exact_ssp(const uint32_t (&u)[M * M], int& status, uint32_t* su, uint4* spot, uint4* sdist, int T) {
+// Called by all 32 lanes of a warp.  flow_smem: the CTA's region of flow_shared_bytes_per_thread(M) bytes per thread, T =
+// threads per CTA (a constant, so that every cell offset is one), tid = this thread; live: the lane holds a block of the matrix (the others only keep the votes whole).
+template <int N, int M, int T>
+__device__ __forceinline__ uint64_t exact_ssp(const uint32_t (&u)[M * M], int& status, unsigned char* flow_smem, int tid, bool live) {
     int Emin, Emax;
     if (!exponent_range<M * M>(u, Emin, Emax)) { Emin = 1; Emax = 1; }
     // 128-bit costs: 64 tie bits + 24 significand bits + spread; paths (<= 2M arcs) and potentials (<= M(M-N)
     // updates) add 4 + 5 bits, the sign one more; beyond that the block takes the wide integers, on its own
     const bool wide = Emax - Emin > 26;
-    uint64_t kept = exact_flow_warp<N, M>(u, Emin, !wide, status, su, spot, sdist, T);
-    if (wide) kept = exact_flow_run<CostWide, N, M>(u, Emin, status);
+    FlowCell* base = reinterpret_cast<FlowCell*>(flow_smem) + tid;
+    // first without the tie term, in 64-bit words
+    bool certified = false;
+    uint64_t kept = exact_flow_warp<Flow64<M>, N, M, T>(u, Emin, live && !wide, status, base, &certified);
+    // blocks whose optimum is not certified unique (magnitude ties, as a rule): the full costs decide
+    const bool again = live && !wide && !certified;
+    if (__any_sync(0xFFFFFFFFu, again)) {
+        const uint64_t k2 = exact_flow_warp<Flow128<M>, N, M, T>(u, Emin, again, status, base, nullptr);
+        kept = again ? k2 : kept;
+    }
+    if (live && wide) kept = exact_flow_run<CostWide, N, M>(u, Emin, status);
     return kept;
 }
 
