@@ -333,15 +333,23 @@ __device__ __forceinline__ uint32_t shared_column_case32(const uint32_t (&v)[4][
     constexpr int ca = pair_index(C, a), cb = pair_index(C, b), da = pair_index(D, a), db = pair_index(D, b);
     return max(v[0][ca] + v[1][cb], v[0][cb] + v[1][ca]) + max(v[2][da] + v[3][db], v[2][db] + v[3][da]);
 }
+// SCALED: Emin >= 19 (all entries normal numbers or zero), so the integer image is a product: |w| * 2^(146 - Emin) is the
+// integer q * 2^12 (at most 29 bits, exact in fp32), one multiplication and one conversion off the logic pipe per entry.
+template <bool SCALED>
 __device__ __forceinline__ uint64_t exact_2_4_classes32(const uint32_t (&u)[16], int Emin) {
     uint32_t v[4][6];
+    const float scale = __uint_as_float((uint32_t)(127 + 146 - Emin) << 23);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         uint32_t q[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            uint32_t sig; int E; split_float(u[i * 4 + j], sig, E);
-            q[j] = sig ? ((sig >> 16) << (E - Emin + 12)) : 0u;
+            if constexpr (SCALED) {
+                q[j] = __float2uint_rz(__uint_as_float(u[i * 4 + j]) * scale);
+            } else {
+                uint32_t sig; int E; split_float(u[i * 4 + j], sig, E);
+                q[j] = sig ? ((sig >> 16) << (E - Emin + 12)) : 0u;
+            }
         }
 #pragma unroll
         for (int b = 1; b < 4; ++b)
@@ -371,10 +379,20 @@ __device__ __forceinline__ uint64_t exact_2_4_classes32(const uint32_t (&u)[16],
 // drop_bits: low significand bits known to be zero in every entry (16 for widened bf16 inputs).
 // Called by all 32 lanes of a warp (the 32-bit scorer is taken when every lane's block fits it).
 __device__ __forceinline__ uint64_t exact_2_4(const uint32_t (&u)[16], int drop_bits) {
+    if (drop_bits == 16) {
+        // bf16 data, the common case first: exponent range from the largest and the smallest non-zero pattern (u - 1 sends
+        // zero to the top), no per-entry unpacking
+        uint32_t umax = 0, umin1 = 0xFFFFFFFFu;
+#pragma unroll
+        for (int p = 0; p < 16; ++p) { umax = max(umax, u[p]); umin1 = min(umin1, u[p] - 1u); }
+        const int emax = (int)(umax >> 23), emin = (int)((umin1 + 1u) >> 23);
+        const bool fits = umax == 0u || (emin >= 19 && emax - emin <= 9);      // all zero: every sum is 0, the largest code wins
+        if (__all_sync(0xFFFFFFFFu, fits)) return exact_2_4_classes32<true>(u, umax ? emin : 127);
+    }
     int Emin, Emax;
     if (!exponent_range<16>(u, Emin, Emax)) { Emin = 1; Emax = 1; }     // all zero: every sum is 0, the largest code wins
     const int spread = Emax - Emin;
-    if (__all_sync(0xFFFFFFFFu, drop_bits == 16 && spread <= 9)) return exact_2_4_classes32(u, Emin);
+    if (__all_sync(0xFFFFFFFFu, drop_bits == 16 && spread <= 9)) return exact_2_4_classes32<false>(u, Emin);
     // (24 - drop) significand bits + spread + 3 bits for eight terms + 16 code bits must stay below 2^63
     if (spread <= 19 + drop_bits) return exact_2_4_classes(u, Emin, drop_bits);
     if (spread <= 34) return exact_2_4_int64(u, Emin);
