@@ -32,10 +32,11 @@ FULL_ROWS, COLS = 12288, 49152
 ROWS = FULL_ROWS
 N_KEEP, M_BLOCK = 2, 4
 BYTES_PER_WEIGHT = 2 + 2 + 1.0 / 8          # read W, write masked W, write one mask bit (bf16)
-# dram__bytes_read.sum + dram__bytes_write.sum of the search kernel, from an ncu capture (see profiles/); None until the
-# counters have been taken again for the kernel as it stands
-TRAFFIC_BYTES_PER_LAUNCH = None
-TRAFFIC_SOURCE = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch of the search kernel in steady state (mean of four
+# consecutive launches, caches not flushed between them); None when the kernel has changed since the counters were taken
+TRAFFIC_BYTES_PER_LAUNCH = 1208.02e6 + 1282.56e6
+TRAFFIC_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --cache-control none on the full-size launch "
+                  "(profiles/tma24_kernel_approx_2_4_bf16_12288x49152_launches.md)")
 METRIC = "transposable-mask weights/s (2:4 approx, bf16, 1 GPU: achieved HBM GB/s vs peak in `roofline`)"
 WORKLOAD = "%dx49152 bf16, N(0,0.02) quantised to 256 levels (frequent ties), 2:4 approximate, per-step recompute"
 

@@ -405,6 +405,13 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             if (__any_sync(0xFFFFFFFFu, watch != watch)) relations48_f32(blk, rel, worst);       // integer keys, bit-pattern order
             else relations48_f32_arith(f, rel);
         }
+        // refill the stage of the previous item -- its store, issued one item ago, has long been read -- so that the copy
+        // runs under the rest of this item
+        if (loaded < n_items) {
+            if constexpr (HAS_OUT) { if (lane == 0 && it > 0) tma_wait_read<0>(); }
+            __syncwarp();
+            issue_next();
+        }
         u64 kept = cover_4_8(rel);
         if constexpr (METHOD == kMethodApprox) {
             Short48 L = line_short(kept);
@@ -464,12 +471,6 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             const int idx = lane + 32 * h, row = idx >> 3, word = cur.cj * 8 + (idx & 7);
             const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + row * 32 + (idx & 7) * 4);
             if (word < p_wpr) p_mask[((long long)cur.bi * kRows8 + row) * p_wpr + word] = w;
-        }
-        // refill: the stage of the previous item is free once its store has been read
-        if (loaded < n_items) {
-            if constexpr (HAS_OUT) { if (lane == 0) tma_wait_read<1>(); }
-            __syncwarp();
-            issue_next();
         }
         cur.advance(tab, count);
         if ((it & 15) == 15) { acc += (double)facc; facc = 0.f; }           // keep the fp32 partial short
