@@ -165,7 +165,7 @@ int build_plan(const tm_problem* probs, int count, int N, int M, int method, voi
             pg.entry_store.resize(esz * (size_t)n + 128);
             pg.entries = pg.entry_store.data() + ((128 - (uintptr_t)pg.entry_store.data() % 128) % 128);
             long long total = 0;
-            if (!tmask::tma_build_entries(group[g].data(), n, pg.entries, &total, M)) return TM_ERR_CUDA;
+            if (!tmask::tma_build_entries(group[g].data(), n, pg.entries, &total, M, method)) return TM_ERR_CUDA;
             tmask::TmaLaunch& a = pg.bandwidth;
             a.entries_host = pg.entries; a.count = n; a.total_items = total; a.partials = partials;
             a.status = nullptr; a.dtype = (g - 1) / 2; a.method = method; a.M = M; a.has_out = ((g - 1) & 1) != 0; a.stream = nullptr;
@@ -516,7 +516,7 @@ int tm_nm_mask_1d(const tm_problem* prob_host, int N, int M, int flags, unsigned
         if (tmask::tma_eligible(dp, N, 4, tmask::kMethodRows)) {
             alignas(128) unsigned char entry[512];
             long long total = 0;
-            if (tmask::tma_entry_bytes() <= sizeof(entry) && tmask::tma_build_entries(&dp, 1, entry, &total, 4)) {
+            if (tmask::tma_entry_bytes() <= sizeof(entry) && tmask::tma_build_entries(&dp, 1, entry, &total, 4, tmask::kMethodRows)) {
                 tmask::TmaLaunch t;
                 t.entries_host = entry; t.entries_dev = nullptr; t.count = 1; t.total_items = total; t.partials = op; t.status = status_dev;
                 t.dtype = p.dtype; t.M = 4; t.has_out = p.masked_w_out != nullptr;

@@ -580,10 +580,10 @@ bool tma_eligible(const DevProblem& p, int N, int M, int method) {
     return encode_fn() != nullptr;
 }
 
-// Fills `entries_host` (count TmaEntry records) for problems that all passed tma_eligible(); an item is one block row
-// of 4 x 512 (M = 4) or 8 x 256 (M = 8) elements.
-bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M) {
-    if (M == 8) return build_entries(probs, count, static_cast<TmaEntry*>(entries_host), total_items, 8, 256);
+// Fills `entries_host` (count TmaEntry records) for problems that all passed tma_eligible() and share a dtype; an item is
+// one block row of 4 x 512 (M = 4) or 8 x 256 (M = 8; 8 x 128 where fp32 runs the split kernel) elements.
+bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M, int method) {
+    if (M == 8) return build_entries(probs, count, static_cast<TmaEntry*>(entries_host), total_items, 8, tma48_item_cols(count > 0 ? probs[0].dtype : kF32, method));
     return build_entries(probs, count, static_cast<TmaEntry*>(entries_host), total_items, kItemRows, kItemCols);
 }
 

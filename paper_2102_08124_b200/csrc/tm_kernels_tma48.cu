@@ -213,14 +213,6 @@ __device__ __forceinline__ void relations48_f32_arith(const float (&f)[64], Rel4
     complete_relations8(rel);
 }
 
-// Keep flags of a row of eight fp32 entries as eight words of 0 or 1: entry e of the 256-entry table (two 16-byte halves).
-__device__ __forceinline__ void fill_keep_lut32(uint4* lut, int tid, int nthreads) {
-    for (int e = tid; e < 256; e += nthreads) {
-        lut[2 * e] = make_uint4(e & 1, (e >> 1) & 1, (e >> 2) & 1, (e >> 3) & 1);
-        lut[2 * e + 1] = make_uint4((e >> 4) & 1, (e >> 5) & 1, (e >> 6) & 1, (e >> 7) & 1);
-    }
-}
-
 // magnitude pattern of entry p of the lane's block, read back from the stage
 template <int DT>
 __device__ __forceinline__ uint32_t key_at(const unsigned char* blk, int p) {
@@ -502,7 +494,12 @@ cudaError_t launch_one48(const TmaLaunch& a, const TmaEntry& single, const TmaEn
 
 }  // namespace
 
+// fp32 with the full search runs on the kernel that splits a block over two lanes (tm_kernels_tma48s.cu)
+static bool takes_split_kernel(int dtype, int method) { return dtype == kF32 && method == kMethodApprox; }
+int tma48_item_cols(int dtype, int method) { return takes_split_kernel(dtype, method) ? tma48s_item_cols() : kCols8; }
+
 int tma48_warps_per_cta(int dtype, int method) {
+    if (takes_split_kernel(dtype, method)) return tma48s_warps_per_cta();
     if (method == kMethodApprox) return dtype == kF32 ? Geo48<kF32, kMethodApprox>::kWarps : Geo48<kBF16, kMethodApprox>::kWarps;
     return dtype == kF32 ? Geo48<kF32, kMethodCover>::kWarps : Geo48<kBF16, kMethodCover>::kWarps;
 }
@@ -516,7 +513,8 @@ cudaError_t launch_tma48(const TmaLaunch& a) {
     if (a.total_items > 0) {
 #define TM_DISPATCH(DT, METHOD)                                                                                   \
     err = a.has_out ? launch_one48<DT, METHOD, true>(a, host[0], table) : launch_one48<DT, METHOD, false>(a, host[0], table)
-        if (a.dtype == kF32) { if (a.method == kMethodApprox) TM_DISPATCH(kF32, kMethodApprox); else TM_DISPATCH(kF32, kMethodCover); }
+        if (takes_split_kernel(a.dtype, a.method)) err = launch_tma48s(a);
+        else if (a.dtype == kF32) TM_DISPATCH(kF32, kMethodCover);
         else { if (a.method == kMethodApprox) TM_DISPATCH(kBF16, kMethodApprox); else TM_DISPATCH(kBF16, kMethodCover); }
 #undef TM_DISPATCH
         if (err != cudaSuccess) return err;

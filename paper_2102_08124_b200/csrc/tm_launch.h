@@ -58,11 +58,16 @@ struct TmaLaunch {
 size_t tma_entry_bytes();
 int tma_warps_per_cta(int dtype, int M, int method);
 bool tma_eligible(const DevProblem& p, int N, int M, int method);
-bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M);
+bool tma_build_entries(const DevProblem* probs, int count, void* entries_host, long long* total_items, int M, int method);
 cudaError_t tma_reduce(const void* entries_host, const void* entries_dev, int count, const double* partials, long long stride, cudaStream_t stream);
 // 4:8 variant (tm_kernels_tma48.cu), reached through launch_tma()
 int tma48_warps_per_cta(int dtype, int method);
+int tma48_item_cols(int dtype, int method);
 cudaError_t launch_tma48(const TmaLaunch& a);
+// the same search for fp32 with a block split over two lanes (tm_kernels_tma48s.cu), reached through launch_tma48()
+int tma48s_warps_per_cta();
+int tma48s_item_cols();
+cudaError_t launch_tma48s(const TmaLaunch& a);
 cudaError_t launch_tma(const TmaLaunch& a);
 
 

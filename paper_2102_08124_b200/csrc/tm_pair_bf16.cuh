@@ -155,6 +155,14 @@ __device__ __forceinline__ void fill_lane_lut(uint4* lut, int tid, int nthreads)
     }
 }
 
+// Keep flags of a row of eight fp32 entries as eight words of 0 or 1: entry e of the 256-entry table (two 16-byte halves).
+__device__ __forceinline__ void fill_keep_lut32(uint4* lut, int tid, int nthreads) {
+    for (int e = tid; e < 256; e += nthreads) {
+        lut[2 * e] = make_uint4(e & 1, (e >> 1) & 1, (e >> 2) & 1, (e >> 3) & 1);
+        lut[2 * e + 1] = make_uint4((e >> 4) & 1, (e >> 5) & 1, (e >> 6) & 1, (e >> 7) & 1);
+    }
+}
+
 // The four mask bytes of a pair mask, byte i = (row i of block B) << 4 | (row i of block A): the layout
 // of the packed mask for the thread's eight columns.
 __device__ __forceinline__ uint32_t mask_bytes_2_4(uint32_t kept) {
