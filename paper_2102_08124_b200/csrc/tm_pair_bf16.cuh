@@ -85,14 +85,29 @@ template <bool ARITH> __device__ __forceinline__ uint32_t earlier_heavier(uint32
 // byte 0/1 <- decisions of dx/dy for block A, byte 2/3 <- for block B; every byte is 0x00 or 0xFF
 __device__ __forceinline__ uint32_t pick(uint32_t dx, uint32_t dy) { return prmt(dx, dy, 0xFBD9); }
 
-// p[b] (bytes of equal bits) carries the decision destined for bit 7-b of every byte, negated where bit b of NEG is set
+// p[b] (bytes of equal bits) carries the decision destined for bit 7-b of every byte, negated where bit b of NEG is set.
+// As an integer, a word of 0x00 / 0xFF bytes is 255 times the word of 0 / 1 bytes, so the weighted sum 128 p[0] + 64 p[1] +
+// ... + p[7] is 255 times the gathered word (modulo 2^32, carries between bytes and all), and the factor leaves by a
+// multiplication with the inverse of 255 modulo 2^32, -0x01010101: eight integer multiply-adds on the multiply-add pipe,
+// which has room, instead of seven bit selects on the logic pipe, which has none.  The factors sit in constant memory so
+// that the compiler keeps the multiply-adds.
+__constant__ uint32_t g_gather_mul[2] = {2u, 0xFEFEFEFFu};
+__device__ __forceinline__ uint32_t imad(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t r;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    return r;
+}
 template <unsigned NEG>
 __device__ __forceinline__ uint32_t gather8(const uint32_t (&p)[8]) {
-    const uint32_t t01 = bitsel_n<(NEG & 1) != 0, (NEG & 2) != 0>(p[0], p[1], 0x80808080u);
-    const uint32_t t23 = bitsel_n<(NEG & 4) != 0, (NEG & 8) != 0>(p[2], p[3], 0x20202020u);
-    const uint32_t t45 = bitsel_n<(NEG & 16) != 0, (NEG & 32) != 0>(p[4], p[5], 0x08080808u);
-    const uint32_t t67 = bitsel_n<(NEG & 64) != 0, (NEG & 128) != 0>(p[6], p[7], 0x02020202u);
-    return bitsel(bitsel(t01, t23, 0xC0C0C0C0u), bitsel(t45, t67, 0x0C0C0C0Cu), 0xF0F0F0F0u);
+    const uint32_t two = g_gather_mul[0];
+    uint32_t acc = imad(p[0], two, p[1]);
+#pragma unroll
+    for (int b = 2; b < 8; ++b) acc = imad(acc, two, p[b]);
+    acc *= g_gather_mul[1];
+    uint32_t turn = 0;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) turn |= ((NEG >> b) & 1u) ? (0x01010101u << (7 - b)) : 0u;
+    return NEG ? acc ^ turn : acc;
 }
 
 template <bool ARITH>
