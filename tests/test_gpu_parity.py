@@ -271,6 +271,14 @@ def test_batched_4_8():
     mats = [workloads.laplace_f32(32, 264, 0.05, 31), workloads.normal_bf16(16, 520, 0.02, 32)]
     for method in METHODS:
         _batched_parity(mats, 4, 8, method)
+    # fp32 with the full search runs on the kernel that splits a block over two lanes (items of 8 x 128): many small
+    # matrices in one call, ragged last items, rows inside a wider buffer, ties everywhere
+    rng = np.random.Generator(np.random.PCG64(33))
+    small = [workloads.laplace_f32(8 * (1 + k % 4), 8 * (1 + (k * 13) % 61), 0.05, 340 + k) for k in range(40)]
+    small.append(rng.integers(-2, 3, size=(24, 392)).astype(np.float32))
+    small.append(np.zeros((8, 136), np.float32))
+    _batched_parity(small, 4, 8, tm.TM_APPROX)
+    _batched_parity(small, 4, 8, tm.TM_APPROX, strided=True)
 
 
 def test_config2_whole_model_approx():
