@@ -283,19 +283,10 @@ __device__ __forceinline__ uint32_t pair_nibble(uint32_t m) {
     return (uint32_t)(kTable >> (4 * m)) & 0xFu;
 }
 
-// STAGED (bf16, 16-byte aligned rows of W and of the mask): the 128 x 128 tile of W and its 128 x 4 mask words arrive by
-// bulk-tensor copies into one of two shared-memory stages, the next tile's while this one is packed, so that no warp waits
-// for its own global loads; otherwise every thread loads its rows itself.
-constexpr int kStageW = 128 * 128 * 2, kStageM = 128 * 16, kStageBytes = kStageW + kStageM;
-
-template <int DT, bool STAGED>
+template <int DT>
 __global__ void __launch_bounds__(256)
 compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __restrict__ meta, void* __restrict__ values_t,
-                  uint32_t* __restrict__ meta_t, int* __restrict__ status_out, const __grid_constant__ CUtensorMap wmap,
-                  const __grid_constant__ CUtensorMap mmap) {
-    static_assert(!STAGED || DT == kBF16, "the staged variant is the bf16 one");
-    extern __shared__ __align__(1024) unsigned char stages[];     // STAGED: two stages of kStageBytes
-    __shared__ __align__(8) uint64_t bars[2];
+                  uint32_t* __restrict__ meta_t, int* __restrict__ status_out) {
     constexpr int kVW = DT == kF32 ? 2 : 1;             // words per kept pair
     constexpr int kPitch = 32 * kVW + 1;
     __shared__ uint32_t tile_t[128 * kPitch];
@@ -316,32 +307,10 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
     const long long wpr_t = (P.rows + 31) / 32, half_c = P.cols / 2, half_r = P.rows / 2;
     const size_t ebytes = DT == kF32 ? 4 : 2;
     const bool vec_t = (uintptr_t)values_t % 16 == 0 && ((size_t)half_r * ebytes) % 16 == 0;
-    bool bad = false, lost = false;
-    auto issue = [&](long long t, int s) {                 // thread 0: both copies of tile t into stage s
-        const long long tr = t / tiles_c, tc = t - tr * tiles_c;
-        mbar_expect_tx(&bars[s], kStageBytes);
-        tma_load_2d(stages + s * kStageBytes, &wmap, (int)(tc * 128), (int)(tr * 128), &bars[s]);
-        tma_load_2d(stages + s * kStageBytes + kStageW, &mmap, (int)(tc * 4), (int)(tr * 128), &bars[s]);
-    };
-    if constexpr (STAGED) {
-        if (threadIdx.x == 0) {
-            mbar_init(&bars[0], 1); mbar_init(&bars[1], 1);
-            fence_mbar_init();
-            if ((long long)blockIdx.x < tiles_r * tiles_c) issue(blockIdx.x, 0);
-        }
-        __syncthreads();
-    }
-    int iter = 0;
-    for (long long t = blockIdx.x; t < tiles_r * tiles_c; t += gridDim.x, ++iter) {
+    bool bad = false;
+    for (long long t = blockIdx.x; t < tiles_r * tiles_c; t += gridDim.x) {
         const long long tr = t / tiles_c, tc = t - tr * tiles_c;
         const long long c0 = tc * 128 + lane * 4;
-        const unsigned char* stage = stages + (iter & 1) * kStageBytes;
-        if constexpr (STAGED) {
-            // the other stage was last read before the barrier that ended the previous tile
-            if (threadIdx.x == 0 && t + gridDim.x < tiles_r * tiles_c) issue(t + gridDim.x, (iter & 1) ^ 1);
-            if (!mbar_wait_bounded(&bars[iter & 1], (uint32_t)((iter >> 1) & 1))) lost = true;
-            if (__syncthreads_or(lost ? 1 : 0)) break;   // a copy that never landed: stop before packing an unfilled stage
-        }
         uint32_t col_nibbles[4] = {0, 0, 0, 0};      // nibble `it` = metadata of column j in block row 4 * warp + it
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
@@ -350,15 +319,7 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
             const bool active = r0 < P.rows && c0 < P.cols;
             uint32_t v[4][4] = {}, mbits = 0;            // mbits bit 4i+j = mask of (row i, column j)
             uint2 raw[4] = {};                           // bf16: the row's four values as loaded
-            if constexpr (STAGED) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    raw[i] = *reinterpret_cast<const uint2*>(stage + (br * 4 + i) * 256 + lane * 8);
-                    const uint32_t word = *reinterpret_cast<const uint32_t*>(stage + kStageW + (br * 4 + i) * 16 + (lane >> 3) * 4);
-                    mbits |= ((word >> (4 * (lane & 7))) & 0xFu) << (4 * i);
-                }
-                if (!active) mbits = 0;
-            } else if (active) {
+            if (active) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if constexpr (DT == kF32) {
@@ -456,11 +417,6 @@ compress24_kernel(const AuxProblem P, void* __restrict__ values, uint32_t* __res
         __syncthreads();
     }
     if (bad && status_out) atomicOr(status_out, kDevBadMask);
-    if constexpr (STAGED) {
-        if (lost && status_out) atomicOr(status_out, kDevInternal);
-        // a copy may still be in flight when the loop ended early: give it a bounded chance to land before the stages die
-        if (lost && threadIdx.x == 0) { mbar_wait_bounded(&bars[0], 0, 1u << 14); mbar_wait_bounded(&bars[0], 1, 1u << 14); mbar_wait_bounded(&bars[1], 0, 1u << 14); mbar_wait_bounded(&bars[1], 1, 1u << 14); }
-    }
 }
 
 }  // namespace
@@ -519,33 +475,11 @@ cudaError_t launch_compress24(const AuxProblem& P, void* values, uint32_t* meta,
                               int sms, cudaStream_t stream) {
     const long long tiles = ((P.rows + 127) / 128) * ((P.cols + 127) / 128);
     if (tiles == 0) return cudaSuccess;
-    CUtensorMap wmap, mmap;
-    memset(&wmap, 0, sizeof wmap); memset(&mmap, 0, sizeof mmap);
-    // staged variant: bf16, rows of W and of the mask on 16-byte boundaries, sizes within the tensor maps' 32-bit coordinates
-    bool staged = P.dtype == kBF16 && (uintptr_t)P.W % 16 == 0 && ((size_t)P.ld * 2) % 16 == 0 && (uintptr_t)P.mask % 16 == 0 && P.wpr % 4 == 0 &&
-                  P.rows < (1ll << 31) && P.cols < (1ll << 31) && encode_fn() != nullptr;
-    if (staged) {
-        EncodeTiledFn fn = encode_fn();
-        const cuuint64_t wd[2] = {(cuuint64_t)P.cols, (cuuint64_t)P.rows}, ws[1] = {(cuuint64_t)P.ld * 2};
-        const cuuint64_t md[2] = {(cuuint64_t)P.wpr, (cuuint64_t)P.rows}, ms[1] = {(cuuint64_t)P.wpr * 4};
-        const cuuint32_t wb[2] = {128, 128}, mb[2] = {4, 128}, es[2] = {1, 1};
-        staged = fn(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(P.W), wd, ws, wb, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS &&
-                 fn(&mmap, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, P.mask, md, ms, mb, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-    }
-    if (staged) {
-        constexpr int smem = 2 * kStageBytes;
-        static PerDeviceOnce configured;
-        const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(compress24_kernel<kBF16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); });
-        if (e != cudaSuccess) return e;
-        const int grid = (int)(tiles < (long long)sms * 2 ? tiles : (long long)sms * 2);
-        compress24_kernel<kBF16, true><<<grid, 256, smem, stream>>>(P, values, meta, values_t, meta_t, status, wmap, mmap);
-        return cudaGetLastError();
-    }
+    // bf16 matrices with 16-byte aligned rows and mask rows stream through per-warp pipelines (tm_kernels_compress.cu)
+    if (compress24_stream_eligible(P, values, meta, meta_t)) return launch_compress24_stream(P, values, meta, values_t, meta_t, status, sms, stream);
     const int grid = (int)(tiles < (long long)sms * 8 ? tiles : (long long)sms * 8);
-    if (P.dtype == kF32) compress24_kernel<kF32, false><<<grid, 256, 0, stream>>>(P, values, meta, values_t, meta_t, status, wmap, mmap);
-    else compress24_kernel<kBF16, false><<<grid, 256, 0, stream>>>(P, values, meta, values_t, meta_t, status, wmap, mmap);
+    if (P.dtype == kF32) compress24_kernel<kF32><<<grid, 256, 0, stream>>>(P, values, meta, values_t, meta_t, status);
+    else compress24_kernel<kBF16><<<grid, 256, 0, stream>>>(P, values, meta, values_t, meta_t, status);
     return cudaGetLastError();
 }
 

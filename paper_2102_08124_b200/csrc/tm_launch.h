@@ -80,6 +80,10 @@ cudaError_t launch_nm1d(const AuxProblem& P, int N, int M, int flags, bool viola
                         int* status, int sms, cudaStream_t stream);
 cudaError_t launch_hamming(const uint32_t* a, const uint32_t* b, long long words, unsigned long long* partials, unsigned long long* out,
                            int sms, cudaStream_t stream);
+// the streaming form of the compression for bf16 matrices with 16-byte aligned rows and mask rows (tm_kernels_compress.cu)
+bool compress24_stream_eligible(const AuxProblem& P, const void* values, const void* meta, const void* meta_t);
+cudaError_t launch_compress24_stream(const AuxProblem& P, void* values, uint32_t* meta, void* values_t, uint32_t* meta_t, int* status,
+                                     int sms, cudaStream_t stream);
 cudaError_t launch_compress24(const AuxProblem& P, void* values, uint32_t* meta, void* values_t, uint32_t* meta_t, int* status,
                               int sms, cudaStream_t stream);
 

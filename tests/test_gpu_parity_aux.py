@@ -129,8 +129,11 @@ def test_mask_violations(dtype):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_compress_2_4(dtype):
-    # the last shape gives some CTAs of the staged bf16 variant a second tile (more tiles than twice the SM count) and a ragged last tile row
-    for rows, cols, seed in [(4, 4, 21), (36, 132, 22), (64, 512, 23), (100, 260, 24), (272, 384, 25), (2180, 2560, 26)]:
+    # bf16 shapes whose mask rows are multiples of 16 bytes take the streaming kernel (items of 32 rows x 128 columns): single
+    # and ragged items, rows that allow 16-byte stores of the column form (rows % 16 == 0) and of its metadata (rows % 128 == 0)
+    # and rows that do not, several items per warp down one column tile and across tiles
+    for rows, cols, seed in [(4, 4, 21), (36, 132, 22), (64, 512, 23), (100, 260, 24), (272, 384, 25), (2180, 2560, 26),
+                             (36, 128, 27), (512, 256, 28), (1024, 384, 29), (4096, 1280, 30), (1156, 3968, 32)]:
         W = _case(dtype, rows, cols, seed)
         Wd = to_device(W)
         fn = tm.tm_find_mask_bf16 if dtype == "bf16" else tm.tm_find_mask
@@ -153,3 +156,14 @@ def test_compress_2_4(dtype):
     want = orc.compress_2_4(W, to_host_bits(one_d))
     assert np.array_equal(to_host_bits(values_t), want["values_t"].view(np.uint32)) and np.array_equal(to_host_bits(meta_t), want["meta_t"])
     assert np.array_equal(to_host_bits(values), want["values"].view(np.uint32))
+    # the same through the streaming bf16 kernel: bad groups inside full items and inside a ragged one
+    for rows, cols in [(64, 256), (100, 128)]:
+        W = _case("bf16", rows, cols, 33); Wd = to_device(W)
+        one_d, _, _, _, _ = tm.tm_nm_mask_1d(Wd, 2, 4)
+        values, meta, values_t, meta_t, status = tm.tm_compress_2_4(Wd, one_d)
+        torch.cuda.synchronize()
+        assert int(status.item()) == tm.TM_DEV_BADMASK
+        want = orc.compress_2_4(W, to_host_bits(one_d))
+        assert want["bad_groups"] > 0
+        assert np.array_equal(to_host_bits(values_t), want["values_t"].view(np.uint16)) and np.array_equal(to_host_bits(meta_t), want["meta_t"])
+        assert np.array_equal(to_host_bits(values), want["values"].view(np.uint16)) and np.array_equal(to_host_bits(meta), want["meta"])
