@@ -84,6 +84,132 @@ __device__ __forceinline__ const DevProblem& find_problem(const DevProblem* tabl
     return table[k];
 }
 
+// The flow solver runs a warp's 32 blocks in lockstep: every lane waits for the block that needs the most augmenting
+// paths.  How many a block needs is known beforehand -- the units by which its columns exceed M - N once every row has
+// pruned its M - N lightest entries -- so the blocks of kSortItems consecutive work items are dealt to the solver's
+// rounds in the order of that number, and the 32 blocks of a round need about the same.
+constexpr int kSortItems = 8;
+constexpr int kSortBytesPerWarp = kSortItems * 32 * (8 + 1);          // a kept mask and an order entry per block
+
+template <int N, int M>
+__device__ __forceinline__ int repair_units(const uint32_t (&u)[M * M]) {
+    int load[M];
+#pragma unroll
+    for (int j = 0; j < M; ++j) load[j] = 0;
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+#pragma unroll
+        for (int j = 0; j < M; ++j) {
+            int heavier = 0;
+#pragma unroll
+            for (int k = 0; k < M; ++k)
+                heavier += (k != j) && (u[i * M + k] > u[i * M + j] || (u[i * M + k] == u[i * M + j] && k > j));
+            load[j] += heavier >= N ? 1 : 0;
+        }
+    }
+    int d = 0;
+#pragma unroll
+    for (int j = 0; j < M; ++j) d += max(0, load[j] - (M - N));
+    return d;
+}
+
+template <int M>
+__device__ __forceinline__ void magnitudes(const uint32_t (&w)[M * M], uint32_t (&u)[M * M], int& status) {
+    bool bad = false;
+#pragma unroll
+    for (int p = 0; p < M * M; ++p) { u[p] = w[p] & 0x7FFFFFFFu; bad |= (u[p] >> 23) == 0xFFu; }
+    if (bad) status |= kDevNonFinite;
+}
+
+// mask words of one work item: row i of the item spans M words; a lane's M bits sit at M * (lane % (32 / M))
+template <int M>
+__device__ __forceinline__ void store_mask_words(const DevProblem& P, long long row0, int chunk, int lane, uint64_t kept) {
+    constexpr int kLanesPerWord = 32 / M;          // lanes whose blocks share one mask word
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+        uint32_t bits = (uint32_t)((kept >> (i * M)) & ((1u << M) - 1)) << (M * (lane % kLanesPerWord));
+#pragma unroll
+        for (int o = 1; o < kLanesPerWord; o <<= 1) bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, o);
+        const int word = chunk * M + lane / kLanesPerWord;
+        if (lane % kLanesPerWord == 0 && word < P.wpr) P.mask[(row0 + i) * P.wpr + word] = bits;
+    }
+}
+
+// Items [item, item + n) of problem P (n <= kSortItems) through the flow solver; returns the lane's share of the objective.
+template <int N, int M>
+__device__ __forceinline__ double flow_group(const DevProblem& P, long long item, int n, unsigned char* flow_smem, unsigned char* sort_smem, int& status) {
+    const int lane = threadIdx.x & 31;
+    const unsigned lt = (1u << lane) - 1u;
+    uint64_t* keptbuf = reinterpret_cast<uint64_t*>(sort_smem);
+    unsigned char* order = sort_smem + kSortItems * 32 * 8;
+    const long long local0 = item - P.item_begin;
+    // ---- how many units each block needs ----
+    int need[kSortItems], dmax = -1;
+#pragma unroll
+    for (int r = 0; r < kSortItems; ++r) {
+        need[r] = -1;
+        if (r < n) {
+            const long long local = local0 + r, bi = local / P.chunks;
+            const int chunk = (int)(local - bi * P.chunks), bj = chunk * 32 + lane;
+            if (bj < P.bcols) {
+                uint32_t w[M * M], u[M * M];
+                int ignored = 0;
+                load_block<M>(P, bi * M, (long long)bj * M, true, w);
+                magnitudes<M>(w, u, ignored);
+                need[r] = repair_units<N, M>(u);
+            }
+        }
+        dmax = max(dmax, need[r]);
+    }
+    for (int o = 16; o; o >>= 1) dmax = max(dmax, __shfl_xor_sync(0xFFFFFFFFu, dmax, o));
+    // ---- the blocks in descending order of that number (a counting sort by warp votes) ----
+    int sorted = 0;
+    for (int v = dmax; v >= 0; --v) {
+#pragma unroll
+        for (int r = 0; r < kSortItems; ++r) {
+            const bool mine = need[r] == v;
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, mine);
+            if (mine) order[sorted + __popc(m & lt)] = (unsigned char)(r * 32 + lane);
+            sorted += __popc(m);
+        }
+    }
+    __syncwarp();
+    // ---- the solver, 32 blocks of about equal need at a time ----
+    double acc = 0.0;
+    for (int base = 0; base < sorted; base += 32) {
+        const bool live = base + lane < sorted;
+        const int id = live ? order[base + lane] : 0, r = id >> 5, l = id & 31;
+        const long long local = local0 + r, bi = local / P.chunks;
+        const int chunk = (int)(local - bi * P.chunks);
+        const long long row0 = bi * M, col0 = ((long long)chunk * 32 + l) * M;
+        uint32_t w[M * M], u[M * M];
+        load_block<M>(P, row0, col0, live, w);
+        magnitudes<M>(w, u, status);
+        uint64_t kept = exact_ssp<N, M, kWarpsPerCta * 32>(u, status, flow_smem, (int)threadIdx.x, live);
+        if (!live) kept = 0;
+        float sum = 0.f;
+#pragma unroll
+        for (int p = 0; p < M * M; ++p) sum += ((kept >> p) & 1) ? pattern_as_float(u[p]) : 0.f;
+        acc += (double)sum;
+        if (P.masked && live) {
+#pragma unroll
+            for (int p = 0; p < M * M; ++p) w[p] = ((kept >> p) & 1) ? w[p] : 0u;
+            store_block<M>(P, row0, col0, w);
+        }
+        if (live) keptbuf[id] = kept;
+    }
+    __syncwarp();
+    // ---- the items' mask words ----
+    for (int r = 0; r < n; ++r) {
+        const long long local = local0 + r, bi = local / P.chunks;
+        const int chunk = (int)(local - bi * P.chunks);
+        const uint64_t kept = chunk * 32 + lane < P.bcols ? keptbuf[r * 32 + lane] : 0ull;
+        store_mask_words<M>(P, bi * M, chunk, lane, kept);
+    }
+    __syncwarp();
+    return acc;
+}
+
 template <int N, int M, int METHOD>
 // the exact 2:4 scorer is register-hungry: two CTAs per SM cap it at 128 registers (its rare wide-integer path spills)
 __global__ void __launch_bounds__(kWarpsPerCta * 32, (METHOD == kMethodExact && M == 4 && N == 2) ? 2 : 1)
@@ -116,6 +242,7 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
         }
         k = n;
     }
+    constexpr bool kFlow = METHOD == kMethodExact && !(M == 4 && N == 2);
     for (long long item = begin; item < end; ++item) {
         const DevProblem& P = find_problem(tab, count, item, k);
         if (k != acc_k) {
@@ -124,6 +251,15 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
                 if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
             }
             acc = 0.0; acc_k = k;
+        }
+        if constexpr (kFlow) {
+            // a group of consecutive items of this problem at a time
+            const long long stop = k + 1 < count ? min(end, tab[k + 1].item_begin) : end;
+            const int n = (int)min((long long)kSortItems, stop - item);
+            unsigned char* sort_smem = flow_smem + (size_t)flow_shared_bytes_per_thread(M) * kWarpsPerCta * 32 + (threadIdx.x >> 5) * kSortBytesPerWarp;
+            acc += flow_group<N, M>(P, item, n, flow_smem, sort_smem, status);
+            item += n - 1;
+            continue;
         }
         const long long local = item - P.item_begin;
         const long long bi = local / P.chunks;
@@ -212,7 +348,7 @@ cudaError_t launch_nm(const LaunchArgs& a) {
     switch (a.method) {
     case kMethodExact: {
         // the flow solver (everything but 2:4) keeps its state in shared memory
-        constexpr size_t smem = (N == 2 && M == 4) ? 0 : (size_t)flow_shared_bytes_per_thread(M) * kWarpsPerCta * 32;
+        constexpr size_t smem = (N == 2 && M == 4) ? 0 : (size_t)flow_shared_bytes_per_thread(M) * kWarpsPerCta * 32 + (size_t)kSortBytesPerWarp * kWarpsPerCta;
         static PerDeviceOnce configured;   // per instantiation
         if (smem > 48 * 1024) {
             const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(generic_kernel<N, M, kMethodExact>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });
