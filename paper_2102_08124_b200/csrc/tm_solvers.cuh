@@ -733,7 +733,7 @@ __device__ __noinline__ uint64_t exact_flow_warp(const uint32_t (&u)[M * M], int
 // (the Flow64 layout).  Same algorithm, same votes, same results as exact_flow_warp<Flow64<M>, ...>; about a third fewer
 // instructions per step and an eighth of its shared-memory traffic.
 template <int N, int M, int T>
-__device__ __noinline__ uint64_t exact_flow_warp_reg(const uint32_t (&u)[M * M], int Emin, bool enabled, int& status, FlowCell* base, bool* certified) {
+__device__ __forceinline__ uint64_t exact_flow_warp_reg(const uint32_t (&u)[M * M], int Emin, bool enabled, int& status, FlowCell* base, bool* certified) {
     typedef Flow64<M> A;
     typedef long long V;
     constexpr int P = M - N;
