@@ -154,9 +154,10 @@ int build_plan(const tm_problem* probs, int count, int N, int M, int method, voi
             tmask::LaunchArgs& a = pg.generic;
             a.count = n; a.total_items = total; a.N = N; a.M = M; a.method = method; a.stream = nullptr; a.status = nullptr;
             a.partials = partials;
-            const int wpc = tmask::generic_warps_per_cta();
+            const int wpc = tmask::generic_warps_per_cta(N, M, method);
             const long long want = (total + wpc - 1) / wpc;
-            const int cap = dev.sms * 4 < kPartialSlots / wpc ? dev.sms * 4 : kPartialSlots / wpc;
+            const int fill = dev.sms * tmask::generic_ctas_per_sm(N, M, method);
+            const int cap = fill < kPartialSlots / wpc ? fill : kPartialSlots / wpc;
             a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));
             a.single = pg.probs[0];
             a.table = n > 1 ? dtab + used : nullptr;

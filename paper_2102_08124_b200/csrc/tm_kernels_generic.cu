@@ -14,6 +14,11 @@ namespace tmask {
 namespace {
 
 constexpr int kWarpsPerCta = 8;
+// The flow solver keeps three warps per scheduler busy where its 168 registers allow it (a CTA of 12 warps holds all of an
+// SM's registers and, at 512 bytes of edge costs per thread, nearly all of its shared memory).
+constexpr int kFlowWarpsPerCta = 12;
+constexpr bool takes_flow(int N, int M, int method) { return method == kMethodExact && !(M == 4 && N == 2); }
+constexpr int warps_for(int N, int M, int method) { return takes_flow(N, M, method) ? kFlowWarpsPerCta : kWarpsPerCta; }
 
 template <int M>
 __device__ __forceinline__ void load_block(const DevProblem& P, long long row0, long long col0, bool active, uint32_t (&w)[M * M]) {
@@ -88,10 +93,13 @@ __device__ __forceinline__ const DevProblem& find_problem(const DevProblem* tabl
 // paths.  How many a block needs is known beforehand -- the units by which its columns exceed M - N once every row has
 // pruned its M - N lightest entries -- so the blocks of kSortItems consecutive work items are dealt to the solver's
 // rounds in the order of that number, and the 32 blocks of a round need about the same.
+// The same block can be solved as it stands or turned (rows for columns): the optimum is the same set of entries, and the
+// turned start often needs fewer paths, so every block takes the cheaper of the two.
 constexpr int kSortItems = 8;
-constexpr int kSortBytesPerWarp = kSortItems * 32 * (8 + 1);          // a kept mask and an order entry per block
+constexpr int kSortBytesPerWarp = kSortItems * 32 * (8 + 2);          // a kept mask and an order entry per block
 
-template <int N, int M>
+// TURNED: the count for the block with rows and columns exchanged
+template <int N, int M, bool TURNED>
 __device__ __forceinline__ int repair_units(const uint32_t (&u)[M * M]) {
     int load[M];
 #pragma unroll
@@ -101,9 +109,12 @@ __device__ __forceinline__ int repair_units(const uint32_t (&u)[M * M]) {
 #pragma unroll
         for (int j = 0; j < M; ++j) {
             int heavier = 0;
+            const uint32_t me = TURNED ? u[j * M + i] : u[i * M + j];
 #pragma unroll
-            for (int k = 0; k < M; ++k)
-                heavier += (k != j) && (u[i * M + k] > u[i * M + j] || (u[i * M + k] == u[i * M + j] && k > j));
+            for (int k = 0; k < M; ++k) {
+                const uint32_t other = TURNED ? u[k * M + i] : u[i * M + k];
+                heavier += (k != j) && (other > me || (other == me && k > j));
+            }
             load[j] += heavier >= N ? 1 : 0;
         }
     }
@@ -136,15 +147,16 @@ __device__ __forceinline__ void store_mask_words(const DevProblem& P, long long 
 }
 
 // Items [item, item + n) of problem P (n <= kSortItems) through the flow solver; returns the lane's share of the objective.
-template <int N, int M>
+template <int N, int M, int W>
 __device__ __forceinline__ double flow_group(const DevProblem& P, long long item, int n, unsigned char* flow_smem, unsigned char* sort_smem, int& status) {
     const int lane = threadIdx.x & 31;
     const unsigned lt = (1u << lane) - 1u;
     uint64_t* keptbuf = reinterpret_cast<uint64_t*>(sort_smem);
-    unsigned char* order = sort_smem + kSortItems * 32 * 8;
+    unsigned short* order = reinterpret_cast<unsigned short*>(sort_smem + kSortItems * 32 * 8);   // block | turned << 15
     const long long local0 = item - P.item_begin;
     // ---- how many units each block needs ----
     int need[kSortItems], dmax = -1;
+    unsigned turned = 0;                                                // bit r: block r of this lane is solved turned
 #pragma unroll
     for (int r = 0; r < kSortItems; ++r) {
         need[r] = -1;
@@ -156,7 +168,9 @@ __device__ __forceinline__ double flow_group(const DevProblem& P, long long item
                 int ignored = 0;
                 load_block<M>(P, bi * M, (long long)bj * M, true, w);
                 magnitudes<M>(w, u, ignored);
-                need[r] = repair_units<N, M>(u);
+                const int as_is = repair_units<N, M, false>(u), other_way = repair_units<N, M, true>(u);
+                need[r] = min(as_is, other_way);
+                turned |= (other_way < as_is ? 1u : 0u) << r;
             }
         }
         dmax = max(dmax, need[r]);
@@ -169,7 +183,7 @@ __device__ __forceinline__ double flow_group(const DevProblem& P, long long item
         for (int r = 0; r < kSortItems; ++r) {
             const bool mine = need[r] == v;
             const unsigned m = __ballot_sync(0xFFFFFFFFu, mine);
-            if (mine) order[sorted + __popc(m & lt)] = (unsigned char)(r * 32 + lane);
+            if (mine) order[sorted + __popc(m & lt)] = (unsigned short)((r * 32 + lane) | (((turned >> r) & 1u) << 15));
             sorted += __popc(m);
         }
     }
@@ -178,14 +192,15 @@ __device__ __forceinline__ double flow_group(const DevProblem& P, long long item
     double acc = 0.0;
     for (int base = 0; base < sorted; base += 32) {
         const bool live = base + lane < sorted;
-        const int id = live ? order[base + lane] : 0, r = id >> 5, l = id & 31;
+        const int entry = live ? order[base + lane] : 0, id = entry & 0x7FFF, r = id >> 5, l = id & 31;
+        const bool turn = (entry >> 15) != 0;
         const long long local = local0 + r, bi = local / P.chunks;
         const int chunk = (int)(local - bi * P.chunks);
         const long long row0 = bi * M, col0 = ((long long)chunk * 32 + l) * M;
         uint32_t w[M * M], u[M * M];
         load_block<M>(P, row0, col0, live, w);
         magnitudes<M>(w, u, status);
-        uint64_t kept = exact_ssp<N, M, kWarpsPerCta * 32>(u, status, flow_smem, (int)threadIdx.x, live);
+        uint64_t kept = exact_ssp<N, M, W * 32>(u, status, flow_smem, (int)threadIdx.x, live, turn);
         if (!live) kept = 0;
         float sum = 0.f;
 #pragma unroll
@@ -212,12 +227,13 @@ __device__ __forceinline__ double flow_group(const DevProblem& P, long long item
 
 template <int N, int M, int METHOD>
 // the exact 2:4 scorer is register-hungry: two CTAs per SM cap it at 128 registers (its rare wide-integer path spills)
-__global__ void __launch_bounds__(kWarpsPerCta * 32, (METHOD == kMethodExact && M == 4 && N == 2) ? 2 : 1)
+__global__ void __launch_bounds__(warps_for(N, M, METHOD) * 32, (METHOD == kMethodExact && M == 4 && N == 2) ? 2 : 1)
 generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, int count, long long total_items,
                double* __restrict__ partials, int* __restrict__ status_out) {
+    constexpr int kW = warps_for(N, M, METHOD);
     const int lane = threadIdx.x & 31;
-    const long long gw = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-    const long long nwarps = (long long)gridDim.x * kWarpsPerCta;
+    const long long gw = (long long)blockIdx.x * kW + (threadIdx.x >> 5);
+    const long long nwarps = (long long)gridDim.x * kW;
     // even split: total / nwarps items each, the first warps one more
     const long long order = gw;
     const long long share = total_items / nwarps, surplus = total_items - share * nwarps;
@@ -256,8 +272,8 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
             // a group of consecutive items of this problem at a time
             const long long stop = k + 1 < count ? min(end, tab[k + 1].item_begin) : end;
             const int n = (int)min((long long)kSortItems, stop - item);
-            unsigned char* sort_smem = flow_smem + (size_t)flow_shared_bytes_per_thread(M) * kWarpsPerCta * 32 + (threadIdx.x >> 5) * kSortBytesPerWarp;
-            acc += flow_group<N, M>(P, item, n, flow_smem, sort_smem, status);
+            unsigned char* sort_smem = flow_smem + (size_t)flow_shared_bytes_per_thread(M) * kW * 32 + (threadIdx.x >> 5) * kSortBytesPerWarp;
+            acc += flow_group<N, M, kW>(P, item, n, flow_smem, sort_smem, status);
             item += n - 1;
             continue;
         }
@@ -278,7 +294,7 @@ generic_kernel(const DevProblem single, const DevProblem* __restrict__ table, in
         uint64_t kept;
         if constexpr (METHOD == kMethodExact) {
             if constexpr (M == 4 && N == 2) kept = exact_2_4(u, P.dtype == kBF16 ? 16 : 0);
-            else kept = exact_ssp<N, M, kWarpsPerCta * 32>(u, status, flow_smem, (int)threadIdx.x, active);
+            else kept = exact_ssp<N, M, kW * 32>(u, status, flow_smem, (int)threadIdx.x, active, false);
         } else {
             kept = cover_mask<N, M>(u);
             if constexpr (METHOD == kMethodApprox) {
@@ -344,11 +360,13 @@ reduce_kernel(const DevProblem single, const DevProblem* __restrict__ table, con
 
 template <int N, int M>
 cudaError_t launch_nm(const LaunchArgs& a) {
-    const dim3 grid((unsigned)a.ctas), block(kWarpsPerCta * 32);
+    const dim3 grid((unsigned)a.ctas), block(warps_for(N, M, a.method) * 32);
     switch (a.method) {
     case kMethodExact: {
-        // the flow solver (everything but 2:4) keeps its state in shared memory
-        constexpr size_t smem = (N == 2 && M == 4) ? 0 : (size_t)flow_shared_bytes_per_thread(M) * kWarpsPerCta * 32 + (size_t)kSortBytesPerWarp * kWarpsPerCta;
+        // the flow solver (everything but 2:4) keeps its edge costs in shared memory, and the sorted rounds their bookkeeping
+        constexpr int kW = warps_for(N, M, kMethodExact);
+        constexpr size_t smem = (N == 2 && M == 4) ? 0 : (size_t)flow_shared_bytes_per_thread(M) * kW * 32 + (size_t)kSortBytesPerWarp * kW;
+        static_assert(smem <= 232448, "at most 227 KB of shared memory per CTA");
         static PerDeviceOnce configured;   // per instantiation
         if (smem > 48 * 1024) {
             const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(generic_kernel<N, M, kMethodExact>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });
@@ -365,17 +383,22 @@ cudaError_t launch_nm(const LaunchArgs& a) {
 
 }  // namespace
 
-int generic_warps_per_cta() { return kWarpsPerCta; }
+int generic_warps_per_cta(int N, int M, int method) { return warps_for(N, M, method); }
+// CTAs per SM worth launching.  A flow CTA fills its SM, but its blocks take very different times: four CTAs per SM queued
+// one behind the other even out what a single fat share per warp does not (8192^2, 4:8: 4.05 ms against 5.12 ms), although
+// shorter shares leave the warps fewer items to sort at a time.
+int generic_ctas_per_sm(int, int, int) { return 4; }
 
 cudaError_t launch_generic(const LaunchArgs& a) {
-    cudaError_t e = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * kWarpsPerCta, a.stream);
+    const int wpc = warps_for(a.N, a.M, a.method);
+    cudaError_t e = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * wpc, a.stream);
     if (e != cudaSuccess) return e;
     if (a.total_items > 0) {
         if (a.M == 4) e = a.N == 2 ? launch_nm<2, 4>(a) : (a.N == 1 ? launch_nm<1, 4>(a) : launch_nm<3, 4>(a));
         else e = a.N == 4 ? launch_nm<4, 8>(a) : (a.N == 2 ? launch_nm<2, 8>(a) : launch_nm<6, 8>(a));
         if (e != cudaSuccess) return e;
     }
-    reduce_kernel<<<a.count, 256, 0, a.stream>>>(a.single, a.table, a.partials, (long long)a.ctas * kWarpsPerCta);
+    reduce_kernel<<<a.count, 256, 0, a.stream>>>(a.single, a.table, a.partials, (long long)a.ctas * wpc);
     return cudaGetLastError();
 }
 

@@ -38,7 +38,8 @@ struct LaunchArgs {
 // Generic path: any supported (N, M, method, dtype, ld).  Zeroes the partials, runs the search and
 // the fixed-order objective reduction on a.stream.
 cudaError_t launch_generic(const LaunchArgs& a);
-int generic_warps_per_cta();
+int generic_warps_per_cta(int N, int M, int method);
+int generic_ctas_per_sm(int N, int M, int method);
 
 // Bandwidth path (TMA-staged, bit-parallel): approximate 2:4 search on 16-byte aligned matrices.
 struct TmaLaunch {

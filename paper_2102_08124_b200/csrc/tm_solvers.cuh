@@ -506,13 +506,13 @@ __device__ __noinline__ uint64_t exact_flow_run(const uint32_t (&u)[M * M], int 
 // magnitudes at every use).  Flow64 carries q_p alone, precomputed: half the words in every load, sum and
 // comparison.  Without the tie term the optimum it finds is the wanted one only if it is the only one; that is
 // certified afterwards (tight_forest below), and a block without the certificate is solved again in full.
-// Shared-memory state.  A thread owns the 8-byte cells t, T + t, 2T + t, ... of the CTA's region (T threads; consecutive
-// threads touch consecutive cells, so 8-byte accesses do not collide) -- the same cells in either format, because warps
-// of a CTA can be in different formats at the same time.  cell(base, k, T) is the k-th cell of the thread whose first is base.
-constexpr int flow_cells_per_thread(int M) { return M * M + 2 * (2 * M); }                   // Flow64: a cell per cost, potential, distance
-constexpr int flow_shared_bytes_per_thread(int M) {                                         // Flow128: two cells per potential / distance, half a cell per magnitude
-    return 8 * (flow_cells_per_thread(M) > 4 * (2 * M) + M * M / 2 ? flow_cells_per_thread(M) : 4 * (2 * M) + M * M / 2);
-}
+// State.  The first pass (exact_flow_warp_reg) keeps potentials and distances in registers and its 64-bit edge costs in
+// shared memory: a thread owns the 8-byte cells t, T + t, 2T + t, ... of the CTA's region (T threads; consecutive threads
+// touch consecutive cells, so 8-byte accesses do not collide).  The 128-bit pass, which only the blocks without the
+// uniqueness certificate take, keeps everything in cells of the thread's local memory (T = 1).  cell(base, k, T) is the
+// k-th cell of the thread whose first is base.
+constexpr int flow_cells128_per_thread(int M) { return 4 * (2 * M) + M * M / 2; }          // Flow128: two cells per potential / distance, half a cell per magnitude
+constexpr int flow_shared_bytes_per_thread(int M) { return 8 * M * M; }                    // shared memory holds the 64-bit edge costs of the first pass only
 typedef unsigned long long FlowCell;
 __device__ __forceinline__ FlowCell* cell(FlowCell* base, int k, int T) { return base + (size_t)k * T; }
 
@@ -859,8 +859,11 @@ __device__ __forceinline__ uint64_t exact_flow_warp_reg(const uint32_t (&u)[M * 
 
 // Called by all 32 lanes of a warp.  flow_smem: the CTA's region of flow_shared_bytes_per_thread(M) bytes per thread, T =
 // threads per CTA (a constant, so that every cell offset is one), tid = this thread; live: the lane holds a block of the matrix (the others only keep the votes whole).
+// turn: run the first pass on the block with rows and columns exchanged (the caller found that its start needs fewer
+// paths); the optimum is the same set of entries, and the certificate of uniqueness holds for either view.  The pass that
+// decides ties by position always sees the block as it stands.
 template <int N, int M, int T>
-__device__ __forceinline__ uint64_t exact_ssp(const uint32_t (&u)[M * M], int& status, unsigned char* flow_smem, int tid, bool live) {
+__device__ __forceinline__ uint64_t exact_ssp(const uint32_t (&u)[M * M], int& status, unsigned char* flow_smem, int tid, bool live, bool turn) {
     int Emin, Emax;
     if (!exponent_range<M * M>(u, Emin, Emax)) { Emin = 1; Emax = 1; }
     // 128-bit costs: 64 tie bits + 24 significand bits + spread; paths (<= 2M arcs) and potentials (<= M(M-N)
@@ -869,11 +872,27 @@ __device__ __forceinline__ uint64_t exact_ssp(const uint32_t (&u)[M * M], int& s
     FlowCell* base = reinterpret_cast<FlowCell*>(flow_smem) + tid;
     // first without the tie term, in 64-bit words
     bool certified = false;
-    uint64_t kept = exact_flow_warp_reg<N, M, T>(u, Emin, live && !wide, status, base, &certified);
+    uint64_t kept;
+    {
+        uint32_t ut[M * M];
+#pragma unroll
+        for (int i = 0; i < M; ++i)
+#pragma unroll
+            for (int j = 0; j < M; ++j) ut[i * M + j] = turn ? u[j * M + i] : u[i * M + j];
+        const uint64_t k1 = exact_flow_warp_reg<N, M, T>(ut, Emin, live && !wide, status, base, &certified);
+        uint64_t back = 0;                                              // k1 with rows and columns exchanged
+#pragma unroll
+        for (int i = 0; i < M; ++i)
+#pragma unroll
+            for (int j = 0; j < M; ++j) back |= ((k1 >> (j * M + i)) & 1ull) << (i * M + j);
+        kept = turn ? back : k1;
+    }
     // blocks whose optimum is not certified unique (magnitude ties, as a rule): the full costs decide
     const bool again = live && !wide && !certified;
     if (__any_sync(0xFFFFFFFFu, again)) {
-        const uint64_t k2 = exact_flow_warp<Flow128<M>, N, M, T>(u, Emin, again, status, base, nullptr);
+        // its state lives in the thread's local memory (cells one after the other): shared memory is all taken by the first pass
+        FlowCell cells[flow_cells128_per_thread(M)];
+        const uint64_t k2 = exact_flow_warp<Flow128<M>, N, M, 1>(u, Emin, again, status, cells, nullptr);
         kept = again ? k2 : kept;
     }
     if (live && wide) kept = exact_flow_run<CostWide, N, M>(u, Emin, status);
