@@ -3,11 +3,13 @@
 //
 // compress24_meta_kernel    mask -> meta, meta_t.  The metadata nibble idx0 | idx1 << 2 of a group is a function of the
 //   group's keep nibble alone, so both metadata arrays come from the packed mask without a look at W.  A warp takes a
-//   unit of 256 rows x 256 columns, 32 rows at a time, lane = row: the row's eight mask words become its eight metadata
-//   words by bit-parallel logic on all eight nibbles of a word at once; each of the eight 32 x 32 bit tiles is transposed
-//   across the warp (five shuffle steps), after which lane = column and the same logic gives the column's metadata word
-//   for these 32 rows.  Those words wait in the warp's shared buffer until the unit's 256 rows are done and leave as
-//   32-byte runs.  The same pass checks that every group keeps exactly two and raises the bad-mask status otherwise.
+//   unit of 256 rows x 256 columns, 32 rows at a time.  A word of eight keep nibbles becomes eight metadata nibbles by
+//   three logic operations; for the transposed metadata the nibbles of a column's eight block rows have to meet in one
+//   word, a 32 x 32 bit transpose across the warp.  Units inside the matrix hold four rows per lane, which makes the
+//   column groups' nibbles come out bit-sliced and leaves only three of the transpose's five steps to shuffles
+//   (meta_rows_fast); units on an edge, and rows with a bad group, take the plainer lane-per-row form (meta_rows).  The
+//   transposed words wait in the warp's shared buffer until the unit's 256 rows are done and leave as 32-byte runs.  The
+//   same pass checks that every group keeps exactly two and raises the bad-mask status otherwise.
 //
 // compress24_values_kernel  W, mask -> values, values_t.  Every warp is a pipeline of its own over work items of 32 rows
 //   x 128 columns.  An item arrives as two halves of 16 rows (4 KB of weights and 256 bytes of mask words each, two
@@ -208,7 +210,64 @@ __device__ __forceinline__ bool meta_rows(const CompressArgs& A, const MetaUnit&
     return bad;
 }
 
-__global__ void __launch_bounds__(kMWarps * 32)
+// The same 32 rows for a unit that lies wholly inside the matrix, with four rows per lane: lane = (block row b = lane & 7,
+// word pair q = lane >> 3) holds rows 4b .. 4b+3 of words 2q, 2q+1.  A column group's four keep bits then sit in the same
+// bit of the lane's four words, so the group's metadata nibble comes out bit-sliced (four words of "bit n of the nibble of
+// column c") with four logic operations for 32 columns, and the 32 x 32 transpose that gathers a column's eight nibbles
+// starts with its two finest steps inside the lane; only the three coarse steps cross lanes (12 shuffles per 32 columns
+// instead of 40).  The row form needs no exchange at all: four lanes write the 32 bytes of a row in one instruction.
+// r[i][t]: row 4b + i, word 2q + t.  Returns false, having written nothing, if some group does not keep exactly two.
+__device__ __forceinline__ bool meta_rows_fast(const CompressArgs& A, const MetaUnit& U, int g, const uint2 (&r)[4], uint32_t* park, int lane) {
+    const int b = lane & 7, q = lane >> 3;
+    uint32_t bad = 0;
+    uint2 mrow[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        mrow[i] = make_uint2(meta_of(r[i].x), meta_of(r[i].y));
+        bad |= (nibble_counts(r[i].x) ^ 0x22222222u) | (nibble_counts(r[i].y) ^ 0x22222222u);
+    }
+    uint32_t t4[2][4];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const uint32_t b0 = t ? r[0].y : r[0].x, b1 = t ? r[1].y : r[1].x, b2 = t ? r[2].y : r[2].x, b3 = t ? r[3].y : r[3].x;
+        // exactly two of the four: the pairs (b0, b1) and (b2, b3) hold one each, or one holds both and the other none
+        const uint32_t a = b0 ^ b1, p = b0 & b1, c = b2 ^ b3, d = b2 & b3;
+        bad |= ~((a & c) | ((p ^ d) & ~(a | c)));
+        uint32_t x0 = ~b0 & b1, x1 = ~b0 & ~b1, x2 = b3 | ~b2, x3 = b3 | b2;      // bit n of the columns' metadata nibbles
+        // transpose steps 1 and 2: rows 4b + n of the bit matrix are the lane's own four words
+        uint32_t e = ((x0 >> 1) ^ x1) & 0x55555555u; x1 ^= e; x0 ^= e << 1;
+        e = ((x2 >> 1) ^ x3) & 0x55555555u; x3 ^= e; x2 ^= e << 1;
+        e = ((x0 >> 2) ^ x2) & 0x33333333u; x2 ^= e; x0 ^= e << 2;
+        e = ((x1 >> 2) ^ x3) & 0x33333333u; x3 ^= e; x1 ^= e << 2;
+        t4[t][0] = x0; t4[t][1] = x1; t4[t][2] = x2; t4[t][3] = x3;
+    }
+    if (__any_sync(0xFFFFFFFFu, bad != 0)) return false;
+    // steps 4, 8, 16 across the lanes b ^ 1, b ^ 2, b ^ 4
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const int j = 4 << k, lb = 1 << k;
+        const uint32_t m = j == 16 ? 0x0000FFFFu : (j == 8 ? 0x00FF00FFu : 0x0F0F0F0Fu);
+        const uint32_t keep = (b & lb) ? ~m : m;
+        const int rot = (b & lb) ? 32 - j : j;
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+#pragma unroll
+            for (int n = 0; n < 4; ++n) {
+                const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, t4[t][n], lb);
+                t4[t][n] = lop3<lut3(f_sel)>(t4[t][n], __funnelshift_l(y, y, rot), keep);
+            }
+    }
+    // word n of the lane now belongs to column 4b + n of its 32: eight nibbles, one per block row
+    const long long row = U.ur * 256 + g * 32 + 4 * b;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) *reinterpret_cast<uint2*>(A.meta + (row + i) * A.wpr + U.word0 + 2 * q) = mrow[i];
+#pragma unroll
+    for (int t = 0; t < 2; ++t)
+        *reinterpret_cast<uint4*>(park + g * 256 + 64 * q + 32 * t + 4 * b) = make_uint4(t4[t][0], t4[t][1], t4[t][2], t4[t][3]);
+    return true;
+}
+
+__global__ void __launch_bounds__(kMWarps * 32, 6)
 compress24_meta_kernel(const __grid_constant__ CompressArgs A, int* __restrict__ status_out) {
     __shared__ uint32_t park_all[kMWarps][kMParkWords];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -224,22 +283,46 @@ compress24_meta_kernel(const __grid_constant__ CompressArgs A, int* __restrict__
         U.groups_left = (int)min((long long)64, (A.cols - U.word0 * 32) / 4);
         const int n_g = (int)min((long long)8, (A.rows - U.ur * 256 + 31) / 32);
         const bool full = U.groups_left == 64 && U.ur * 256 + 256 <= A.rows;
-        // the rows are read one group ahead of their use
-        auto load = [&](int g, uint4& a, uint4& b) {
-            const long long row = U.ur * 256 + g * 32 + lane;
-            const uint4* src = reinterpret_cast<const uint4*>(A.mask + row * A.wpr + U.word0);
-            a = make_uint4(0, 0, 0, 0); b = a;
-            if (full || (row < A.rows && U.word0 < A.wpr)) a = __ldg(src);
-            if (full || (row < A.rows && U.word0 + 4 < A.wpr)) b = __ldg(src + 1);
-        };
-        uint4 na, nb;
-        load(0, na, nb);
+        if (full) {
+            // four rows per lane; the rows are read one group ahead of their use
+            const int b = lane & 7, q = lane >> 3;
+            auto load4 = [&](int g, uint2 (&r)[4]) {
+                const uint32_t* src = A.mask + (U.ur * 256 + g * 32 + 4 * b) * A.wpr + U.word0 + 2 * q;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) r[i] = __ldg(reinterpret_cast<const uint2*>(src + (long long)i * A.wpr));
+            };
+            uint2 next[4];
+            load4(0, next);
 #pragma unroll 1
-        for (int g = 0; g < n_g; ++g) {
-            const uint4 a = na, b = nb;
-            if (g + 1 < n_g) load(g + 1, na, nb);
-            if (full) bad |= meta_rows<true>(A, U, g, a, b, plan, park, lane);
-            else bad |= meta_rows<false>(A, U, g, a, b, plan, park, lane);
+            for (int g = 0; g < 8; ++g) {
+                uint2 r[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) r[i] = next[i];
+                if (g + 1 < 8) load4(g + 1, next);
+                if (!meta_rows_fast(A, U, g, r, park, lane)) {
+                    // a bad group somewhere in these rows: the lane-per-row form, which writes zeros for it
+                    const long long row = U.ur * 256 + g * 32 + lane;
+                    const uint4* src = reinterpret_cast<const uint4*>(A.mask + row * A.wpr + U.word0);
+                    bad |= meta_rows<true>(A, U, g, __ldg(src), __ldg(src + 1), plan, park, lane);
+                }
+            }
+        } else {
+            // the rows are read one group ahead of their use
+            auto load = [&](int g, uint4& a, uint4& b) {
+                const long long row = U.ur * 256 + g * 32 + lane;
+                const uint4* src = reinterpret_cast<const uint4*>(A.mask + row * A.wpr + U.word0);
+                a = make_uint4(0, 0, 0, 0); b = a;
+                if (row < A.rows && U.word0 < A.wpr) a = __ldg(src);
+                if (row < A.rows && U.word0 + 4 < A.wpr) b = __ldg(src + 1);
+            };
+            uint4 na, nb;
+            load(0, na, nb);
+#pragma unroll 1
+            for (int g = 0; g < n_g; ++g) {
+                const uint4 a = na, b = nb;
+                if (g + 1 < n_g) load(g + 1, na, nb);
+                bad |= meta_rows<false>(A, U, g, a, b, plan, park, lane);
+            }
         }
         // ---- the unit's transposed metadata: eight words per column ----
         __syncwarp();
