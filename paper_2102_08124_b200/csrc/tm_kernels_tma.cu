@@ -360,6 +360,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         // a copy that never landed: stop before anything is computed on, or stored from, the unfilled stage
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bars[s], parity))) { status |= kDevInternal; alive = false; break; }
         int qn = 0;
+        bool redo = false;                                      // exact search on bf16: the item needs the later tiers
         if (cur.k != acc_k) {                                   // a new matrix starts: flush the objective partial
             if (acc_k >= 0) {
                 acc += (double)facc;
@@ -400,7 +401,10 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
 #pragma unroll
                     for (int p = 0; p < 16; ++p) bad |= (u[p] >> 23) == 0xFFu;
                     if (bad) status |= kDevNonFinite;
-                    k |= (uint32_t)exact_2_4(u, DT == kBF16 ? 16 : 0) << (16 * b);
+                    uint64_t code = 0;
+                    if constexpr (DT == kBF16) { if (!redo) redo = !exact_2_4_bf16_first(u, code); }     // first tier or, later, all four blocks again
+                    else code = exact_2_4(u, 0);
+                    k |= (uint32_t)code << (16 * b);
                 }
             } else {
             front_end<DT, kRows>(stage + h * G::kHalfBytes, lane, rel, worst, nonzero);
@@ -453,6 +457,16 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             if (h == 0 && loaded < n_items) {       // refill the stage of the previous item: its store was issued one item ago
                 if constexpr (HAS_OUT) { if (lane == 0 && it > 0) tma_wait_read<0>(); }
                 issue_next((s + G::kStages - 1) % G::kStages);
+            }
+        }
+        if constexpr (METHOD == kMethodExact && DT == kBF16) {
+            if (redo) {                    // some block of this item (warp-uniform) does not fit the first tier
+#pragma unroll 1
+                for (int h = 0; h < kHalves; ++h) {
+                    uint32_t codes[2];
+                    exact_2_4_bf16_rest(stage + h * G::kHalfBytes + lane * (8 * G::kElem), G::kRowPitch, 4 * G::kElem, 2, codes);
+                    kbuf[h * 32 + lane] = codes[0] | (codes[1] << 16);
+                }
             }
         }
         __syncwarp();

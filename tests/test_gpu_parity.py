@@ -126,6 +126,13 @@ def test_exact_2_4_bf16_narrow_blocks_take_the_32_bit_scorer():
     V = W.copy()
     V[5, 100] = 0x0001; V[40, 777] = 0x7F00; V[41, 20] = 0x0080         # blocks with a wide exponent spread
     assert_parity(V, 2, 4, tm.TM_EXACT)
+    # the same on the staged kernel (above a million weights): most work items take the 32-bit scorer as a whole, a few
+    # hold one block that cannot and are scored again by the later tiers, and one item has such blocks in both halves
+    B = workloads.quantised_bf16(260, 4104, 0.02, 42)
+    assert_parity(B, 2, 4, tm.TM_EXACT)
+    B[9, 300] = 0x0001; B[130, 2048] = 0x7F00; B[131, 2050] = 0x0003; B[200, 10] = 0x0080; B[201, 400] = 0x7F7F
+    B[258, 4100] = 0x0002; B[64, 0:512] = 0                              # a ragged item, and a row of zeros across one item
+    assert_parity(B, 2, 4, tm.TM_EXACT)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
