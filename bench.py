@@ -294,7 +294,7 @@ def run_gpu(args):
                    "ms_x_sm_mhz": ms * sm_mhz if sm_mhz else None,
                    "note": "value = median over the blocks; every block is exactly K steps, timed with CUDA events on the launching stream"},
         "e2e": e2e,
-        "gpu_launches": 2 * args.steps * repeats,
+        "gpu_launches": args.steps * repeats,               # a step is one launch: the search kernel reduces its own objective
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": TRAFFIC_BYTES_PER_LAUNCH if ROWS == FULL_ROWS else None, "traffic_source": TRAFFIC_SOURCE,
@@ -303,7 +303,7 @@ def run_gpu(args):
                      "cold": {"ms_per_step": ms_cold, "achieved": weights * BYTES_PER_WEIGHT / (ms_cold * 1e-3) / 1e9,
                               "frac": weights * BYTES_PER_WEIGHT / (ms_cold * 1e-3) / 1e9 / peak,
                               "note": "K steps timed right after W warm-up steps, before the sustained warm-up under the clock sampler"},
-                     "note": "duration = CUDA-event time of one step (search kernel + its tiny partial-zeroing and reduction launches)"},
+                     "note": "duration = CUDA-event time of one step = one launch of the search kernel (its last CTA adds up the objective)"},
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))

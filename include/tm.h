@@ -110,8 +110,9 @@ size_t tm_mask_words(int64_t rows, int64_t cols);
  * tm_find_mask / tm_find_mask_bf16 -- Section 4, Eq. 1 (TM_EXACT), Algorithm 1 (TM_APPROX*).
  * One matrix, fp32 resp. bf16, ld == cols, on the legacy default stream (stream 0) of the current
  * device.  All pointers are device pointers.  The first call on a device allocates a small scratch
- * buffer (objective partials and a status word) that the library keeps until the process exits;
- * tm_find_mask_batched() never allocates.  Device status bits of these calls accumulate in that
+ * buffer (objective partials, a status word and a count of finished thread blocks) that the library keeps
+ * until the process exits; tm_find_mask_batched() never allocates.  For a 16-byte aligned matrix the call is a
+ * single kernel launch: the thread block that finishes last adds up the objective partials in a fixed order.  Device status bits of these calls accumulate in that
  * scratch and are fetched with tm_device_status().
  */
 int tm_find_mask(const void* W, int64_t rows, int64_t cols, int N, int M, int method,
@@ -148,9 +149,12 @@ size_t tm_workspace_bytes(const tm_problem* probs_host, int count);
  * scratch": the mask is refreshed every 40 iterations).  tm_plan_create validates the descriptors, builds the
  * tensor maps and copies the descriptor tables into the workspace once (synchronising stream 0; it allocates
  * host memory for the plan, nothing on the device).  tm_plan_run then only clears the objective partials and
- * launches the kernels on cuda_stream: it touches no host memory asynchronously, so it can be recorded by a
- * stream capture and replayed.  The workspace belongs to the plan until tm_plan_destroy; the matrices must stay
- * where they were (same pointers, shapes, pitches).  Results equal tm_find_mask_batched()'s bit for bit.
+ * launches the kernels on cuda_stream (a group of one matrix is a single launch that reduces its own objective
+ * and needs no clearing): it touches no host memory asynchronously, so it can be recorded by a stream capture
+ * and replayed.  The workspace belongs to the plan until tm_plan_destroy -- its first 256 bytes are cleared at
+ * creation and must not be written by anyone else -- and the matrices must stay where they were (same pointers,
+ * shapes, pitches).  Masks and masked weights equal tm_find_mask_batched()'s bit for bit; objectives too, except
+ * that a single-matrix group adds its partial sums in another (fixed) order, i.e. equal up to fp64 rounding.
  */
 typedef struct tm_plan tm_plan;
 int tm_plan_create(const tm_problem* probs_host, int count, int N, int M, int method, void* workspace_dev, size_t workspace_bytes,

@@ -18,6 +18,9 @@ constexpr int kPartialSlots = 8192;   // objective partials per matrix: (CTAs x 
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
 constexpr size_t kHeaderBytes = 256;  // reserved head of every workspace
+// Inside the header: the count of finished CTAs of a single-matrix bandwidth launch that reduces its own objective.  Only
+// workspaces whose header the library itself has cleared use it (every such launch leaves it at zero again).
+constexpr size_t kDoneOffset = 128;
 
 size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 int at_least_one(int count) { return count > 0 ? count : 1; }
@@ -116,7 +119,9 @@ int validate_call(const tm_problem* probs, int count, int N, int M, int method, 
     return TM_OK;
 }
 
-int build_plan(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes, const DeviceState& dev, Plan& plan) {
+// header_clear: the workspace's header was zeroed by this library and nothing but its launches has touched it since.
+int build_plan(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes, const DeviceState& dev, Plan& plan,
+               bool header_clear) {
     const int rc = validate_call(probs, count, N, M, method, ws, ws_bytes);
     if (rc != TM_OK) return rc;
     plan.N = N; plan.M = M; plan.method = method; plan.count = count; plan.ws = ws;
@@ -175,6 +180,7 @@ int build_plan(const tm_problem* probs, int count, int N, int M, int method, voi
             const int cap = dev.sms < kPartialSlots / wpc ? dev.sms : kPartialSlots / wpc;
             a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));
             a.entries_dev = n > 1 ? dent + (size_t)used * esz : nullptr;
+            a.done = header_clear && n == 1 ? reinterpret_cast<unsigned int*>(base + kDoneOffset) : nullptr;
         }
         used += n;
     }
@@ -214,9 +220,9 @@ int launch_plan(const Plan& plan, int* status_dev, cudaStream_t stream) {
 }
 
 int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes, int* status_dev,
-        cudaStream_t stream, const DeviceState& dev) {
+        cudaStream_t stream, const DeviceState& dev, bool header_clear) {
     Plan plan;
-    int rc = build_plan(probs, count, N, M, method, ws, ws_bytes, dev, plan);
+    int rc = build_plan(probs, count, N, M, method, ws, ws_bytes, dev, plan, header_clear);
     if (rc != TM_OK) return rc;
     if ((rc = upload_plan(plan, stream)) != TM_OK) return rc;
     return launch_plan(plan, status_dev, stream);
@@ -249,7 +255,7 @@ int plain_call(const void* W, int dtype, int64_t rows, int64_t cols, int N, int 
     if ((rc = current_device(&d)) != TM_OK) return rc;
     if ((rc = ensure_scratch(*d)) != TM_OK) return rc;
     void* scratch = d->scratch.load(std::memory_order_acquire);
-    return run(&p, 1, N, M, method, scratch, d->scratch_bytes, static_cast<int*>(scratch), nullptr, *d);
+    return run(&p, 1, N, M, method, scratch, d->scratch_bytes, static_cast<int*>(scratch), nullptr, *d, true);
 }
 
 int grow(void** p, size_t* have, size_t want) {
@@ -337,7 +343,8 @@ int tm_find_mask_batched(const tm_problem* probs_host, int count, int N, int M, 
     if (count == 0) return TM_OK;
     DeviceState* d = nullptr;
     if ((rc = current_device(&d)) != TM_OK) return rc;
-    return run(probs_host, count, N, M, method, workspace_dev, workspace_bytes, status_dev, static_cast<cudaStream_t>(cuda_stream), *d);
+    // the caller's workspace arrives with unknown contents: partials cleared, search, reduction kernel
+    return run(probs_host, count, N, M, method, workspace_dev, workspace_bytes, status_dev, static_cast<cudaStream_t>(cuda_stream), *d, false);
 }
 
 int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols, int N, int M, int method,
@@ -376,7 +383,8 @@ int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols,
     char* ws = static_cast<char*>(d->stage_ws);
     int* status_dev = reinterpret_cast<int*>(ws);                       // first 256 bytes: status + 16 objectives
     double* obj_dev = reinterpret_cast<double*>(ws + 64);
-    if (cudaMemsetAsync(ws, 0, kAlign, d->s_run) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    // status and objectives, and the headers of the strips' workspaces (their launches count finished CTAs there)
+    if (cudaMemsetAsync(ws, 0, (one_ws + kAlign) * 16 + kAlign, d->s_run) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
 
     std::vector<cudaEvent_t> ev_in((size_t)strips), ev_run((size_t)strips);
     bool ok = true;
@@ -397,7 +405,7 @@ int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols,
         p.mask_out = static_cast<uint32_t*>(d->stage_mask) + (size_t)r0 * wpr;
         p.masked_w_out = masked_w_out_host ? static_cast<char*>(d->stage_masked) + off : nullptr;
         p.objective_out = obj_dev + s;
-        rc = run(&p, 1, N, M, method, ws + kAlign + (size_t)s * (one_ws + kAlign), one_ws, status_dev, d->s_run, *d);
+        rc = run(&p, 1, N, M, method, ws + kAlign + (size_t)s * (one_ws + kAlign), one_ws, status_dev, d->s_run, *d, true);
         if (rc != TM_OK) { ok = false; break; }
         ok &= cudaEventRecord(ev_run[s], d->s_run) == cudaSuccess;
         ok &= cudaStreamWaitEvent(d->s_out, ev_run[s], 0) == cudaSuccess;
@@ -438,7 +446,7 @@ int tm_find_mask_batched_static(const tm_problem* probs_host, int count, int N, 
     void* scratch = nullptr;
     if ((rc = static_scratch_address(&scratch)) != TM_OK) return rc;
     // every launch below clears the objective partials it uses before its kernel runs on the same stream
-    return run(probs_host, count, N, M, method, scratch, TM_STATIC_SCRATCH_BYTES, status_dev, static_cast<cudaStream_t>(cuda_stream), *d);
+    return run(probs_host, count, N, M, method, scratch, TM_STATIC_SCRATCH_BYTES, status_dev, static_cast<cudaStream_t>(cuda_stream), *d, false);
 }
 
 struct tm_plan { Plan plan; };
@@ -454,7 +462,9 @@ int tm_plan_create(const tm_problem* probs_host, int count, int N, int M, int me
     if ((rc = current_device(&d)) != TM_OK) return rc;
     tm_plan* p = new (std::nothrow) tm_plan();
     if (!p) return TM_ERR_CUDA;
-    if ((rc = build_plan(probs_host, count, N, M, method, workspace_dev, workspace_bytes, *d, p->plan)) != TM_OK) { delete p; return rc; }
+    // the plan owns the workspace from here on: its header is cleared once, below, and single-matrix launches keep it clear
+    if ((rc = build_plan(probs_host, count, N, M, method, workspace_dev, workspace_bytes, *d, p->plan, true)) != TM_OK) { delete p; return rc; }
+    if (count > 0 && cudaMemset(workspace_dev, 0, kHeaderBytes) != cudaSuccess) { cudaGetLastError(); delete p; return TM_ERR_CUDA; }
     cudaGetDevice(&p->plan.device);
     // the tables are uploaded once, synchronously: tm_plan_run() then issues kernels only
     if ((rc = upload_plan(p->plan, nullptr)) != TM_OK || cudaStreamSynchronize(nullptr) != cudaSuccess) { cudaGetLastError(); delete p; return rc != TM_OK ? rc : TM_ERR_CUDA; }

@@ -288,7 +288,8 @@ __device__ __forceinline__ float back_end_absorb(unsigned char* stage, unsigned 
 template <int DT, int METHOD, bool HAS_OUT>
 __global__ void __launch_bounds__(Geometry<DT, METHOD>::kWarps * 32, 1)
 tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict__ table, int count, long long total_items,
-             double* __restrict__ partials, int* __restrict__ status_out, int n_keep, unsigned long long* __restrict__ vpartials) {
+             double* __restrict__ partials, int* __restrict__ status_out, int n_keep, unsigned long long* __restrict__ vpartials,
+             unsigned int* __restrict__ done) {
     using G = Geometry<DT, METHOD>;
     constexpr bool kRows = METHOD == kMethodRows || METHOD == kMethodRowsAbsorb;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -528,15 +529,16 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         for (int s = 0; s < G::kStages; ++s) { mbar_wait_bounded(&bars[s], 0, 1u << 14); mbar_wait_bounded(&bars[s], 1, 1u << 14); }
     }
     if (lane == 0) tma_wait_all<0>();
-    if (acc_k >= 0) {
+    if (acc_k >= 0 || done) {                  // a launch that reduces its own objective wants a partial (a zero) from idle warps too
         acc += (double)facc;
         for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-        if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
+        if (lane == 0) partials[(long long)(acc_k >= 0 ? acc_k : 0) * nwarps + gw] = acc;
     }
     if constexpr (DT == kF32) { if (worst >= 0x7F800000u) status |= kDevNonFinite; }
     else { if (nonfinite_bf16x2(worst)) status |= kDevNonFinite; }
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(0xFFFFFFFFu, status, o);
     if (lane == 0 && status && status_out) atomicOr(status_out, status);
+    if (done) finish_objective(done, partials, nwarps, tab[0].p.objective, reinterpret_cast<double*>(smem_raw));      // the stages are idle by now
     if constexpr (kRows) {
         for (int o = 16; o; o >>= 1) viol += __shfl_xor_sync(0xFFFFFFFFu, viol, o);
         if (lane == 0 && vpartials) vpartials[gw] = viol;
@@ -567,7 +569,7 @@ cudaError_t launch_one(const TmaLaunch& a, const TmaEntry& single, const TmaEntr
     static PerDeviceOnce configured;       // per instantiation
     const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });
     if (e != cudaSuccess) return e;
-    kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status, a.n_keep, a.vpartials);
+    kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status, a.n_keep, a.vpartials, a.done);
     return cudaGetLastError();
 }
 
@@ -608,10 +610,16 @@ cudaError_t tma_reduce(const void* entries_host, const void* entries_dev, int co
 }
 
 // All problems of one launch share dtype and the presence of masked_w_out (the caller groups them).
-cudaError_t launch_tma(const TmaLaunch& a) {
+// A single matrix with work items and a counter word at hand (a_in.done) is one launch: the search kernel reduces its own
+// objective.  Everything else: partials cleared, search, reduction kernel.
+cudaError_t launch_tma(const TmaLaunch& a_in) {
+    TmaLaunch a = a_in;
+    const bool rows_method = a.method == kMethodRows || a.method == kMethodRowsAbsorb;
+    if (!(a.count == 1 && a.total_items > 0 && !rows_method)) a.done = nullptr;
     if (a.M == 8) return launch_tma48(a);
     const int wpc = tma_warps_per_cta(a.dtype, 4, a.method);
-    cudaError_t err = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * wpc, a.stream);
+    cudaError_t err = cudaSuccess;
+    if (!a.done) err = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * wpc, a.stream);
     if (err != cudaSuccess) return err;
     const TmaEntry* host = static_cast<const TmaEntry*>(a.entries_host);
     const TmaEntry* table = static_cast<const TmaEntry*>(a.entries_dev);   // nullptr when count == 1
@@ -623,7 +631,8 @@ cudaError_t launch_tma(const TmaLaunch& a) {
 #undef TM_DISPATCH
         if (err != cudaSuccess) return err;
     }
-    if (a.method == kMethodRows || a.method == kMethodRowsAbsorb) return cudaSuccess;       // the caller sums objective and violation partials together
+    if (rows_method) return cudaSuccess;       // the caller sums objective and violation partials together
+    if (a.done) return cudaSuccess;            // the search kernel has written the objective
     reduce_tma_kernel<<<a.count, 256, 0, a.stream>>>(host[0], table, a.partials, (long long)a.ctas * wpc);
     return cudaGetLastError();
 }

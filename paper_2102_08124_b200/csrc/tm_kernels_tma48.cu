@@ -297,7 +297,7 @@ __device__ __forceinline__ float back_end48(unsigned char* blk, unsigned char* m
 template <int DT, int METHOD, bool HAS_OUT>
 __global__ void __launch_bounds__(Geo48<DT, METHOD>::kWarps * 32, 1)
 tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict__ table, int count, long long total_items,
-             double* __restrict__ partials, int* __restrict__ status_out) {
+             double* __restrict__ partials, int* __restrict__ status_out, unsigned int* __restrict__ done) {
     using G = Geo48<DT, METHOD>;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -469,15 +469,16 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         __syncwarp();
     }
     if (lane == 0) tma_wait_all<0>();
-    if (acc_k >= 0) {
+    if (acc_k >= 0 || done) {                  // a launch that reduces its own objective wants a partial (a zero) from idle warps too
         acc += (double)facc;
         for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-        if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
+        if (lane == 0) partials[(long long)(acc_k >= 0 ? acc_k : 0) * nwarps + gw] = acc;
     }
     if constexpr (DT == kF32) { if (worst >= 0x7F800000u) status |= kDevNonFinite; }
     else { if (nonfinite_bf16x2(worst)) status |= kDevNonFinite; }
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(0xFFFFFFFFu, status, o);
     if (lane == 0 && status && status_out) atomicOr(status_out, status);
+    if (done) finish_objective(done, partials, nwarps, tab[0].p.objective, reinterpret_cast<double*>(smem_raw));      // the stages are idle by now
 }
 
 template <int DT, int METHOD, bool HAS_OUT>
@@ -488,7 +489,7 @@ cudaError_t launch_one48(const TmaLaunch& a, const TmaEntry& single, const TmaEn
     static PerDeviceOnce configured;       // per instantiation
     const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });
     if (e != cudaSuccess) return e;
-    kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status);
+    kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status, a.done);
     return cudaGetLastError();
 }
 
@@ -506,7 +507,9 @@ int tma48_warps_per_cta(int dtype, int method) {
 
 cudaError_t launch_tma48(const TmaLaunch& a) {
     const int wpc = tma48_warps_per_cta(a.dtype, a.method);
-    cudaError_t err = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * wpc, a.stream);
+    // a.done (set only for a single matrix with work items): the search kernel is the whole call
+    cudaError_t err = cudaSuccess;
+    if (!a.done) err = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * wpc, a.stream);
     if (err != cudaSuccess) return err;
     const TmaEntry* host = static_cast<const TmaEntry*>(a.entries_host);
     const TmaEntry* table = static_cast<const TmaEntry*>(a.entries_dev);
@@ -519,6 +522,7 @@ cudaError_t launch_tma48(const TmaLaunch& a) {
 #undef TM_DISPATCH
         if (err != cudaSuccess) return err;
     }
+    if (a.done) return cudaSuccess;
     return tma_reduce(a.entries_host, a.entries_dev, a.count, a.partials, (long long)a.ctas * wpc, a.stream);
 }
 

@@ -275,7 +275,7 @@ __device__ __forceinline__ float back_end_w(unsigned char* blk, int h, unsigned 
 template <bool HAS_OUT>
 __global__ void __launch_bounds__(kSWarps * 32, 1)
 tma48s_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict__ table, int count, long long total_items,
-              double* __restrict__ partials, int* __restrict__ status_out) {
+              double* __restrict__ partials, int* __restrict__ status_out, unsigned int* __restrict__ done) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int b = lane >> 1, h = lane & 1;               // my block of the item, my half of its rows
@@ -421,14 +421,15 @@ tma48s_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restric
         __syncwarp();
     }
     if (lane == 0) tma_wait_all<0>();
-    if (acc_k >= 0) {
+    if (acc_k >= 0 || done) {                  // a launch that reduces its own objective wants a partial (a zero) from idle warps too
         acc += (double)facc;
         for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(kAll, acc, o);
-        if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
+        if (lane == 0) partials[(long long)(acc_k >= 0 ? acc_k : 0) * nwarps + gw] = acc;
     }
     if (nonfinite) status |= kDevNonFinite;
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(kAll, status, o);
     if (lane == 0 && status && status_out) atomicOr(status_out, status);
+    if (done) finish_objective(done, partials, nwarps, tab[0].p.objective, reinterpret_cast<double*>(smem_raw));      // the stages are idle by now
 }
 
 template <bool HAS_OUT>
@@ -438,7 +439,7 @@ cudaError_t launch_one48s(const TmaLaunch& a, const TmaEntry& single, const TmaE
     static PerDeviceOnce configured;       // per instantiation
     const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });
     if (e != cudaSuccess) return e;
-    kern<<<a.ctas, kSWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status);
+    kern<<<a.ctas, kSWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status, a.done);
     return cudaGetLastError();
 }
 
@@ -447,7 +448,7 @@ cudaError_t launch_one48s(const TmaLaunch& a, const TmaEntry& single, const TmaE
 int tma48s_warps_per_cta() { return kSWarps; }
 int tma48s_item_cols() { return kSCols; }
 
-// The search kernel only (launch_tma48 clears the partials before and reduces them after).
+// The search kernel only (launch_tma48 clears the partials before and reduces them after, unless a.done makes the kernel do it).
 cudaError_t launch_tma48s(const TmaLaunch& a) {
     const TmaEntry* host = static_cast<const TmaEntry*>(a.entries_host);
     const TmaEntry* table = static_cast<const TmaEntry*>(a.entries_dev);

@@ -44,6 +44,33 @@ __device__ __forceinline__ int find_matrix(const TmaEntry* tab, int count, long 
     return n;
 }
 
+// End of a single-matrix launch that reduces its own objective (`done` is a 32-bit count in device memory that is zero when
+// the launch starts).  Every warp of the grid has stored its partial sum -- a zero if it had no work item -- at
+// partials[its index]; all threads of the CTA call this once, as the last thing they do.  The CTA that arrives last adds the
+// nwarps partials in an order that depends on nothing but nwarps and the CTA's size (so the same launch gives the same
+// bits whichever CTA that is), writes the objective and sets the count back to zero for the next launch.  Nobody waits for
+// anybody: the earlier CTAs just leave.  `scratch`: 32 doubles of shared memory that nothing else uses any more.
+__device__ __forceinline__ void finish_objective(unsigned int* done, const double* partials, long long nwarps, double* objective, double* scratch) {
+    __shared__ int is_last;
+    __threadfence();                                   // my warp's partial is visible to the grid before the CTA is counted
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = atomicAdd(done, 1u) == gridDim.x - 1 ? 1 : 0;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    double s = 0.0;
+    for (long long i = threadIdx.x; i < nwarps; i += blockDim.x) s += __ldcg(partials + i);
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += scratch[w];
+        if (objective) *objective = t;
+        *done = 0u;
+    }
+}
+
 // Walks the work items of a table of problems in order: problem k, block row bi, column chunk cj.
 struct Cursor {
     int k, bi, cj, cchunks, brows;
