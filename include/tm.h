@@ -149,12 +149,13 @@ size_t tm_workspace_bytes(const tm_problem* probs_host, int count);
  * scratch": the mask is refreshed every 40 iterations).  tm_plan_create validates the descriptors, builds the
  * tensor maps and copies the descriptor tables into the workspace once (synchronising stream 0; it allocates
  * host memory for the plan, nothing on the device).  tm_plan_run then only clears the objective partials and
- * launches the kernels on cuda_stream (a group of one matrix is a single launch that reduces its own objective
- * and needs no clearing): it touches no host memory asynchronously, so it can be recorded by a stream capture
+ * launches the kernels on cuda_stream (the full searches on 16-byte aligned matrices are a single launch that
+ * reduces its own objectives and needs no clearing): it touches no host memory asynchronously, so it can be recorded by a stream capture
  * and replayed.  The workspace belongs to the plan until tm_plan_destroy -- its first 256 bytes are cleared at
  * creation and must not be written by anyone else -- and the matrices must stay where they were (same pointers,
  * shapes, pitches).  Masks and masked weights equal tm_find_mask_batched()'s bit for bit; objectives too, except
- * that a single-matrix group adds its partial sums in another (fixed) order, i.e. equal up to fp64 rounding.
+ * that a launch which reduces its own objectives adds the partial sums in another (fixed) order, i.e. equal
+ * up to fp64 rounding.
  */
 typedef struct tm_plan tm_plan;
 int tm_plan_create(const tm_problem* probs_host, int count, int N, int M, int method, void* workspace_dev, size_t workspace_bytes,

@@ -18,7 +18,7 @@ constexpr int kPartialSlots = 8192;   // objective partials per matrix: (CTAs x 
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
 constexpr size_t kHeaderBytes = 256;  // reserved head of every workspace
-// Inside the header: the count of finished CTAs of a single-matrix bandwidth launch that reduces its own objective.  Only
+// Inside the header: the count of finished CTAs of a bandwidth launch that reduces its own objectives.  Only
 // workspaces whose header the library itself has cleared use it (every such launch leaves it at zero again).
 constexpr size_t kDoneOffset = 128;
 
@@ -180,7 +180,7 @@ int build_plan(const tm_problem* probs, int count, int N, int M, int method, voi
             const int cap = dev.sms < kPartialSlots / wpc ? dev.sms : kPartialSlots / wpc;
             a.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));
             a.entries_dev = n > 1 ? dent + (size_t)used * esz : nullptr;
-            a.done = header_clear && n == 1 ? reinterpret_cast<unsigned int*>(base + kDoneOffset) : nullptr;
+            a.done = header_clear ? reinterpret_cast<unsigned int*>(base + kDoneOffset) : nullptr;
         }
         used += n;
     }

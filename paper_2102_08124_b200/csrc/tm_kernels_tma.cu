@@ -306,6 +306,10 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     }
 
     const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
+    // several matrices in a launch that reduces its own objectives: a warp's partial for matrix k goes to slot order + k
+    // (see finish_objectives_ranged; the warps hold contiguous item ranges in even_share()'s order)
+    const bool ranged = done != nullptr && count > 1;
+    const long long order = (long long)warp * gridDim.x + blockIdx.x;
     // A fixed deal of the items, so the objective's partial sums are reproducible.  Where the kernel waits for memory
     // (Algorithm 1 alone, the 1-D pruning) the warps take the items round-robin -- first, first + nwarps, ... -- so that the
     // whole grid works on one dense window of the matrix (3 % faster there); the full search, which also waits for the
@@ -366,7 +370,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             if (acc_k >= 0) {
                 acc += (double)facc;
                 for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-                if (lane == 0) partials[(long long)acc_k * nwarps + gw] = acc;
+                if (lane == 0) partials[ranged ? order + acc_k : (long long)acc_k * nwarps + gw] = acc;
             }
             acc = 0.0; facc = 0.f; acc_k = cur.k;
             const DevProblem& P = tab[cur.k].p;
@@ -529,16 +533,19 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         for (int s = 0; s < G::kStages; ++s) { mbar_wait_bounded(&bars[s], 0, 1u << 14); mbar_wait_bounded(&bars[s], 1, 1u << 14); }
     }
     if (lane == 0) tma_wait_all<0>();
-    if (acc_k >= 0 || done) {                  // a launch that reduces its own objective wants a partial (a zero) from idle warps too
+    if (acc_k >= 0 || (done && !ranged)) {     // a single-matrix launch that reduces its own objective wants a partial (a zero) from idle warps too
         acc += (double)facc;
         for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-        if (lane == 0) partials[(long long)(acc_k >= 0 ? acc_k : 0) * nwarps + gw] = acc;
+        if (lane == 0) partials[ranged ? order + acc_k : (long long)(acc_k >= 0 ? acc_k : 0) * nwarps + gw] = acc;
     }
     if constexpr (DT == kF32) { if (worst >= 0x7F800000u) status |= kDevNonFinite; }
     else { if (nonfinite_bf16x2(worst)) status |= kDevNonFinite; }
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(0xFFFFFFFFu, status, o);
     if (lane == 0 && status && status_out) atomicOr(status_out, status);
-    if (done) finish_objective(done, partials, nwarps, tab[0].p.objective, reinterpret_cast<double*>(smem_raw));      // the stages are idle by now
+    if (done) {                                // the launch reduces its own objectives; the stages are idle by now
+        if (ranged) finish_objectives_ranged(done, partials, tab, count, total_items, nwarps);
+        else finish_objective(done, partials, nwarps, tab[0].p.objective, reinterpret_cast<double*>(smem_raw));
+    }
     if constexpr (kRows) {
         for (int o = 16; o; o >>= 1) viol += __shfl_xor_sync(0xFFFFFFFFu, viol, o);
         if (lane == 0 && vpartials) vpartials[gw] = viol;
@@ -610,12 +617,14 @@ cudaError_t tma_reduce(const void* entries_host, const void* entries_dev, int co
 }
 
 // All problems of one launch share dtype and the presence of masked_w_out (the caller groups them).
-// A single matrix with work items and a counter word at hand (a_in.done) is one launch: the search kernel reduces its own
-// objective.  Everything else: partials cleared, search, reduction kernel.
+// With a counter word at hand (a_in.done) a single matrix, or several under a full search, is one launch: the search kernel
+// reduces its own objectives.  Everything else: partials cleared, search, reduction kernel.
 cudaError_t launch_tma(const TmaLaunch& a_in) {
     TmaLaunch a = a_in;
     const bool rows_method = a.method == kMethodRows || a.method == kMethodRowsAbsorb;
-    if (!(a.count == 1 && a.total_items > 0 && !rows_method)) a.done = nullptr;
+    // several matrices only where the warps hold contiguous item ranges (the full searches; Algorithm 1 alone deals round-robin)
+    const bool contiguous = a.method == kMethodApprox || (a.method == kMethodExact && a.M == 4);
+    if (!((a.count == 1 || contiguous) && a.total_items > 0 && !rows_method)) a.done = nullptr;
     if (a.M == 8) return launch_tma48(a);
     const int wpc = tma_warps_per_cta(a.dtype, 4, a.method);
     cudaError_t err = cudaSuccess;

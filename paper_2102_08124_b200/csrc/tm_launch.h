@@ -54,8 +54,8 @@ struct TmaLaunch {
     bool has_out;               // masked_w_out present (all problems of one launch agree)
     int n_keep = 2;             // kMethodRows / kMethodRowsAbsorb: entries kept per group of four (1..3)
     unsigned long long* vpartials = nullptr;   // kMethodRows / kMethodRowsAbsorb (count == 1): ctas * warps pattern-violation partials; the caller reduces
-    unsigned int* done = nullptr;              // a device word that is zero between launches, or nullptr: with it a single-matrix search is ONE
-                                               // launch (every warp stores a partial, the CTA that finishes last adds them up) instead of three
+    unsigned int* done = nullptr;              // a device word that is zero between launches, or nullptr: with it a search is ONE launch where
+                                               // it can be (the warps store partials, the CTA that finishes last adds them up) instead of three
     cudaStream_t stream;
 };
 size_t tma_entry_bytes();

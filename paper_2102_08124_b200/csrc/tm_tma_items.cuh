@@ -71,6 +71,40 @@ __device__ __forceinline__ void finish_objective(unsigned int* done, const doubl
     }
 }
 
+// The same for a launch over several matrices whose warps hold contiguous item ranges dealt by even_share().  A warp that
+// worked on matrix k has stored its partial sum for it at partials[order + k] (order = its place in even_share()'s order;
+// the pairs (order, k) of a launch are strictly increasing in both, so the slots are distinct and number at most
+// nwarps + count), and nothing else is ever read: which warps worked on matrix k follows from its first and last item, so
+// the buffer needs no clearing.  The CTA that arrives last gives every matrix to one of its warps, which adds the matrix's
+// partials in a fixed order.
+__device__ __forceinline__ long long even_share_owner(long long item, long long q, long long rem) {
+    return item < rem * (q + 1) ? item / (q + 1) : rem + (item - rem * (q + 1)) / q;
+}
+__device__ __forceinline__ void finish_objectives_ranged(unsigned int* done, const double* partials, const TmaEntry* tab, int count,
+                                                          long long total_items, long long nwarps) {
+    __shared__ int is_last_r;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last_r = atomicAdd(done, 1u) == gridDim.x - 1 ? 1 : 0;
+    __syncthreads();
+    if (!is_last_r) return;
+    __threadfence();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
+    const long long q = total_items / nwarps, rem = total_items - q * nwarps;
+    for (int k = warp; k < count; k += warps) {
+        const long long n = (long long)tab[k].brows * tab[k].cchunks, begin = tab[k].p.item_begin;
+        double s = 0.0;
+        if (n > 0) {
+            const long long o0 = even_share_owner(begin, q, rem), o1 = even_share_owner(begin + n - 1, q, rem);
+            for (long long o = o0 + lane; o <= o1; o += 32) s += __ldcg(partials + o + k);
+        }
+        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        if (lane == 0 && tab[k].p.objective) *tab[k].p.objective = s;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) *done = 0u;
+}
+
 // Walks the work items of a table of problems in order: problem k, block row bi, column chunk cj.
 struct Cursor {
     int k, bi, cj, cchunks, brows;

@@ -42,13 +42,41 @@ def test_plan_equals_batched_call(N, M, method):
         for k in range(len(Ws)):
             assert np.array_equal(to_host_bits(masks[k]), to_host_bits(ref_masks[k]))
             assert np.array_equal(to_host_bits(maskeds[k]), to_host_bits(ref_maskeds[k]))
-        assert np.array_equal(objs.cpu().numpy(), ref_obj.cpu().numpy())
+        # a plan's launch adds up its own partial sums, in another fixed order than the batched call's reduction kernel
+        assert np.allclose(objs.cpu().numpy(), ref_obj.cpu().numpy(), rtol=1e-12, atol=0.0)
     # and, directly, the CPU oracle's answer on the same bytes
     for k, m in enumerate(mats):
         want = orc.find_mask(m, N, M, {tm.TM_APPROX: orc.APPROX, tm.TM_EXACT: orc.EXACT}[method])
         assert np.array_equal(to_host_bits(masks[k]), want["mask"])
         assert np.array_equal(to_host_bits(maskeds[k]), want["masked"].view(np.uint16 if m.dtype == np.uint16 else np.uint32))
         assert abs(float(objs[k].item()) - want["objective"]) <= 1e-6 * abs(want["objective"])
+    tm.tm_plan_destroy(plan)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("N,M,method", [(2, 4, tm.TM_APPROX), (4, 8, tm.TM_APPROX), (2, 4, tm.TM_EXACT), (2, 4, tm.TM_APPROX_COVER)])
+def test_plan_reduces_its_own_objectives(N, M, method):
+    """Many matrices of one dtype in a plan: one launch whose last thread block adds up every matrix's partial sums.  Sizes from
+    a single work item (most warps idle) to thousands (every warp holds several matrices or a piece of one), an empty matrix in
+    the middle; run three times in a row (the count of finished blocks must return to zero)."""
+    shapes = [(8, 520), (256, 2056), (8, 8), (0, 64), (1024, 4096), (16, 136), (64, 1032), (8, 16), (2048, 1024), (40, 3080)]
+    mats = [workloads.quantised_bf16(r, c, 0.02, 300 + i) if r else np.zeros((0, c), np.uint16) for i, (r, c) in enumerate(shapes)]
+    Ws = [to_device(m) if m.size else torch.empty((0, m.shape[1]), dtype=torch.bfloat16, device="cuda") for m in mats]
+    plan = tm.tm_plan_create(Ws, N, M, method)
+    omethod = {tm.TM_APPROX: orc.APPROX, tm.TM_EXACT: orc.EXACT, tm.TM_APPROX_COVER: orc.APPROX_COVER}[method]
+    want = [orc.find_mask(m, N, M, omethod) if m.size else None for m in mats]
+    for rep in range(3):
+        plan.batch.objectives.fill_(-1.0)
+        masks, maskeds, objs, status = tm.tm_plan_run(plan)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for k, m in enumerate(mats):
+            if want[k] is None:
+                assert float(objs[k].item()) == 0.0
+                continue
+            assert np.array_equal(to_host_bits(masks[k]), want[k]["mask"]), (rep, k)
+            assert np.array_equal(to_host_bits(maskeds[k]), want[k]["masked"].view(np.uint16)), (rep, k)
+            assert abs(float(objs[k].item()) - want[k]["objective"]) <= 1e-6 * abs(want[k]["objective"]), (rep, k)
     tm.tm_plan_destroy(plan)
 
 
