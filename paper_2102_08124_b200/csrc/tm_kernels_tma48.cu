@@ -310,10 +310,10 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     __syncthreads();
 
     const long long gw = (long long)blockIdx.x * G::kWarps + warp, nwarps = (long long)gridDim.x * G::kWarps;
-    // several matrices in a launch that reduces its own objectives: a warp's partial for matrix k goes to slot order + k
-    // (see finish_objectives_ranged; the warps hold contiguous item ranges in even_share()'s order)
+    // where this warp's objective partial for matrix k goes: k * pstride + pbase (a launch over several matrices that reduces
+    // its own objectives packs them: slot = the warp's place in the deal + k, see finish_objectives_ranged)
     const bool ranged = done != nullptr && count > 1;
-    const long long order = (long long)warp * gridDim.x + blockIdx.x;
+    const long long pstride = ranged ? 1 : nwarps, pbase = ranged ? (long long)warp * gridDim.x + blockIdx.x : gw;
     // Algorithm 1 alone takes its items round-robin over the warps of the grid (one dense window of the matrix at a time),
     // the full search contiguous ranges (see the 2:4 kernel)
     constexpr bool kRoundRobin = METHOD != kMethodApprox;
@@ -449,7 +449,7 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             if (acc_k >= 0) {
                 acc += (double)facc;
                 for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-                if (lane == 0) partials[ranged ? order + acc_k : (long long)acc_k * nwarps + gw] = acc;
+                if (lane == 0) partials[(long long)acc_k * pstride + pbase] = acc;
             }
             acc = 0.0; facc = 0.f; acc_k = cur.k;
             const DevProblem& P = tab[cur.k].p;
@@ -473,18 +473,19 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         __syncwarp();
     }
     if (lane == 0) tma_wait_all<0>();
-    if (acc_k >= 0 || (done && !ranged)) {     // a single-matrix launch that reduces its own objective wants a partial (a zero) from idle warps too
+    if (acc_k >= 0 || (done && count == 1)) {  // a single-matrix launch that reduces its own objective wants a partial (a zero) from idle warps too
         acc += (double)facc;
         for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-        if (lane == 0) partials[ranged ? order + acc_k : (long long)(acc_k >= 0 ? acc_k : 0) * nwarps + gw] = acc;
+        if (lane == 0) partials[(long long)(acc_k >= 0 ? acc_k : 0) * pstride + pbase] = acc;
     }
     if constexpr (DT == kF32) { if (worst >= 0x7F800000u) status |= kDevNonFinite; }
     else { if (nonfinite_bf16x2(worst)) status |= kDevNonFinite; }
     for (int o = 16; o; o >>= 1) status |= __shfl_xor_sync(0xFFFFFFFFu, status, o);
     if (lane == 0 && status && status_out) atomicOr(status_out, status);
     if (done) {                                // the launch reduces its own objectives; the stages are idle by now
-        if (ranged) finish_objectives_ranged(done, partials, tab, count, total_items, nwarps);
-        else finish_objective(done, partials, nwarps, tab[0].p.objective, reinterpret_cast<double*>(smem_raw));
+        const long long nw = (long long)gridDim.x * G::kWarps;
+        if (count > 1) finish_objectives_ranged(done, partials, tab, count, total_items, nw, reinterpret_cast<double*>(smem_raw));
+        else finish_objective(done, partials, nw, tab[0].p.objective, reinterpret_cast<double*>(smem_raw));
     }
 }
 

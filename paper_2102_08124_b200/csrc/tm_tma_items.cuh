@@ -49,14 +49,17 @@ __device__ __forceinline__ int find_matrix(const TmaEntry* tab, int count, long 
 // partials[its index]; all threads of the CTA call this once, as the last thing they do.  The CTA that arrives last adds the
 // nwarps partials in an order that depends on nothing but nwarps and the CTA's size (so the same launch gives the same
 // bits whichever CTA that is), writes the objective and sets the count back to zero for the next launch.  Nobody waits for
-// anybody: the earlier CTAs just leave.  `scratch`: 32 doubles of shared memory that nothing else uses any more.
-__device__ __forceinline__ void finish_objective(unsigned int* done, const double* partials, long long nwarps, double* objective, double* scratch) {
-    __shared__ int is_last;
+// anybody: the earlier CTAs just leave.  `scratch`: 33 doubles of shared memory that nothing else uses any more.
+#ifndef TMX_FIN
+#define TMX_FIN static __device__ __noinline__
+#endif
+TMX_FIN void finish_objective(unsigned int* done, const double* partials, long long nwarps, double* objective, double* scratch) {
+    volatile int* is_last = reinterpret_cast<volatile int*>(scratch + 32);
     __threadfence();                                   // my warp's partial is visible to the grid before the CTA is counted
     __syncthreads();
-    if (threadIdx.x == 0) is_last = atomicAdd(done, 1u) == gridDim.x - 1 ? 1 : 0;
+    if (threadIdx.x == 0) *is_last = atomicAdd(done, 1u) == gridDim.x - 1 ? 1 : 0;
     __syncthreads();
-    if (!is_last) return;
+    if (!*is_last) return;
     __threadfence();
     double s = 0.0;
     for (long long i = threadIdx.x; i < nwarps; i += blockDim.x) s += __ldcg(partials + i);
@@ -80,14 +83,14 @@ __device__ __forceinline__ void finish_objective(unsigned int* done, const doubl
 __device__ __forceinline__ long long even_share_owner(long long item, long long q, long long rem) {
     return item < rem * (q + 1) ? item / (q + 1) : rem + (item - rem * (q + 1)) / q;
 }
-__device__ __forceinline__ void finish_objectives_ranged(unsigned int* done, const double* partials, const TmaEntry* tab, int count,
-                                                          long long total_items, long long nwarps) {
-    __shared__ int is_last_r;
+TMX_FIN void finish_objectives_ranged(unsigned int* done, const double* partials, const TmaEntry* tab, int count,
+                                      long long total_items, long long nwarps, double* scratch) {
+    volatile int* is_last = reinterpret_cast<volatile int*>(scratch);
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) is_last_r = atomicAdd(done, 1u) == gridDim.x - 1 ? 1 : 0;
+    if (threadIdx.x == 0) *is_last = atomicAdd(done, 1u) == gridDim.x - 1 ? 1 : 0;
     __syncthreads();
-    if (!is_last_r) return;
+    if (!*is_last) return;
     __threadfence();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
     const long long q = total_items / nwarps, rem = total_items - q * nwarps;
