@@ -21,6 +21,10 @@ constexpr size_t kHeaderBytes = 256;  // reserved head of every workspace
 // Inside the header: the count of finished CTAs of a bandwidth launch that reduces its own objectives.  Only
 // workspaces whose header the library itself has cleared use it (every such launch leaves it at zero again).
 constexpr size_t kDoneOffset = 128;
+// tm_find_mask_host(): row strips whose copy-in, search and copy-out overlap, and the head of its device workspace (status word,
+// then one objective per strip from byte 64 on)
+constexpr int kHostStrips = 16;       // 32 and 64 strips measured the same (27.3 ms on a 12288 x 49152 bf16 matrix) and slower (28.4 ms): the bus is the bound
+constexpr size_t kHostHead = (64 + 8 * (size_t)kHostStrips + kAlign - 1) / kAlign * kAlign;
 
 size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 int at_least_one(int count) { return count > 0 ? count : 1; }
@@ -365,7 +369,7 @@ int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols,
     const size_t row_bytes = (size_t)cols * elem, wpr = tm_mask_words_per_row(cols);
     // row strips: copy-in, search and copy-out of neighbouring strips overlap on three streams
     const int64_t brows = rows / M;
-    const int strips = (int)(brows < 16 ? brows : 16);
+    const int strips = (int)(brows < kHostStrips ? brows : kHostStrips);
     const int64_t strip_brows = (brows + strips - 1) / strips;
     const size_t one_ws = tm_workspace_bytes(nullptr, 1);
     {
@@ -378,13 +382,13 @@ int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols,
         if ((rc = grow(&d->stage_w, &d->stage_w_bytes, (size_t)rows * row_bytes)) != TM_OK) return rc;
         if (masked_w_out_host && (rc = grow(&d->stage_masked, &d->stage_masked_bytes, (size_t)rows * row_bytes)) != TM_OK) return rc;
         if ((rc = grow(&d->stage_mask, &d->stage_mask_bytes, (size_t)rows * wpr * 4)) != TM_OK) return rc;
-        if ((rc = grow(&d->stage_ws, &d->stage_ws_bytes, (one_ws + kAlign) * 16 + kAlign)) != TM_OK) return rc;
+        if ((rc = grow(&d->stage_ws, &d->stage_ws_bytes, (one_ws + kAlign) * kHostStrips + kHostHead)) != TM_OK) return rc;
     }
     char* ws = static_cast<char*>(d->stage_ws);
-    int* status_dev = reinterpret_cast<int*>(ws);                       // first 256 bytes: status + 16 objectives
+    int* status_dev = reinterpret_cast<int*>(ws);                       // the head: status, then the strips' objectives
     double* obj_dev = reinterpret_cast<double*>(ws + 64);
     // status and objectives, and the headers of the strips' workspaces (their launches count finished CTAs there)
-    if (cudaMemsetAsync(ws, 0, (one_ws + kAlign) * 16 + kAlign, d->s_run) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    if (cudaMemsetAsync(ws, 0, (one_ws + kAlign) * kHostStrips + kHostHead, d->s_run) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
 
     std::vector<cudaEvent_t> ev_in((size_t)strips), ev_run((size_t)strips);
     bool ok = true;
@@ -405,7 +409,7 @@ int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols,
         p.mask_out = static_cast<uint32_t*>(d->stage_mask) + (size_t)r0 * wpr;
         p.masked_w_out = masked_w_out_host ? static_cast<char*>(d->stage_masked) + off : nullptr;
         p.objective_out = obj_dev + s;
-        rc = run(&p, 1, N, M, method, ws + kAlign + (size_t)s * (one_ws + kAlign), one_ws, status_dev, d->s_run, *d, true);
+        rc = run(&p, 1, N, M, method, ws + kHostHead + (size_t)s * (one_ws + kAlign), one_ws, status_dev, d->s_run, *d, true);
         if (rc != TM_OK) { ok = false; break; }
         ok &= cudaEventRecord(ev_run[s], d->s_run) == cudaSuccess;
         ok &= cudaStreamWaitEvent(d->s_out, ev_run[s], 0) == cudaSuccess;
@@ -413,7 +417,7 @@ int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols,
         if (masked_w_out_host)
             ok &= cudaMemcpyAsync(static_cast<char*>(masked_w_out_host) + off, p.masked_w_out, nbytes, cudaMemcpyDeviceToHost, d->s_out) == cudaSuccess;
     }
-    double obj_host[16] = {0}; int status_host = 0;
+    double obj_host[kHostStrips] = {0}; int status_host = 0;
     if (ok) {
         ok &= cudaStreamSynchronize(d->s_run) == cudaSuccess;
         ok &= cudaMemcpy(obj_host, obj_dev, sizeof(double) * (size_t)strips, cudaMemcpyDeviceToHost) == cudaSuccess;
