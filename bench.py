@@ -34,7 +34,7 @@ N_KEEP, M_BLOCK = 2, 4
 BYTES_PER_WEIGHT = 2 + 2 + 1.0 / 8          # read W, write masked W, write one mask bit (bf16)
 # dram__bytes_read.sum + dram__bytes_write.sum of one full-size launch of the search kernel in steady state (mean of three
 # consecutive launches after the first, caches not flushed between them); None when the kernel has changed since the counters were taken
-TRAFFIC_BYTES_PER_LAUNCH = 1207.96e6 + 1282.74e6
+TRAFFIC_BYTES_PER_LAUNCH = 1207.99e6 + 1282.66e6
 TRAFFIC_SOURCE = ("ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --cache-control none on the full-size launch "
                   "(profiles/tma24_kernel_approx_2_4_bf16_12288x49152_launches.md)")
 METRIC = "transposable-mask weights/s (2:4 approx, bf16, 1 GPU: achieved HBM GB/s vs peak in `roofline`)"

@@ -54,8 +54,11 @@ template <int DT, int METHOD> struct Geometry {
     static constexpr int kRowPitch = kItemCols * kElem;        // bytes between rows inside a stage
     static constexpr int kHalfBytes = kHalfCols * kElem;       // from the first half of a row to the second
     static constexpr int kStageBytes = kItemRows * kRowPitch;
-    // stages | mask bytes [half][4][32] | kept [2][32] | queue [128] | barriers
-    static constexpr int kWarpBytes = kStages * kStageBytes + 256 + 256 + 128 + 128;
+    // exact search: one bit per item of the warp, set when the item is set aside for the out-of-line scorer after the loop
+    static constexpr int kAsideBytes = METHOD == kMethodExact ? 2048 : 0;
+    static constexpr int kAsideItems = kAsideBytes * 8;
+    // stages | mask bytes [half][4][32] | kept [2][32] | queue [128] | barriers | set-aside bits
+    static constexpr int kWarpBytes = kStages * kStageBytes + 256 + 256 + 128 + 128 + kAsideBytes;
     static constexpr int kSmemBytes = kWarps * kWarpBytes + (DT == kBF16 ? kLaneLutBytes : 0);
     static_assert(kSmemBytes <= 232448, "at most 227 KB of shared memory per CTA");
     static_assert(kWarpBytes % 128 == 0, "stages stay 128-byte aligned");
@@ -161,6 +164,87 @@ __device__ __forceinline__ bool swap_apply_smem(const unsigned char* blk, uint32
         if constexpr (DT == kBF16) return *reinterpret_cast<const unsigned short*>(at) & 0x7FFFu;
         else return *reinterpret_cast<const uint32_t*>(at) & 0x7FFFFFFFu;
     });
+}
+
+// Exact search, after the item loop: the items that were set aside because some block of theirs does not fit the first tier
+// of the scorer (bit `it` of `aside` for the warp's item number `it`; the warp's items start at `first`).  Nothing of such an
+// item has been written.  They are few, so they go the plain way: every lane reads its four blocks of the item from the
+// matrix, scores them with exact_2_4_any() -- every tier, out of line -- and stores masked weights and mask words itself; the
+// warp's sum goes on top of the partial it has already stored for the item's matrix.
+template <int DT>
+static __device__ __noinline__ void exact_aside_pass(const TmaEntry* tab, int count, long long first, int n_items, const uint32_t* aside,
+                                                      double* partials, long long pstride, long long pbase) {
+    constexpr int kWords = DT == kF32 ? 4 : 2;                     // 32-bit words of a block's row
+    const int lane = threadIdx.x & 31;
+    const int words = ((n_items < Geometry<DT, kMethodExact>::kAsideItems ? n_items : Geometry<DT, kMethodExact>::kAsideItems) + 31) >> 5;
+    for (int w = 0; w < words; ++w) {
+        uint32_t bits = aside[w];                                  // the same word for every lane
+        while (bits) {
+            const int it = w * 32 + __ffs((int)bits) - 1;
+            bits &= bits - 1;
+            Cursor c;
+            c.seek(tab, count, first + it);
+            const DevProblem& P = tab[c.k].p;
+            const long long r0 = (long long)c.bi * kItemRows;
+            const size_t pitch = (size_t)P.ld * (DT == kF32 ? 4 : 2);
+            float sum = 0.f;
+            for (int h = 0; h < kHalves; ++h) {
+                const long long c0 = (long long)c.cj * kItemCols + h * kHalfCols + lane * 8;
+                uint32_t nib[4] = {0, 0, 0, 0};                    // row i: block A's keep nibble, block B's above it
+                for (int b = 0; b < 2; ++b) {
+                    const long long cb = c0 + 4 * b;
+                    const bool present = cb < P.cols;              // cols % 4 == 0: a block is inside or outside as a whole
+                    uint32_t raw[4][kWords], u[16];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const unsigned char* src = static_cast<const unsigned char*>(P.W) + (size_t)(r0 + i) * pitch + (size_t)cb * (DT == kF32 ? 4 : 2);
+                        if constexpr (DT == kF32) {
+                            const uint4 v = present ? *reinterpret_cast<const uint4*>(src) : make_uint4(0, 0, 0, 0);
+                            raw[i][0] = v.x; raw[i][1] = v.y; raw[i][2] = v.z; raw[i][3] = v.w;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) u[4 * i + j] = raw[i][j] & 0x7FFFFFFFu;
+                        } else {
+                            const uint2 v = present ? *reinterpret_cast<const uint2*>(src) : make_uint2(0, 0);
+                            raw[i][0] = v.x; raw[i][1] = v.y;
+                            u[4 * i] = (v.x << 16) & 0x7FFFFFFFu; u[4 * i + 1] = v.x & 0x7FFF0000u;
+                            u[4 * i + 2] = (v.y << 16) & 0x7FFFFFFFu; u[4 * i + 3] = v.y & 0x7FFF0000u;
+                        }
+                    }
+                    uint32_t code = exact_2_4_any(u, DT == kBF16 ? 16 : 0);      // all 32 lanes call
+                    if (!present) code = 0;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t n = (code >> (4 * i)) & 15u;
+                        nib[i] |= n << (4 * b);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) sum += ((n >> j) & 1u) ? __uint_as_float(u[4 * i + j]) : 0.f;
+                        if (P.masked && present) {
+                            unsigned char* dst = static_cast<unsigned char*>(P.masked) + (size_t)(r0 + i) * pitch + (size_t)cb * (DT == kF32 ? 4 : 2);
+                            if constexpr (DT == kF32) {
+                                *reinterpret_cast<uint4*>(dst) = make_uint4((n & 1u) ? raw[i][0] : 0u, (n & 2u) ? raw[i][1] : 0u, (n & 4u) ? raw[i][2] : 0u, (n & 8u) ? raw[i][3] : 0u);
+                            } else {
+                                const uint32_t m0 = ((n & 1u) ? 0x0000FFFFu : 0u) | ((n & 2u) ? 0xFFFF0000u : 0u);
+                                const uint32_t m1 = ((n & 4u) ? 0x0000FFFFu : 0u) | ((n & 8u) ? 0xFFFF0000u : 0u);
+                                *reinterpret_cast<uint2*>(dst) = make_uint2(raw[i][0] & m0, raw[i][1] & m1);
+                            }
+                        }
+                    }
+                }
+                // four lanes share a mask word
+                const long long word = c0 >> 5;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint32_t wbits = nib[i] << (8 * (lane & 3));
+                    wbits |= __shfl_xor_sync(0xFFFFFFFFu, wbits, 1);
+                    wbits |= __shfl_xor_sync(0xFFFFFFFFu, wbits, 2);
+                    if ((lane & 3) == 0 && word < P.wpr) P.mask[(r0 + i) * P.wpr + word] = wbits;
+                }
+            }
+            double t = (double)sum;
+            for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+            if (lane == 0) partials[(long long)c.k * pstride + pbase] += t;
+        }
+    }
 }
 
 // Masked weights back into the stage, mask bytes, objective contribution of the lane's two blocks.
@@ -299,6 +383,10 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     uint32_t* kbuf = reinterpret_cast<uint32_t*>(mbytes + 256);
     unsigned char* queue = reinterpret_cast<unsigned char*>(kbuf + kHalves * 32);
     uint64_t* bars = reinterpret_cast<uint64_t*>(queue + 128);
+    uint32_t* aside = reinterpret_cast<uint32_t*>(queue + 256);            // exact search only
+    if constexpr (METHOD == kMethodExact) {
+        for (int w = lane; w < G::kAsideBytes / 4; w += 32) aside[w] = 0u;
+    }
     uint4* lut = reinterpret_cast<uint4*>(smem_raw + (size_t)G::kWarps * G::kWarpBytes);
     if constexpr (DT == kBF16) {           // the only CTA-wide step: the lane-mask table
         fill_lane_lut(lut, threadIdx.x, G::kWarps * 32);
@@ -358,14 +446,21 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     const unsigned char* msrc = mbytes + (mw >> 3) * 128 + mr * 32 + (mw & 7) * 4;
     unsigned long long viol = 0;                                         // kMethodRows: non-zero entries pruned by this lane
 
-    for (int it = 0; it < n_items && alive; ++it) {
+    // The item loop.  The exact search on bf16 has it twice: with the 32-bit first tier of the scorer and, for a warp whose
+    // items leave that tier often (ordinary continuous data does, quantised data never), with the 64-bit one; a warp
+    // starts with the first and may change over once, between two items (the pipeline's state is the captured variables).
+    constexpr bool kTwoTiers = METHOD == kMethodExact && DT == kBF16;
+    auto run_items = [&](auto wide_mode, int it_begin) -> int {
+    constexpr bool kWideTier = decltype(wide_mode)::value;
+    int it = it_begin, recent_aside = 0;
+    for (; it < n_items && alive; ++it) {
         const int s = it % G::kStages;
         const uint32_t parity = (uint32_t)((it / G::kStages) & 1);
         unsigned char* stage = stages + s * G::kStageBytes;
         // a copy that never landed: stop before anything is computed on, or stored from, the unfilled stage
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&bars[s], parity))) { status |= kDevInternal; alive = false; break; }
         int qn = 0;
-        bool redo = false;                                      // exact search on bf16: the item needs the later tiers
+        bool redo = false;                                      // exact search: some block of the item is outside the first tier (warp-uniform)
         if (cur.k != acc_k) {                                   // a new matrix starts: flush the objective partial
             if (acc_k >= 0) {
                 acc += (double)facc;
@@ -407,8 +502,7 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                     for (int p = 0; p < 16; ++p) bad |= (u[p] >> 23) == 0xFFu;
                     if (bad) status |= kDevNonFinite;
                     uint64_t code = 0;
-                    if constexpr (DT == kBF16) { if (!redo) redo = !exact_2_4_bf16_first(u, code); }     // first tier or, later, all four blocks again
-                    else code = exact_2_4(u, 0);
+                    if (!redo) redo = !exact_2_4_first<DT == kBF16, kWideTier>(u, code);       // once set, the whole item is scored again after the loop
                     k |= (uint32_t)code << (16 * b);
                 }
             } else {
@@ -464,16 +558,6 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                 issue_next((s + G::kStages - 1) % G::kStages);
             }
         }
-        if constexpr (METHOD == kMethodExact && DT == kBF16) {
-            if (redo) {                    // some block of this item (warp-uniform) does not fit the first tier
-#pragma unroll 1
-                for (int h = 0; h < kHalves; ++h) {
-                    uint32_t codes[2];
-                    exact_2_4_bf16_rest(stage + h * G::kHalfBytes + lane * (8 * G::kElem), G::kRowPitch, 4 * G::kElem, 2, codes);
-                    kbuf[h * 32 + lane] = codes[0] | (codes[1] << 16);
-                }
-            }
-        }
         __syncwarp();
         // ---- step C on the queued blocks ---------------------------------------------------------
         if constexpr (METHOD == kMethodApprox) {
@@ -491,6 +575,12 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             __syncwarp();
         }
         // ---- outputs ---------------------------------------------------------------------------
+        if (METHOD == kMethodExact && redo) {
+            // set aside: nothing of this item is written here (in place, its weights stay as they are); exact_aside_pass() does it
+            if (it >= G::kAsideItems) status |= kDevInternal;              // the launcher refuses calls whose warps would get that many items
+            else if (lane == 0) aside[it >> 5] |= 1u << (it & 31);
+            ++recent_aside;
+        } else {
         // blocks past the last column (zero-filled by the copy) contribute nothing
         uint32_t colmask[kHalves] = {0xFFFFFFFFu, 0xFFFFFFFFu};
         if (!inside_cols) {
@@ -524,9 +614,20 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                 if (row + 2 < p_rows) dst[2 * (long long)p_wpr] = w1;
             }
         }
+        }
         cur.advance(tab, count);
         if ((it & 31) == 31) { acc += (double)facc; facc = 0.f; }           // keep the fp32 partial short
         __syncwarp();
+        if constexpr (kTwoTiers && !kWideTier) {
+            if (recent_aside >= 2) { ++it; break; }                         // two items set aside within a window of four: the wider tier from here on
+            if (((it - it_begin) & 3) == 3) recent_aside = 0;
+        }
+    }
+    return it;
+    };
+    {
+        const int reached = run_items(std::false_type{}, 0);
+        if constexpr (kTwoTiers) { if (reached < n_items && alive) run_items(std::true_type{}, reached); }
     }
     if (!alive && lane == 0) {
         // a copy never landed: give the copies still in flight a bounded chance to finish before the stages die
@@ -537,6 +638,10 @@ tma24_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         acc += (double)facc;
         for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
         if (lane == 0) partials[(long long)(acc_k >= 0 ? acc_k : 0) * pstride + pbase] = acc;
+    }
+    if constexpr (METHOD == kMethodExact) {
+        __syncwarp();
+        if (alive) exact_aside_pass<DT>(tab, count, first, n_items, aside, partials, pstride, pbase);
     }
     if constexpr (DT == kF32) { if (worst >= 0x7F800000u) status |= kDevNonFinite; }
     else { if (nonfinite_bf16x2(worst)) status |= kDevNonFinite; }
@@ -628,6 +733,9 @@ cudaError_t launch_tma(const TmaLaunch& a_in) {
     if (!((a.count == 1 || contiguous) && a.total_items > 0 && !rows_method)) a.done = nullptr;
     if (a.M == 8) return launch_tma48(a);
     const int wpc = tma_warps_per_cta(a.dtype, 4, a.method);
+    // the exact search keeps one bit per item of a warp (16 384 of them: more than 180 GB of weights on a full grid)
+    if (a.method == kMethodExact && (a.total_items + (long long)a.ctas * wpc - 1) / ((long long)a.ctas * wpc) > Geometry<kBF16, kMethodExact>::kAsideItems)
+        return cudaErrorInvalidValue;
     cudaError_t err = cudaSuccess;
     if (!a.done) err = cudaMemsetAsync(a.partials, 0, sizeof(double) * (size_t)a.count * (size_t)a.ctas * wpc, a.stream);
     if (err != cudaSuccess) return err;

@@ -399,36 +399,38 @@ __device__ __forceinline__ uint64_t exact_2_4(const uint32_t (&u)[16], int drop_
     return exact_2_4_wide(u, Emin);
 }
 
-// The two halves of exact_2_4() for bf16 blocks that sit in shared memory, kept apart so that the common case pays nothing
-// for the rare one: with the later tiers inlined beside it the first tier's caller spilled 480 bytes a thread at 96
-// registers, and waiting for those loads was most of its time (0.84 ms against 0.52 ms on a 12288 x 49152 matrix).
-// exact_2_4_bf16_first: the first tier alone; false (nothing computed) unless every lane's block fits it.
-// exact_2_4_bf16_rest: out of line and called where little is live: scores the lane's n_blocks blocks (block_pitch bytes
-// apart, row_pitch bytes between a block's rows) again from shared memory with whatever tier each needs, 16-bit codes to
-// codes[].  Both are called by all 32 lanes.
-__device__ __forceinline__ bool exact_2_4_bf16_first(const uint32_t (&u)[16], uint64_t& code) {
-    uint32_t umax = 0, umin1 = 0xFFFFFFFFu;
+// exact_2_4() in two parts for the pipelined kernel, so that the common case pays nothing for the rare one.  With the later
+// tiers inlined beside it the first tier's loop spilled 480 bytes a thread at 96 registers; with them behind a call inside
+// the loop the values that live across the call went to local memory on the way of every item (46 local loads per item).  So
+// the loop holds a first tier only, an item with a block outside it is set aside, and exact_2_4_any() -- out of line --
+// scores such items after the loop.  Both are called by all 32 lanes.
+// exact_2_4_first: false (nothing computed) unless every lane's block fits the tier:
+//   bf16  at most 9 binades between the largest and the smallest non-zero entry, no subnormals: 32-bit class sums;
+//   fp32  at most 19 binades: 64-bit class sums.
+//   bf16, WIDE  (for data that leaves the 32-bit tier often) at most 35 binades: 64-bit class sums of the 8-bit significands.
+template <bool BF16, bool WIDE>
+__device__ __forceinline__ bool exact_2_4_first(const uint32_t (&u)[16], uint64_t& code) {
+    uint32_t umax = 0, umin1 = 0xFFFFFFFFu;                  // u - 1 sends zero to the top
 #pragma unroll
     for (int p = 0; p < 16; ++p) { umax = max(umax, u[p]); umin1 = min(umin1, u[p] - 1u); }
     const int emax = (int)(umax >> 23), emin = (int)((umin1 + 1u) >> 23);
-    const bool fits = umax == 0u || (emin >= 19 && emax - emin <= 9);
-    if (!__all_sync(0xFFFFFFFFu, fits)) return false;
-    code = exact_2_4_classes32<true>(u, umax ? emin : 127);
+    if constexpr (BF16 && WIDE) {
+        const bool fits = umax == 0u || (emin >= 1 && emax - emin <= 35);
+        if (!__all_sync(0xFFFFFFFFu, fits)) return false;
+        code = exact_2_4_classes(u, umax ? emin : 1, 16);
+    } else if constexpr (BF16) {
+        const bool fits = umax == 0u || (emin >= 19 && emax - emin <= 9 && emax < 255);      // Inf / NaN patterns take the integer tiers
+        if (!__all_sync(0xFFFFFFFFu, fits)) return false;
+        code = exact_2_4_classes32<true>(u, umax ? emin : 127);
+    } else {
+        const bool fits = umax == 0u || (emin >= 1 && emax - emin <= 19);        // normal numbers: the exponent field is split_float()'s E
+        if (!__all_sync(0xFFFFFFFFu, fits)) return false;
+        code = exact_2_4_classes(u, umax ? emin : 1, 0);
+    }
     return true;
 }
-static __device__ __noinline__ void exact_2_4_bf16_rest(const unsigned char* blocks, int row_pitch, int block_pitch, int n_blocks, uint32_t* codes) {
-    for (int b = 0; b < n_blocks; ++b) {
-        const unsigned char* blk = blocks + b * block_pitch;
-        uint32_t u[16];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint2 v = *reinterpret_cast<const uint2*>(blk + i * row_pitch);
-            u[4 * i] = (v.x << 16) & 0x7FFFFFFFu; u[4 * i + 1] = v.x & 0x7FFF0000u;
-            u[4 * i + 2] = (v.y << 16) & 0x7FFFFFFFu; u[4 * i + 3] = v.y & 0x7FFF0000u;
-        }
-        codes[b] = (uint32_t)exact_2_4(u, 16);
-    }
-}
+// every tier, for blocks given as magnitude patterns; drop_bits as for exact_2_4()
+static __device__ __noinline__ uint32_t exact_2_4_any(const uint32_t (&u)[16], int drop_bits) { return (uint32_t)exact_2_4(u, drop_bits); }
 
 // ------------------------------------------------------------------------------------------
 // Exact, any M <= 8: min-cost flow on the network of Fig. 3

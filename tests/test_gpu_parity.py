@@ -135,6 +135,27 @@ def test_exact_2_4_bf16_narrow_blocks_take_the_32_bit_scorer():
     assert_parity(B, 2, 4, tm.TM_EXACT)
 
 
+def test_exact_2_4_bf16_changes_tier_along_a_warps_items():
+    """The staged exact kernel starts a warp on the 32-bit scorer and moves it to the 64-bit one when its items leave the first
+    often: quantised rows (never leave it), then continuous rows (nearly every item does), with blocks that no in-loop tier
+    takes (subnormals beside large values, Inf) before and after the change -- those are scored after the loop; in place too."""
+    rows, cols = 4096, 8200                                       # about six items per warp, the last item of a row ragged
+    W = workloads.quantised_bf16(rows, cols, 0.02, 91)
+    W[:, 2048:] = workloads.normal_bf16(rows, cols - 2048, 0.02, 92)      # four quantised items, then thirteen continuous ones, per block row
+    W[8, 16] = 0x0001; W[9, 17] = 0x7F00; W[500, 5000] = 0x0002; W[501, 5001] = 0x7E80; W[4092, 8196] = 0x0003; W[4093, 8197] = 0x7F7F
+    W[700:704, 2048:2052] = 0; W[2000:2004, 4096:4608] = 0
+    assert_parity(W, 2, 4, tm.TM_EXACT)
+    V = W.copy(); V[600, 40] = 0x7F80; V[601, 41] = 0xFFC1
+    assert_parity(V, 2, 4, tm.TM_EXACT, rel=None)
+    want = orc.find_mask(W, 2, 4, orc.EXACT)
+    Wd = to_device(W)
+    mask, masked, obj = tm.tm_find_mask_bf16(Wd, 2, 4, tm.TM_EXACT, masked_w_out=Wd)        # in place
+    torch.cuda.synchronize()
+    assert np.array_equal(to_host_bits(Wd), want["masked"].view(np.uint16))
+    assert np.array_equal(to_host_bits(mask), want["mask"])
+    assert abs(float(obj.item()) - want["objective"]) <= 1e-6 * abs(want["objective"])
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_exact_2_4_on_the_bandwidth_kernel(dtype):
     """16-byte aligned matrices take the staged kernel for the exact 2:4 search too: several 512-column items and a ragged
