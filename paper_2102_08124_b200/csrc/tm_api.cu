@@ -18,8 +18,9 @@ constexpr int kPartialSlots = 8192;   // objective partials per matrix: (CTAs x 
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
 constexpr size_t kHeaderBytes = 256;  // reserved head of every workspace
-// Inside the header: the count of finished CTAs of a bandwidth launch that reduces its own objectives.  Only
-// workspaces whose header the library itself has cleared use it (every such launch leaves it at zero again).
+// Inside the header: the count of finished CTAs of a bandwidth launch that reduces its own objectives.  It is zero
+// between launches: cleared once where the library owns the workspace, at the start of the call where the caller does
+// (every such launch leaves it at zero again).
 constexpr size_t kDoneOffset = 128;
 // tm_find_mask_host(): row strips whose copy-in, search and copy-out overlap, and the head of its device workspace (status word,
 // then one objective per strip from byte 64 on)
@@ -123,7 +124,8 @@ int validate_call(const tm_problem* probs, int count, int N, int M, int method, 
     return TM_OK;
 }
 
-// header_clear: the workspace's header was zeroed by this library and nothing but its launches has touched it since.
+// header_clear: the count of finished CTAs in the workspace's header is zero when the launches start (cleared by this
+// library, which also keeps it so), so the bandwidth launches may reduce their own objectives.
 int build_plan(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes, const DeviceState& dev, Plan& plan,
                bool header_clear) {
     const int rc = validate_call(probs, count, N, M, method, ws, ws_bytes);
@@ -223,12 +225,22 @@ int launch_plan(const Plan& plan, int* status_dev, cudaStream_t stream) {
     return TM_OK;
 }
 
+// What is known of the workspace's header when a call starts: cleared by this library and untouched since; contents
+// unknown (the count of finished CTAs is cleared on the stream first -- four bytes instead of the objective partials, and no
+// reduction kernel); or left alone (the launches clear their partials and a reduction kernel follows them).
+enum HeaderState { kHeaderClear, kHeaderUnknown, kHeaderUnused };
+
 int run(const tm_problem* probs, int count, int N, int M, int method, void* ws, size_t ws_bytes, int* status_dev,
-        cudaStream_t stream, const DeviceState& dev, bool header_clear) {
+        cudaStream_t stream, const DeviceState& dev, HeaderState header) {
     Plan plan;
-    int rc = build_plan(probs, count, N, M, method, ws, ws_bytes, dev, plan, header_clear);
+    int rc = build_plan(probs, count, N, M, method, ws, ws_bytes, dev, plan, header != kHeaderUnused);
     if (rc != TM_OK) return rc;
     if ((rc = upload_plan(plan, stream)) != TM_OK) return rc;
+    if (header == kHeaderUnknown) {
+        bool wanted = false;
+        for (const PlanGroup& pg : plan.groups) wanted |= pg.tma && pg.bandwidth.done != nullptr;
+        if (wanted && cudaMemsetAsync(static_cast<char*>(ws) + kDoneOffset, 0, sizeof(unsigned int), stream) != cudaSuccess) { cudaGetLastError(); return TM_ERR_CUDA; }
+    }
     return launch_plan(plan, status_dev, stream);
 }
 
@@ -259,7 +271,7 @@ int plain_call(const void* W, int dtype, int64_t rows, int64_t cols, int N, int 
     if ((rc = current_device(&d)) != TM_OK) return rc;
     if ((rc = ensure_scratch(*d)) != TM_OK) return rc;
     void* scratch = d->scratch.load(std::memory_order_acquire);
-    return run(&p, 1, N, M, method, scratch, d->scratch_bytes, static_cast<int*>(scratch), nullptr, *d, true);
+    return run(&p, 1, N, M, method, scratch, d->scratch_bytes, static_cast<int*>(scratch), nullptr, *d, kHeaderClear);
 }
 
 int grow(void** p, size_t* have, size_t want) {
@@ -347,8 +359,7 @@ int tm_find_mask_batched(const tm_problem* probs_host, int count, int N, int M, 
     if (count == 0) return TM_OK;
     DeviceState* d = nullptr;
     if ((rc = current_device(&d)) != TM_OK) return rc;
-    // the caller's workspace arrives with unknown contents: partials cleared, search, reduction kernel
-    return run(probs_host, count, N, M, method, workspace_dev, workspace_bytes, status_dev, static_cast<cudaStream_t>(cuda_stream), *d, false);
+    return run(probs_host, count, N, M, method, workspace_dev, workspace_bytes, status_dev, static_cast<cudaStream_t>(cuda_stream), *d, kHeaderUnknown);
 }
 
 int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols, int N, int M, int method,
@@ -409,7 +420,7 @@ int tm_find_mask_host(const void* W_host, int dtype, int64_t rows, int64_t cols,
         p.mask_out = static_cast<uint32_t*>(d->stage_mask) + (size_t)r0 * wpr;
         p.masked_w_out = masked_w_out_host ? static_cast<char*>(d->stage_masked) + off : nullptr;
         p.objective_out = obj_dev + s;
-        rc = run(&p, 1, N, M, method, ws + kHostHead + (size_t)s * (one_ws + kAlign), one_ws, status_dev, d->s_run, *d, true);
+        rc = run(&p, 1, N, M, method, ws + kHostHead + (size_t)s * (one_ws + kAlign), one_ws, status_dev, d->s_run, *d, kHeaderClear);
         if (rc != TM_OK) { ok = false; break; }
         ok &= cudaEventRecord(ev_run[s], d->s_run) == cudaSuccess;
         ok &= cudaStreamWaitEvent(d->s_out, ev_run[s], 0) == cudaSuccess;
@@ -450,7 +461,7 @@ int tm_find_mask_batched_static(const tm_problem* probs_host, int count, int N, 
     void* scratch = nullptr;
     if ((rc = static_scratch_address(&scratch)) != TM_OK) return rc;
     // every launch below clears the objective partials it uses before its kernel runs on the same stream
-    return run(probs_host, count, N, M, method, scratch, TM_STATIC_SCRATCH_BYTES, status_dev, static_cast<cudaStream_t>(cuda_stream), *d, false);
+    return run(probs_host, count, N, M, method, scratch, TM_STATIC_SCRATCH_BYTES, status_dev, static_cast<cudaStream_t>(cuda_stream), *d, kHeaderUnused);
 }
 
 struct tm_plan { Plan plan; };
