@@ -1,5 +1,5 @@
 // Thin wrappers over the sm_100a bulk-tensor (TMA) copy and mbarrier instructions used by the
-// bandwidth kernels.  Loads never use cluster multicast; every wait is bounded.
+// bandwidth kernels.  Every load is a plain one-CTA copy; every wait is bounded.
 #pragma once
 #include <cstdint>
 #include <cuda.h>
