@@ -536,19 +536,22 @@ int tm_nm_mask_1d(const tm_problem* prob_host, int N, int M, int flags, unsigned
     char* base = static_cast<char*>(workspace_dev) + kHeaderBytes;
     double* op = reinterpret_cast<double*>(base);
     unsigned long long* vp = reinterpret_cast<unsigned long long*>(base + sizeof(double) * (size_t)tmask::aux_partial_slots());
-    // groups of four ride the bandwidth kernel of the 2:4 search (row rule instead of steps A-C)
-    if (M == 4 && N >= 1 && N <= 3 && p.rows > 0 && p.cols > 0) {
-        const DevProblem dp = to_dev(p, 4, 0);
-        if (tmask::tma_eligible(dp, N, 4, tmask::kMethodRows)) {
+    // groups of four and of eight ride the bandwidth kernels of the searches (row rule instead of steps A-C); the mean
+    // absorption only for groups of four
+    const bool absorb = (flags & TM_NM1D_ABSORB_MEAN) && p.masked_w_out != nullptr;
+    if (((M == 4 && N >= 1 && N <= 3) || (M == 8 && N >= 1 && N <= 7 && !absorb)) && p.rows > 0 && p.cols > 0) {
+        const DevProblem dp = to_dev(p, M, 0);
+        const int rows_method = absorb ? tmask::kMethodRowsAbsorb : tmask::kMethodRows;
+        if (tmask::tma_eligible(dp, N, M, rows_method)) {
             alignas(128) unsigned char entry[512];
             long long total = 0;
-            if (tmask::tma_entry_bytes() <= sizeof(entry) && tmask::tma_build_entries(&dp, 1, entry, &total, 4, tmask::kMethodRows)) {
+            if (tmask::tma_entry_bytes() <= sizeof(entry) && tmask::tma_build_entries(&dp, 1, entry, &total, M, rows_method)) {
                 tmask::TmaLaunch t;
                 t.entries_host = entry; t.entries_dev = nullptr; t.count = 1; t.total_items = total; t.partials = op; t.status = status_dev;
-                t.dtype = p.dtype; t.M = 4; t.has_out = p.masked_w_out != nullptr;
-                t.method = (flags & TM_NM1D_ABSORB_MEAN) && t.has_out ? tmask::kMethodRowsAbsorb : tmask::kMethodRows;
+                t.dtype = p.dtype; t.M = M; t.has_out = p.masked_w_out != nullptr;
+                t.method = rows_method;
                 t.stream = static_cast<cudaStream_t>(cuda_stream); t.n_keep = N; t.vpartials = vp;
-                const int wpc = tmask::tma_warps_per_cta(t.dtype, 4, t.method);
+                const int wpc = tmask::tma_warps_per_cta(t.dtype, M, t.method);
                 const long long want = (total + wpc - 1) / wpc;
                 const int cap = d->sms < tmask::aux_partial_slots() / wpc ? d->sms : tmask::aux_partial_slots() / wpc;
                 t.ctas = (int)(want < 1 ? 1 : (want > cap ? cap : want));

@@ -46,6 +46,8 @@ template <int K> TM_HD u64 rot_row8(u64 x) {
 // result bit (i,j) = x bit ((i+k) mod 8, j): the word rotated right by k bytes
 template <int K> TM_HD u64 rot_col8(u64 x) { return (x >> (8 * K)) | (x << (64 - 8 * K)); }
 
+// the row half of complete_relations8()
+TM_HD void complete_row_relations8(Rel48& r);
 // hr[1..3], hc[1..3] given in full, hr[4] for columns 0..3, hc[4] for rows 0..3: the rest by antisymmetry
 // (hr[8-k] bit (i, j+k) = not hr[k] bit (i, j)).
 TM_HD void complete_relations8(Rel48& r) {
@@ -55,10 +57,35 @@ TM_HD void complete_relations8(Rel48& r) {
     r.hc[7] = ~rot_col8<7>(r.hc[1]); r.hc[6] = ~rot_col8<6>(r.hc[2]); r.hc[5] = ~rot_col8<5>(r.hc[3]);
 }
 
+TM_HD void complete_row_relations8(Rel48& r) {
+    r.hr[4] = (r.hr[4] & 0x0F0F0F0F0F0F0F0Full) | ((~r.hr[4] << 4) & 0xF0F0F0F0F0F0F0F0ull);
+    r.hr[7] = ~rot_row8<7>(r.hr[1]); r.hr[6] = ~rot_row8<6>(r.hr[2]); r.hr[5] = ~rot_row8<5>(r.hr[3]);
+}
+
 // at least four of seven masks are set
 TM_HD u64 four_of_seven(u64 a, u64 b, u64 c, u64 d, u64 e, u64 f, u64 g) {
     const u64 s1 = a ^ b ^ c, k1 = maj3_64(a, b, c), s2 = d ^ e ^ f, k2 = maj3_64(d, e, f);
     return maj3_64(k1, k2, maj3_64(s1, s2, g));          // count = (s1 ^ s2 ^ g) + 2 * (k1 + k2 + k3)
+}
+
+// at least n of seven masks are set, n = 1..7 (the same n for every bit): the count bit-sliced as ones, twos, fours
+TM_HD u64 at_least_of_seven(u64 a, u64 b, u64 c, u64 d, u64 e, u64 f, u64 g, int n) {
+    const u64 s1 = a ^ b ^ c, k1 = maj3_64(a, b, c), s2 = d ^ e ^ f, k2 = maj3_64(d, e, f);
+    const u64 ones = s1 ^ s2 ^ g, k3 = maj3_64(s1, s2, g);
+    const u64 twos = k1 ^ k2 ^ k3, fours = maj3_64(k1, k2, k3);
+    switch (n) {
+        case 1: return ones | twos | fours;
+        case 2: return twos | fours;
+        case 3: return fours | (twos & ones);
+        case 4: return fours;
+        case 5: return fours & (twos | ones);
+        case 6: return fours & twos;
+        default: return fours & twos & ones;
+    }
+}
+// 1-D N:M along rows (no column constraint): kept iff fewer than n_keep entries of the row are heavier; n_keep = 1..7
+TM_HD u64 keep_rows_8(const Rel48& r, int n_keep) {
+    return ~at_least_of_seven(r.hr[1], r.hr[2], r.hr[3], r.hr[4], r.hr[5], r.hr[6], r.hr[7], n_keep);
 }
 
 // Step A.

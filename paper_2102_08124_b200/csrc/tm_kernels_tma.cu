@@ -698,7 +698,10 @@ int tma_warps_per_cta(int dtype, int M, int method) {
 }
 
 bool tma_eligible(const DevProblem& p, int N, int M, int method) {
-    if (method == kMethodRows || method == kMethodRowsAbsorb) { if (M != 4 || N < 1 || N > 3) return false; }
+    if (method == kMethodRows || method == kMethodRowsAbsorb) {
+        // groups of four with or without the mean absorption, groups of eight without
+        if (!((M == 4 && N >= 1 && N <= 3) || (M == 8 && N >= 1 && N <= 7 && method == kMethodRows))) return false;
+    }
     else if (method == kMethodExact) { if (N != 2 || M != 4) return false; }
     else if (!((N == 2 && M == 4) || (N == 4 && M == 8)) || (method != kMethodApprox && method != kMethodCover)) return false;
     const size_t elem = p.dtype == kF32 ? 4 : 2;

@@ -123,6 +123,22 @@ __device__ __forceinline__ void relations48_bf16(const uint32_t (&R)[8][4], Rel4
     complete_relations8(rel);
 }
 
+// The row relations alone (1-D pruning along rows needs no column relation)
+template <bool ARITH>
+__device__ __forceinline__ void row_relations48_bf16(const uint32_t (&R)[8][4], Rel48& rel) {
+    uint32_t Y[4][8];
+#pragma unroll
+    for (int ip = 0; ip < 4; ++ip)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            Y[ip][2 * c] = prmt(R[2 * ip][c], R[2 * ip + 1][c], 0x5410);
+            Y[ip][2 * c + 1] = prmt(R[2 * ip][c], R[2 * ip + 1][c], 0x7632);
+        }
+    rel.hr[1] = row_relation<ARITH, 1>(Y); rel.hr[2] = row_relation<ARITH, 2>(Y);
+    rel.hr[3] = row_relation<ARITH, 3>(Y); rel.hr[4] = row_relation<ARITH, 4>(Y);
+    complete_row_relations8(rel);
+}
+
 // ---- fp32: scalar comparisons ------------------------------------------------------------------
 __device__ __forceinline__ void relations48_f32(const unsigned char* blk, Rel48& rel, uint32_t& worst) {
     uint32_t u[64];
@@ -213,6 +229,33 @@ __device__ __forceinline__ void relations48_f32_arith(const float (&f)[64], Rel4
     complete_relations8(rel);
 }
 
+// The row relations alone, finite fp32 data (see relations48_f32_arith)
+__device__ __forceinline__ void row_relations48_f32_arith(const float (&f)[64], Rel48& rel) {
+#pragma unroll
+    for (int k = 1; k <= 4; ++k) {
+        uint32_t rw[2];
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            uint32_t acc = 0;
+#pragma unroll
+            for (int r = 3; r >= 0; --r) {
+                const int i = 4 * w + r;
+                if (k == 4 && r != 3) acc <<= 4;
+#pragma unroll
+                for (int j = (k == 4 ? 3 : 7); j >= 0; --j) {
+                    const int jj = (j + k) & 7;
+                    const float a = fabsf(f[8 * i + jj]), b = fabsf(f[8 * i + j]);
+                    acc = push_sign(acc, (j + k <= 7) ? a - b : b - a);
+                }
+            }
+            const uint32_t later = k == 4 ? 0x0F0F0F0Fu : 0x01010101u * ((1u << (8 - k)) - 1u);
+            rw[w] = acc ^ later;
+        }
+        rel.hr[k] = (u64)rw[0] | ((u64)rw[1] << 32);
+    }
+    complete_row_relations8(rel);
+}
+
 // magnitude pattern of entry p of the lane's block, read back from the stage
 template <int DT>
 __device__ __forceinline__ uint32_t key_at(const unsigned char* blk, int p) {
@@ -297,8 +340,10 @@ __device__ __forceinline__ float back_end48(unsigned char* blk, unsigned char* m
 template <int DT, int METHOD, bool HAS_OUT>
 __global__ void __launch_bounds__(Geo48<DT, METHOD>::kWarps * 32, 1)
 tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict__ table, int count, long long total_items,
-             double* __restrict__ partials, int* __restrict__ status_out, unsigned int* __restrict__ done) {
+             double* __restrict__ partials, int* __restrict__ status_out, unsigned int* __restrict__ done, int n_keep,
+             unsigned long long* __restrict__ vpartials) {
     using G = Geo48<DT, METHOD>;
+    constexpr bool kRows = METHOD == kMethodRows;        // 1-D n_keep of 8 along rows: row relations only, no steps A to C
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned char* stages = smem_raw + (size_t)warp * G::kWarpBytes;
@@ -352,8 +397,10 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
     float facc = 0.f; double acc = 0.0;
     uint32_t worst = 0;
     // the matrix in process: the fields every item needs
-    int p_cols = 0, p_wpr = 0;
+    int p_cols = 0, p_wpr = 0, p_rows = 0;
     uint32_t* p_mask = nullptr;
+    unsigned long long viol = 0;                         // kRows: non-zero entries pruned by this lane
+    u64 nonzero = 0;
 
     for (int it = 0; it < n_items; ++it) {
         const int s = it % G::kStages;
@@ -382,9 +429,20 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
                     const uint4 v = *reinterpret_cast<const uint4*>(blk + i * 512);
                     R[i][0] = v.x & 0x7FFF7FFFu; R[i][1] = v.y & 0x7FFF7FFFu; R[i][2] = v.z & 0x7FFF7FFFu; R[i][3] = v.w & 0x7FFF7FFFu;
                 }
-                relations48_bf16<false>(R, rel);
+                if constexpr (kRows) row_relations48_bf16<false>(R, rel); else relations48_bf16<false>(R, rel);
             } else {
-                relations48_bf16<true>(R, rel);
+                if constexpr (kRows) row_relations48_bf16<true>(R, rel); else relations48_bf16<true>(R, rel);
+            }
+            if constexpr (kRows) {                       // x + 0x7FFF sets the top bit of a 15-bit magnitude iff x != 0
+                uint32_t nz[2] = {0, 0};
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t t = (R[i][c] & 0x7FFF7FFFu) + 0x7FFF7FFFu;
+                        nz[i >> 2] |= (((t >> 15) & 1u) | ((t >> 30) & 2u)) << (8 * (i & 3) + 2 * c);
+                    }
+                nonzero = (u64)nz[0] | ((u64)nz[1] << 32);
             }
         } else {
             float f[64];
@@ -399,7 +457,14 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
 #pragma unroll
             for (int p = 0; p < 64; ++p) watch = fmaf(f[p], 0.f, watch);
             if (__any_sync(0xFFFFFFFFu, watch != watch)) relations48_f32(blk, rel, worst);       // integer keys, bit-pattern order
+            else if constexpr (kRows) row_relations48_f32_arith(f, rel);
             else relations48_f32_arith(f, rel);
+            if constexpr (kRows) {
+                uint32_t nz[2] = {0, 0};
+#pragma unroll
+                for (int p = 0; p < 64; ++p) nz[p >> 5] |= ((__float_as_uint(f[p]) & 0x7FFFFFFFu) ? 1u : 0u) << (p & 31);
+                nonzero = (u64)nz[0] | ((u64)nz[1] << 32);
+            }
         }
         // refill the stage of the previous item -- its store, issued one item ago, has long been read -- so that the copy
         // runs under the rest of this item
@@ -408,7 +473,7 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             __syncwarp();
             issue_next();
         }
-        u64 kept = cover_4_8(rel);
+        u64 kept = kRows ? keep_rows_8(rel, n_keep) : cover_4_8(rel);
         if constexpr (METHOD == kMethodApprox) {
             Short48 L = line_short(kept);
             u64 cand = open_candidates8(kept, L);
@@ -453,9 +518,14 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
             }
             acc = 0.0; facc = 0.f; acc_k = cur.k;
             const DevProblem& P = tab[cur.k].p;
-            p_cols = (int)P.cols; p_wpr = P.wpr; p_mask = P.mask;
+            p_cols = (int)P.cols; p_wpr = P.wpr; p_mask = P.mask; p_rows = (int)P.rows;
         }
         if (cur.cj * kCols8 + lane * 8 >= p_cols) kept = 0;               // blocks past the last column (zero-filled by the copy)
+        if constexpr (kRows) {
+            // pruned non-zero entries; rows past the last one (the 1-D pruning takes any number of rows) and blocks past the
+            // last column were zero-filled by the copy and count nothing
+            if (cur.cj * kCols8 + lane * 8 < p_cols) viol += (unsigned)__popcll(~kept & nonzero);
+        }
         facc += back_end48<DT, HAS_OUT>(blk, mbytes, lut, lane, kept);
         if constexpr (HAS_OUT) fence_proxy_async_smem();
         __syncwarp();
@@ -466,7 +536,7 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         for (int h = 0; h < 2; ++h) {                                      // 8 rows x 8 words of mask
             const int idx = lane + 32 * h, row = idx >> 3, word = cur.cj * 8 + (idx & 7);
             const uint32_t w = *reinterpret_cast<const uint32_t*>(mbytes + row * 32 + (idx & 7) * 4);
-            if (word < p_wpr) p_mask[((long long)cur.bi * kRows8 + row) * p_wpr + word] = w;
+            if (word < p_wpr && (!kRows || cur.bi * kRows8 + row < p_rows)) p_mask[((long long)cur.bi * kRows8 + row) * p_wpr + word] = w;
         }
         cur.advance(tab, count);
         if ((it & 15) == 15) { acc += (double)facc; facc = 0.f; }           // keep the fp32 partial short
@@ -487,6 +557,10 @@ tma48_kernel(const __grid_constant__ TmaEntry single, const TmaEntry* __restrict
         if (count > 1) finish_objectives_ranged(done, partials, tab, count, total_items, nw, reinterpret_cast<double*>(smem_raw));
         else finish_objective(done, partials, nw, tab[0].p.objective, reinterpret_cast<double*>(smem_raw));
     }
+    if constexpr (kRows) {
+        for (int o = 16; o; o >>= 1) viol += __shfl_xor_sync(0xFFFFFFFFu, viol, o);
+        if (lane == 0 && vpartials) vpartials[gw] = viol;
+    }
 }
 
 template <int DT, int METHOD, bool HAS_OUT>
@@ -497,7 +571,7 @@ cudaError_t launch_one48(const TmaLaunch& a, const TmaEntry& single, const TmaEn
     static PerDeviceOnce configured;       // per instantiation
     const cudaError_t e = configured.run([&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });
     if (e != cudaSuccess) return e;
-    kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status, a.done);
+    kern<<<a.ctas, G::kWarps * 32, smem, a.stream>>>(single, table, a.count, a.total_items, a.partials, a.status, a.done, a.n_keep, a.vpartials);
     return cudaGetLastError();
 }
 
@@ -525,12 +599,13 @@ cudaError_t launch_tma48(const TmaLaunch& a) {
 #define TM_DISPATCH(DT, METHOD)                                                                                   \
     err = a.has_out ? launch_one48<DT, METHOD, true>(a, host[0], table) : launch_one48<DT, METHOD, false>(a, host[0], table)
         if (takes_split_kernel(a.dtype, a.method)) err = launch_tma48s(a);
-        else if (a.dtype == kF32) TM_DISPATCH(kF32, kMethodCover);
-        else { if (a.method == kMethodApprox) TM_DISPATCH(kBF16, kMethodApprox); else TM_DISPATCH(kBF16, kMethodCover); }
+        else if (a.dtype == kF32) { if (a.method == kMethodRows) TM_DISPATCH(kF32, kMethodRows); else TM_DISPATCH(kF32, kMethodCover); }
+        else { if (a.method == kMethodApprox) TM_DISPATCH(kBF16, kMethodApprox); else if (a.method == kMethodRows) TM_DISPATCH(kBF16, kMethodRows); else TM_DISPATCH(kBF16, kMethodCover); }
 #undef TM_DISPATCH
         if (err != cudaSuccess) return err;
     }
     if (a.done) return cudaSuccess;
+    if (a.method == kMethodRows) return cudaSuccess;          // the caller sums objective and violation partials together
     return tma_reduce(a.entries_host, a.entries_dev, a.count, a.partials, (long long)a.ctas * wpc, a.stream);
 }
 

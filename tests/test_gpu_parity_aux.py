@@ -40,10 +40,10 @@ def test_nm_1d(dtype, N, M, absorb):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("N", [1, 2, 3])
-def test_nm_1d_groups_of_four_edge_values(dtype, N):
-    """Shapes the bandwidth kernel takes (16-byte aligned rows): zeros of both signs, subnormals, equal magnitudes,
-    an odd number of rows, several column chunks; then Inf and NaN, which must be ordered by bit pattern and flagged."""
+@pytest.mark.parametrize("N,M", [(1, 4), (2, 4), (3, 4), (1, 8), (3, 8), (4, 8), (5, 8), (7, 8)])
+def test_nm_1d_groups_on_the_bandwidth_kernels_edge_values(dtype, N, M):
+    """Shapes the bandwidth kernels take (16-byte aligned rows), groups of four and of eight: zeros of both signs, subnormals,
+    equal magnitudes, an odd number of rows, several column chunks; then Inf and NaN, which must be ordered by bit pattern and flagged."""
     rows, cols = 13, 776
     rng = np.random.Generator(np.random.PCG64(50 + N))
     W = workloads.normal_f32(rows, cols, 0.02, 51)
@@ -59,8 +59,8 @@ def test_nm_1d_groups_of_four_edge_values(dtype, N):
                 W[2, 5] = 0x7F80; W[3, 300] = 0xFFC1; W[3, 301] = 0x7FC0; W[12, 775] = 0xFF80
             else:
                 W[2, 5] = np.inf; W[3, 300] = np.nan; W[3, 301] = -np.nan; W[12, 775] = -np.inf
-        want = orc.nm_mask_1d(W, N, 4)
-        mask, masked, obj, viol, status = tm.tm_nm_mask_1d(to_device(W), N, 4)
+        want = orc.nm_mask_1d(W, N, M)
+        mask, masked, obj, viol, status = tm.tm_nm_mask_1d(to_device(W), N, M)
         torch.cuda.synchronize()
         assert int(status.item()) == (tm.TM_DEV_NONFINITE if nonfinite else 0)
         assert np.array_equal(to_host_bits(mask), want["mask"])
